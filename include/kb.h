@@ -1,0 +1,200 @@
+/*
+ * kb.h -- C ABI of the candidate screen, timing adjudication and survivor
+ * selection used inside a multi-fidelity kernel-search evaluation loop
+ * (KernelBrain, arxiv 2608.02611).
+ *
+ * The library covers the data-parallel interior of the paper's Evaluation
+ * Plane (Sec. 3.4) and of the scheduler's promote/prune step:
+ *
+ *   kb_screen      the Verifier's "output correctness against the reference"
+ *                  check (Sec. 3.4, Evaluation Plane; the correctness
+ *                  indicator K(p) of Sec. 3.1), for K candidates at once,
+ *                  optionally on a fidelity-dependent subset of tiles
+ *                  (low-cost screening, Abstract / Sec. 3.3 Observation 2);
+ *   kb_adjudicate  the reduction of repeated, noisy timings to an
+ *                  "adjudicated latency" (Algorithm 1, "Compute score s(c,r)
+ *                  from adjudicated latency"; Sec. 1 contribution 1
+ *                  "stability adjudication"; Appendix "Relative Variability
+ *                  Metrics"), as median + IQR per candidate plus a K x K
+ *                  matrix of doubled Mann-Whitney win counts;
+ *   kb_select      the promotion decision D (Sec. 3.2 "Promotion decision",
+ *                  Sec. 3.4 "Adaptive Resource Allocation": rank with
+ *                  deterministic tie-breaking, promote the top part).
+ *
+ * Conventions (all entry points)
+ *   - Plain C99 types only.  Every pointer is marked HOST or DEVICE below.
+ *   - Ownership: the caller owns every input and output buffer.  The library
+ *     owns kb_ctx (a device workspace that grows on demand with cudaMalloc
+ *     and is released by kb_ctx_destroy) and kb_mask.
+ *   - Asynchrony: kb_screen / kb_adjudicate / kb_select enqueue work on
+ *     `stream` (a cudaStream_t passed as void*; NULL = the default stream) and
+ *     return without synchronising.  Outputs are valid once the stream has
+ *     been synchronised.  Host arrays passed in (h_cands) are consumed before
+ *     the call returns.  One kb_ctx must not be used from two streams or two
+ *     host threads at the same time.
+ *   - Errors: a kb_status is returned; nothing aborts or throws.  Argument
+ *     errors are detected before any launch and leave the outputs untouched.
+ *     Conditions only the device can see (a non-finite timing, a bounded wait
+ *     that ran out) are recorded in a ctx-owned device status word that
+ *     kb_ctx_poll reads back.
+ *   - Determinism: every output is a pure function of the inputs; it does not
+ *     depend on grid size, scheduling or call history.
+ *   - Arithmetic: IEEE-754 binary32, round-to-nearest-even, no fused
+ *     multiply-add, subnormals honoured.
+ */
+#ifndef KB_H_
+#define KB_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  KB_OK = 0,
+  KB_ERR_INVALID_ARG = 1,   /* null pointer, zero size, out-of-range value        */
+  KB_ERR_ALIGNMENT = 2,     /* a tensor pointer is not 16-byte aligned            */
+  KB_ERR_UNSUPPORTED = 3,   /* unknown dtype / policy                             */
+  KB_ERR_WORKSPACE = 4,     /* the device workspace could not be grown            */
+  KB_ERR_CUDA = 5,          /* a CUDA runtime call failed (see kb_last_error)     */
+  KB_ERR_NONFINITE = 6,     /* device status: a timing was NaN or +-Inf           */
+  KB_ERR_DEVICE_TIMEOUT = 7 /* device status: a bounded device-side wait ran out  */
+} kb_status;
+
+typedef enum { KB_F32 = 0, KB_F16 = 1, KB_BF16 = 2 } kb_dtype;
+
+/* One record per candidate; 48 bytes, 8-byte aligned.
+ * With r = ref[i], c = cand[i] decoded exactly to binary32 and, over the
+ * selected elements i in ascending order,
+ *     d     = |c - r|                       (one rounding)
+ *     tol   = atol + (rtol * |r|)           (product rounded, then sum rounded)
+ *     match = (c == r) || (isfinite(d) && d <= tol)      (NaN never matches)
+ * the fields are: */
+typedef struct {
+  uint64_t mismatch_count; /* selected elements with match == false                 */
+  uint64_t nan_count;      /* selected elements whose CANDIDATE value is NaN        */
+  uint64_t inf_count;      /* selected elements whose CANDIDATE value is +-Inf      */
+  int64_t argmax_idx;      /* flat index in the FULL tensor of max_abs_err, lowest
+                              index on ties; -1 if no selected element has finite d */
+  float max_abs_err;       /* max of d over selected elements with finite d; 0 if none */
+  float max_rel_err;       /* max of d/|r| (correctly rounded) over selected elements
+                              with finite d and r != 0; 0 if none; may be +Inf      */
+  uint32_t pass;           /* 1 iff mismatch_count == 0                             */
+  uint32_t reserved;       /* 0                                                     */
+} kb_screen_result;
+
+typedef struct kb_ctx kb_ctx;   /* device workspace + status word; bound to one device */
+typedef struct kb_mask kb_mask; /* immutable fidelity mask; owns a device tile list    */
+
+/* Limits checked at the boundary. */
+#define KB_MAX_K 65535u         /* candidates per call                               */
+#define KB_MAX_N 4294967296ull  /* elements per tensor (2^32)                        */
+#define KB_MAX_S 32768u         /* timings per candidate (2*S*S must fit uint32)     */
+
+/* ---- context ----------------------------------------------------------- */
+
+/* Create a context on CUDA device `device`.  HOST out pointer. */
+kb_status kb_ctx_create(int device, kb_ctx** out);
+/* Synchronises the device, frees the workspace.  NULL is accepted. */
+kb_status kb_ctx_destroy(kb_ctx* ctx);
+/* Text of the last error recorded on this context (ctx-owned, valid until the
+ * next call on the context); with ctx == NULL, the text of the last failed
+ * kb_ctx_create on this thread. */
+const char* kb_last_error(const kb_ctx* ctx);
+/* Synchronise `stream`, read the device status word into *device_status
+ * (KB_OK, KB_ERR_NONFINITE or KB_ERR_DEVICE_TIMEOUT; HOST pointer) and clear
+ * it.  Returns KB_OK unless the read itself failed. */
+kb_status kb_ctx_poll(kb_ctx* ctx, void* stream, kb_status* device_status);
+/* Test/tuning hook: force the number of thread blocks of the streaming screen
+ * kernel (0 = automatic).  Results do not depend on it. */
+kb_status kb_ctx_set_grid(kb_ctx* ctx, uint32_t blocks);
+
+/* ---- fidelity masks (Sec. 3.2 "Fidelity level", rendered on elements) --- */
+
+/* A mask selects whole tiles of 2^log2_tile consecutive elements: element i is
+ * selected iff tile (i >> log2_tile) is selected; the last tile may be
+ * partial.  log2_tile <= 31.  Tiles of >= 4096 elements let a lower tier skip
+ * DRAM traffic; smaller tiles are legal but every sector is still fetched. */
+
+/* Strided mask: tile t selected iff (t % stride) == phase; stride >= 1,
+ * phase < stride. */
+kb_status kb_mask_create_strided(kb_ctx* ctx, uint64_t N, uint32_t log2_tile, uint32_t stride,
+                                 uint32_t phase, kb_mask** out);
+/* Bitmap mask: tile t selected iff bit (t & 63) of host_bits[t >> 6] is set.
+ * HOST pointer to ceil(ntiles/64) words, consumed before return. */
+kb_status kb_mask_create_bitmap(kb_ctx* ctx, uint64_t N, uint32_t log2_tile,
+                                const uint64_t* host_bits, kb_mask** out);
+/* Number of selected elements (HOST out). */
+kb_status kb_mask_count(const kb_mask* mask, uint64_t* n_selected);
+kb_status kb_mask_destroy(kb_mask* mask);
+
+/* ---- correctness gate (Sec. 3.1 K(p); Sec. 3.2 policy check, output-shape
+ *      and dtype constraints; Sec. 3.4 Verifier) --------------------------- */
+
+/* Compare K candidates with one reference.
+ *   d_ref    DEVICE, N elements of `dtype`, 16-byte aligned.
+ *   h_cands  HOST array of K DEVICE pointers, each N elements of `dtype`,
+ *            16-byte aligned.  All tensors share one dtype and one N: that is
+ *            the shape/dtype part of the policy check.
+ *   atol, rtol  finite and >= 0.
+ *   mask     NULL = every element; else a mask created for the same N.
+ *   d_out    DEVICE, K records, 8-byte aligned; fully overwritten.
+ * 1 <= K <= KB_MAX_K, 1 <= N <= KB_MAX_N. */
+kb_status kb_screen(kb_ctx* ctx, const void* d_ref, const void* const* h_cands, uint32_t K,
+                    uint64_t N, kb_dtype dtype, float atol, float rtol, const kb_mask* mask,
+                    kb_screen_result* d_out, void* stream);
+
+/* Same operation with every tensor in HOST memory (pinned memory gives the
+ * best transfer rate; pageable works).  The reference and the candidates are
+ * copied to ctx-owned device staging in batches of candidates so that copies
+ * overlap the kernel, and the K records are copied back to h_out (HOST).
+ * Synchronous: returns when h_out is complete.  `stream` orders the work. */
+kb_status kb_screen_host(kb_ctx* ctx, const void* h_ref, const void* const* h_cands_host,
+                         uint32_t K, uint64_t N, kb_dtype dtype, float atol, float rtol,
+                         const kb_mask* mask, kb_screen_result* h_out, void* stream);
+
+/* ---- stability adjudication (Algorithm 1 "adjudicated latency"; Sec. 1
+ *      contribution 1; Appendix "Relative Variability Metrics") ------------ */
+
+/* d_timings  DEVICE, [K][S] row-major binary32 milliseconds, all finite
+ *            (otherwise the device status becomes KB_ERR_NONFINITE and the
+ *            outputs are unspecified).
+ * d_median   DEVICE [K]: type-7 (linear) quantile at 1/2 of the sorted row:
+ *            pos = j*(S-1), lo = pos/4, rem = pos%4, hi = min(lo+1, S-1),
+ *            Q_j = x_lo if rem == 0 else x_lo + ((rem*0.25f) * (x_hi - x_lo)),
+ *            each operation rounded.  median = Q_2.
+ * d_iqr      DEVICE [K]: Q_3 - Q_1 (rounded).
+ * d_wins     DEVICE [K][K] row-major uint32:
+ *            W[a][b] = sum_i sum_j ( 2*[t_a,i < t_b,j] + [t_a,i == t_b,j] ),
+ *            i.e. twice the Mann-Whitney U of "a faster than b" with ties
+ *            counted once; W[a][b] + W[b][a] = 2*S*S and W[a][a] = S*S.
+ * Any of the three outputs may be NULL to skip it.
+ * 1 <= K <= KB_MAX_K, 1 <= S <= KB_MAX_S. */
+kb_status kb_adjudicate(kb_ctx* ctx, const float* d_timings, uint32_t K, uint32_t S,
+                        float* d_median, float* d_iqr, uint32_t* d_wins, void* stream);
+
+/* ---- promotion decision (Sec. 3.2; Sec. 3.4 scheduler; Algorithm 1, D) --- */
+
+typedef enum {
+  KB_SELECT_ERR_THEN_TIME = 0, /* key (max_rel_err asc, median asc, index asc) */
+  KB_SELECT_TIME = 1           /* key (median asc, index asc)                   */
+} kb_select_policy;
+
+/* Eligible candidates are those with pass == 1 (failed candidates are never
+ * promoted).  They are ordered by the policy's key, floats compared as values
+ * (none is NaN), ties broken by the lower candidate index; the first
+ * n = min(budget, #eligible) indices are written to d_survivors IN RANK ORDER
+ * and n to *d_n_survivors.  Entries d_survivors[n..budget) are set to -1.
+ *   d_screen     DEVICE [K] records from kb_screen.
+ *   d_median     DEVICE [K] from kb_adjudicate.
+ *   d_survivors  DEVICE [budget] int32.   d_n_survivors  DEVICE uint32.
+ * 1 <= K <= KB_MAX_K, budget >= 1. */
+kb_status kb_select(kb_ctx* ctx, const kb_screen_result* d_screen, const float* d_median,
+                    uint32_t K, kb_select_policy policy, uint32_t budget, int32_t* d_survivors,
+                    uint32_t* d_n_survivors, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KB_H_ */

@@ -1,0 +1,341 @@
+/*
+ * kb_oracle.c -- plain CPU oracle for the candidate screen, the timing
+ * adjudication and the survivor selection.
+ *
+ * THIS IS TEST INFRASTRUCTURE.  It exists so that the CUDA library can be
+ * checked element by element against something slow and obviously correct.
+ * It shares no code, header, table or helper with the CUDA path and is never
+ * linked into, imported by or called from the product.
+ *
+ * Everything is the definition written out: one loop per definition, in the
+ * order the definition states, no blocking, no fusion, no reordering.
+ * All floating point is IEEE-754 binary32, round-to-nearest-even.  Build with
+ *     gcc -O2 -std=c99 -ffp-contract=off -fPIC -shared
+ * (no -ffast-math, no FTZ/DAZ) so that no multiply-add is fused and
+ * subnormals are honoured.
+ *
+ * What the paper fixes and what is a reading of it:
+ *   - The gate is the Verifier's "checks output correctness against the
+ *     reference" (Sec. 3.4, Evaluation Plane) = the correctness indicator
+ *     K(p) "passes task and numerical tests" (Sec. 3.1).  The paper prints no
+ *     tolerance formula; the reading used here is the asymmetric
+ *     |c - r| <= atol + rtol*|r| test, NaN never matching (see kbo_screen).
+ *   - "Adjudicated latency" (Algorithm 1) is read as the median of the
+ *     repeated timings, reported with the inter-quartile range; ranking under
+ *     noise (Appendix, Relative Variability Metrics) is supported by pairwise
+ *     doubled Mann-Whitney win counts (see kbo_quantiles, kbo_wins).
+ *   - The promotion decision (Sec. 3.2; Sec. 3.4 "ranks candidates ... with
+ *     deterministic tie-breaking ... promotes the top fraction") is
+ *     kbo_select.
+ *
+ * Pins: every function here is pinned by the CPU tests (worked examples
+ * stored under tests/golden, numpy/scipy special cases, brute force over small
+ * alphabets, invariants).  Nothing in this file is "parity unpinned".
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+/* dtype codes of this oracle's own interface */
+enum { KBO_F32 = 0, KBO_F16 = 1, KBO_BF16 = 2 };
+
+/* mask kinds */
+enum { KBO_MASK_NONE = 0, KBO_MASK_STRIDED = 1, KBO_MASK_BITMAP = 2 };
+
+typedef struct {
+  uint64_t mismatch_count;
+  uint64_t nan_count;
+  uint64_t inf_count;
+  int64_t argmax_idx;
+  float max_abs_err;
+  float max_rel_err;
+  uint32_t pass;
+  uint32_t reserved;
+} kbo_screen_result;
+
+static float bits_to_float(uint32_t u) {
+  float f;
+  memcpy(&f, &u, sizeof f);
+  return f;
+}
+
+static uint32_t float_to_bits(float f) {
+  uint32_t u;
+  memcpy(&u, &f, sizeof u);
+  return u;
+}
+
+/* Classification by bit pattern, so that no compiler flag can change it. */
+static int is_nan32(float f) {
+  uint32_t u = float_to_bits(f) & 0x7FFFFFFFu;
+  return u > 0x7F800000u;
+}
+static int is_inf32(float f) {
+  uint32_t u = float_to_bits(f) & 0x7FFFFFFFu;
+  return u == 0x7F800000u;
+}
+static int is_finite32(float f) {
+  uint32_t u = float_to_bits(f) & 0x7FFFFFFFu;
+  return u < 0x7F800000u;
+}
+
+/* binary16 -> binary32, exact (every binary16 value is a binary32 value). */
+float kbo_decode_f16(uint16_t h) {
+  uint32_t sign = (uint32_t)(h >> 15) & 1u;
+  uint32_t expo = (uint32_t)(h >> 10) & 0x1Fu;
+  uint32_t frac = (uint32_t)h & 0x3FFu;
+  float mag;
+  if (expo == 0x1Fu) {
+    /* Inf or NaN: keep the payload in the top fraction bits */
+    return bits_to_float((sign << 31) | 0x7F800000u | (frac << 13));
+  }
+  if (expo == 0) {
+    /* zero or subnormal: frac * 2^-24, exact */
+    mag = ldexpf((float)frac, -24);
+  } else {
+    /* normal: (1024 + frac) * 2^(expo - 25), exact */
+    mag = ldexpf((float)(1024u + frac), (int)expo - 25);
+  }
+  return sign ? -mag : mag;
+}
+
+/* bfloat16 -> binary32: the 16 bits are the top half of the binary32 word. */
+float kbo_decode_bf16(uint16_t b) { return bits_to_float((uint32_t)b << 16); }
+
+static float load_as_f32(const void* base, uint64_t i, int dtype) {
+  if (dtype == KBO_F32) return ((const float*)base)[i];
+  if (dtype == KBO_F16) return kbo_decode_f16(((const uint16_t*)base)[i]);
+  return kbo_decode_bf16(((const uint16_t*)base)[i]);
+}
+
+/* Is element i selected by the fidelity mask?  A mask selects whole tiles of
+ * 2^log2_tile consecutive elements. */
+static int selected(uint64_t i, int mask_kind, uint32_t log2_tile, uint32_t stride, uint32_t phase,
+                    const uint64_t* bits) {
+  uint64_t tile;
+  if (mask_kind == KBO_MASK_NONE) return 1;
+  tile = i >> log2_tile;
+  if (mask_kind == KBO_MASK_STRIDED) return (tile % stride) == phase;
+  return (int)((bits[tile >> 6] >> (tile & 63u)) & 1u);
+}
+
+/*
+ * The correctness gate for ONE candidate (Sec. 3.1 K(p); Sec. 3.4 Verifier).
+ * For every selected element i, ascending:
+ *   1. d = |c - r|
+ *   2. tol = atol + (rtol * |r|)            product rounded, then sum rounded
+ *   3. match = (c == r) || (isfinite(d) && d <= tol)
+ *   4. counts of mismatches, of NaN candidates, of +-Inf candidates
+ *   5. max_abs_err / argmax over finite d, first index wins ties, the first
+ *      finite-d element initialises with its own d
+ *   6. max_rel_err = max d/|r| over finite d and r != 0, starting from 0
+ *   7. pass = no mismatch
+ * Returns 0, or -1 on a bad argument.
+ */
+int kbo_screen(const void* ref, const void* cand, uint64_t N, int dtype, float atol, float rtol,
+               int mask_kind, uint32_t log2_tile, uint32_t stride, uint32_t phase,
+               const uint64_t* bits, kbo_screen_result* out) {
+  uint64_t i;
+  uint64_t mism = 0, nans = 0, infs = 0;
+  int have_abs = 0;
+  float max_abs = 0.0f, max_rel = 0.0f;
+  int64_t argmax = -1;
+  if (!ref || !cand || !out || N == 0) return -1;
+  if (dtype != KBO_F32 && dtype != KBO_F16 && dtype != KBO_BF16) return -1;
+  if (mask_kind == KBO_MASK_STRIDED && (stride == 0 || phase >= stride)) return -1;
+  if (mask_kind == KBO_MASK_BITMAP && !bits) return -1;
+
+  for (i = 0; i < N; ++i) {
+    float r, c, d, prod, tol;
+    int match;
+    if (!selected(i, mask_kind, log2_tile, stride, phase, bits)) continue;
+    r = load_as_f32(ref, i, dtype);
+    c = load_as_f32(cand, i, dtype);
+    d = fabsf(c - r);
+    prod = rtol * fabsf(r);
+    tol = atol + prod;
+    match = (c == r) || (is_finite32(d) && d <= tol);
+    if (!match) ++mism;
+    if (is_nan32(c)) ++nans;
+    if (is_inf32(c)) ++infs;
+    if (is_finite32(d)) {
+      if (!have_abs || d > max_abs) {
+        max_abs = d;
+        argmax = (int64_t)i;
+        have_abs = 1;
+      }
+      if (r != 0.0f) {
+        float q = d / fabsf(r);
+        if (q > max_rel) max_rel = q;
+      }
+    }
+  }
+  out->mismatch_count = mism;
+  out->nan_count = nans;
+  out->inf_count = infs;
+  out->argmax_idx = have_abs ? argmax : -1;
+  out->max_abs_err = have_abs ? max_abs : 0.0f;
+  out->max_rel_err = max_rel;
+  out->pass = (mism == 0) ? 1u : 0u;
+  out->reserved = 0;
+  return 0;
+}
+
+static int cmp_float_asc(const void* pa, const void* pb) {
+  float a = *(const float*)pa, b = *(const float*)pb;
+  return (a > b) - (a < b);
+}
+
+/*
+ * Quartiles of one row of S timings (Algorithm 1, "adjudicated latency"):
+ * copy, sort ascending, then for j = 1, 2, 3 the type-7 (linear) quantile
+ *   pos = j*(S-1); lo = pos/4; rem = pos%4; hi = min(lo+1, S-1)
+ *   Q_j = x_lo                                   if rem == 0
+ *       = x_lo + ((rem*0.25f) * (x_hi - x_lo))   otherwise, each op rounded.
+ * out4 = {Q1, median = Q2, Q3, iqr = Q3 - Q1}.  `sorted` (S floats, may be
+ * NULL) receives the sorted copy.
+ * Returns 0; -1 on a bad argument; -2 if a timing is NaN or +-Inf.
+ */
+int kbo_quantiles(const float* row, uint32_t S, float* out4, float* sorted) {
+  float* x;
+  float q[4];
+  uint32_t j, i;
+  if (!row || !out4 || S == 0) return -1;
+  for (i = 0; i < S; ++i)
+    if (!is_finite32(row[i])) return -2;
+  x = (float*)malloc((size_t)S * sizeof(float));
+  if (!x) return -1;
+  memcpy(x, row, (size_t)S * sizeof(float));
+  qsort(x, S, sizeof(float), cmp_float_asc);
+  for (j = 1; j <= 3; ++j) {
+    uint64_t pos = (uint64_t)j * (uint64_t)(S - 1);
+    uint64_t lo = pos / 4u;
+    uint32_t rem = (uint32_t)(pos % 4u);
+    uint64_t hi = (lo + 1 < (uint64_t)S) ? lo + 1 : (uint64_t)S - 1;
+    if (rem == 0) {
+      q[j] = x[lo];
+    } else {
+      float w = (float)rem * 0.25f;
+      float diff = x[hi] - x[lo];
+      float step = w * diff;
+      q[j] = x[lo] + step;
+    }
+  }
+  out4[0] = q[1];
+  out4[1] = q[2];
+  out4[2] = q[3];
+  out4[3] = q[3] - q[1];
+  if (sorted) memcpy(sorted, x, (size_t)S * sizeof(float));
+  free(x);
+  return 0;
+}
+
+/*
+ * Win count of row a over row b: twice the Mann-Whitney U statistic of
+ * "a is faster (smaller) than b", ties counted once:
+ *   W = sum_i sum_j ( 2*[a_i < b_j] + [a_i == b_j] )
+ * by the literal double loop over the rows as given (unsorted).
+ */
+uint64_t kbo_wins_pair(const float* a, const float* b, uint32_t S) {
+  uint64_t w = 0;
+  uint32_t i, j;
+  for (i = 0; i < S; ++i) {
+    for (j = 0; j < S; ++j) {
+      if (a[i] < b[j]) w += 2;
+      if (a[i] == b[j]) w += 1;
+    }
+  }
+  return w;
+}
+
+/*
+ * Full adjudication of timings[K][S]: median[K], iqr[K], W[K][K] (uint32,
+ * row-major).  Any output may be NULL.  Returns 0; -1 bad argument; -2 if any
+ * timing is non-finite (outputs then unspecified).
+ */
+int kbo_adjudicate(const float* timings, uint32_t K, uint32_t S, float* median, float* iqr,
+                   uint32_t* wins) {
+  uint32_t a, b;
+  uint64_t t;
+  if (!timings || K == 0 || S == 0) return -1;
+  for (t = 0; t < (uint64_t)K * S; ++t)
+    if (!is_finite32(timings[t])) return -2;
+  if (median || iqr) {
+    for (a = 0; a < K; ++a) {
+      float q[4];
+      int rc = kbo_quantiles(timings + (size_t)a * S, S, q, NULL);
+      if (rc != 0) return rc;
+      if (median) median[a] = q[1];
+      if (iqr) iqr[a] = q[3];
+    }
+  }
+  if (wins) {
+    for (a = 0; a < K; ++a)
+      for (b = 0; b < K; ++b)
+        wins[(size_t)a * K + b] =
+            (uint32_t)kbo_wins_pair(timings + (size_t)a * S, timings + (size_t)b * S, S);
+  }
+  return 0;
+}
+
+/* Rows [a0, a1) of W only -- lets a caller spread the literal double loop over
+ * several host threads, or time a bounded sample of it. */
+int kbo_wins_rows(const float* timings, uint32_t K, uint32_t S, uint32_t a0, uint32_t a1,
+                  uint32_t* wins_rows /* [(a1-a0)][K] */) {
+  uint32_t a, b;
+  if (!timings || !wins_rows || K == 0 || S == 0 || a0 > a1 || a1 > K) return -1;
+  for (a = a0; a < a1; ++a)
+    for (b = 0; b < K; ++b)
+      wins_rows[(size_t)(a - a0) * K + b] =
+          (uint32_t)kbo_wins_pair(timings + (size_t)a * S, timings + (size_t)b * S, S);
+  return 0;
+}
+
+/*
+ * Promotion decision (Sec. 3.2; Sec. 3.4 scheduler).  Eligible = pass == 1.
+ * policy 0: order by (max_rel_err asc, median asc, index asc);
+ * policy 1: order by (median asc, index asc).
+ * The first n = min(budget, #eligible) indices go to survivors[0..n) in rank
+ * order, survivors[n..budget) = -1, *n_out = n.
+ * Written as a selection sort on the candidate list: find the best remaining
+ * candidate, emit it, repeat.
+ */
+int kbo_select(const kbo_screen_result* screen, const float* median, uint32_t K, int policy,
+               uint32_t budget, int32_t* survivors, uint32_t* n_out) {
+  uint8_t* taken;
+  uint32_t n = 0, k, slot;
+  if (!screen || !median || !survivors || !n_out || K == 0 || budget == 0) return -1;
+  if (policy != 0 && policy != 1) return -1;
+  taken = (uint8_t*)calloc(K, 1);
+  if (!taken) return -1;
+  for (slot = 0; slot < budget; ++slot) {
+    int64_t best = -1;
+    for (k = 0; k < K; ++k) {
+      int better;
+      if (taken[k] || screen[k].pass != 1u) continue;
+      if (best < 0) {
+        best = k;
+        continue;
+      }
+      better = 0;
+      if (policy == 0) {
+        if (screen[k].max_rel_err < screen[best].max_rel_err)
+          better = 1;
+        else if (screen[k].max_rel_err == screen[best].max_rel_err && median[k] < median[best])
+          better = 1;
+      } else {
+        if (median[k] < median[best]) better = 1;
+      }
+      /* equal keys: the lower index (already held in best) stays */
+      if (better) best = k;
+    }
+    if (best < 0) break;
+    taken[best] = 1;
+    survivors[n++] = (int32_t)best;
+  }
+  for (slot = n; slot < budget; ++slot) survivors[slot] = -1;
+  *n_out = n;
+  free(taken);
+  return 0;
+}
