@@ -1,0 +1,237 @@
+"""ctypes binding of the kb C ABI (include/kb.h): argument marshalling only.
+
+Every step of the path runs in the CUDA library; torch is used here for device
+memory and the current stream.  There is no CPU fallback: loading fails loudly
+when ``libkb.so`` is missing, and the entry points need CUDA tensors.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libkb.so")
+
+KB_OK = 0
+STATUS_NAMES = {
+    0: "KB_OK", 1: "KB_ERR_INVALID_ARG", 2: "KB_ERR_ALIGNMENT", 3: "KB_ERR_UNSUPPORTED",
+    4: "KB_ERR_WORKSPACE", 5: "KB_ERR_CUDA", 6: "KB_ERR_NONFINITE", 7: "KB_ERR_DEVICE_TIMEOUT",
+}
+KB_F32, KB_F16, KB_BF16 = 0, 1, 2
+KB_SELECT_ERR_THEN_TIME, KB_SELECT_TIME = 0, 1
+DTYPE_CODE = {torch.float32: KB_F32, torch.float16: KB_F16, torch.bfloat16: KB_BF16}
+
+# kb_screen_result as a numpy record (48 bytes)
+RESULT_DTYPE = np.dtype([
+    ("mismatch_count", "<u8"), ("nan_count", "<u8"), ("inf_count", "<u8"), ("argmax_idx", "<i8"),
+    ("max_abs_err", "<f4"), ("max_rel_err", "<f4"), ("pass", "<u4"), ("reserved", "<u4"),
+])
+RESULT_BYTES = 48
+
+EXPORTS = [
+    "kb_ctx_create", "kb_ctx_destroy", "kb_last_error", "kb_ctx_poll", "kb_ctx_set_grid",
+    "kb_mask_create_strided", "kb_mask_create_bitmap", "kb_mask_count", "kb_mask_destroy",
+    "kb_screen", "kb_screen_host", "kb_adjudicate", "kb_select",
+]
+
+
+class KbError(RuntimeError):
+    def __init__(self, status: int, where: str, text: str = ""):
+        self.status = status
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)} {text}".strip())
+
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Load libkb.so (built by ``python -m paper_2608_02611_b200.build``)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build the CUDA library first "
+            "(python -m paper_2608_02611_b200.build); there is no CPU fallback")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, u32, u64, i32, f32 = (ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint64, ctypes.c_int,
+                              ctypes.c_float)
+    pvp = ctypes.POINTER(ctypes.c_void_p)
+    L.kb_ctx_create.argtypes = [i32, pvp]
+    L.kb_ctx_destroy.argtypes = [vp]
+    L.kb_last_error.argtypes = [vp]
+    L.kb_last_error.restype = ctypes.c_char_p
+    L.kb_ctx_poll.argtypes = [vp, vp, ctypes.POINTER(i32)]
+    L.kb_ctx_set_grid.argtypes = [vp, u32]
+    L.kb_mask_create_strided.argtypes = [vp, u64, u32, u32, u32, pvp]
+    L.kb_mask_create_bitmap.argtypes = [vp, u64, u32, vp, pvp]
+    L.kb_mask_count.argtypes = [vp, ctypes.POINTER(u64)]
+    L.kb_mask_destroy.argtypes = [vp]
+    L.kb_screen.argtypes = [vp, vp, vp, u32, u64, i32, f32, f32, vp, vp, vp]
+    L.kb_screen_host.argtypes = [vp, vp, vp, u32, u64, i32, f32, f32, vp, vp, vp]
+    L.kb_adjudicate.argtypes = [vp, vp, u32, u32, vp, vp, vp, vp]
+    L.kb_select.argtypes = [vp, vp, vp, u32, i32, u32, vp, vp, vp]
+    for name in EXPORTS:
+        if name != "kb_last_error":
+            getattr(L, name).restype = i32
+    _lib = L
+    return L
+
+
+def _stream_ptr(device) -> int:
+    return int(torch.cuda.current_stream(device).cuda_stream)
+
+
+class Mask:
+    """A fidelity mask over tiles of 2**log2_tile elements (owned by a Context)."""
+
+    def __init__(self, ctx: "Context", handle: int, spec: tuple):
+        self._ctx, self._h, self.spec = ctx, handle, spec
+
+    @property
+    def n_selected(self) -> int:
+        n = ctypes.c_uint64(0)
+        rc = load().kb_mask_count(self._h, ctypes.byref(n))
+        if rc != KB_OK:
+            raise KbError(rc, "kb_mask_count")
+        return int(n.value)
+
+    def close(self):
+        if self._h:
+            load().kb_mask_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class Context:
+    """kb_ctx bound to one CUDA device."""
+
+    def __init__(self, device: int = 0):
+        L = load()
+        h = ctypes.c_void_p()
+        rc = L.kb_ctx_create(int(device), ctypes.byref(h))
+        if rc != KB_OK:
+            raise KbError(rc, "kb_ctx_create", (L.kb_last_error(None) or b"").decode())
+        self._h = h.value
+        self.device = torch.device("cuda", int(device))
+
+    # -- plumbing -----------------------------------------------------------
+    def _check(self, rc: int, where: str):
+        if rc != KB_OK:
+            raise KbError(rc, where, (load().kb_last_error(self._h) or b"").decode())
+
+    def close(self):
+        if getattr(self, "_h", None):
+            load().kb_ctx_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def poll(self) -> int:
+        """Synchronise the current stream and return (and clear) the device status."""
+        st = ctypes.c_int(0)
+        self._check(load().kb_ctx_poll(self._h, _stream_ptr(self.device), ctypes.byref(st)),
+                    "kb_ctx_poll")
+        return int(st.value)
+
+    def set_grid(self, blocks: int):
+        self._check(load().kb_ctx_set_grid(self._h, int(blocks)), "kb_ctx_set_grid")
+
+    # -- masks --------------------------------------------------------------
+    def mask_strided(self, N: int, log2_tile: int, stride: int, phase: int) -> Mask:
+        h = ctypes.c_void_p()
+        self._check(load().kb_mask_create_strided(self._h, N, log2_tile, stride, phase,
+                                                  ctypes.byref(h)), "kb_mask_create_strided")
+        return Mask(self, h.value, ("strided", log2_tile, stride, phase))
+
+    def mask_bitmap(self, N: int, log2_tile: int, words: np.ndarray) -> Mask:
+        words = np.ascontiguousarray(words, dtype=np.uint64)
+        h = ctypes.c_void_p()
+        self._check(load().kb_mask_create_bitmap(self._h, N, log2_tile, words.ctypes.data,
+                                                 ctypes.byref(h)), "kb_mask_create_bitmap")
+        return Mask(self, h.value, ("bitmap", log2_tile, words.copy()))
+
+    # -- the three calls ----------------------------------------------------
+    def screen(self, ref: torch.Tensor, cands: Sequence[torch.Tensor], atol: float, rtol: float,
+               mask: Optional[Mask] = None, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """kb_screen.  Returns a uint8 CUDA tensor [K, 48] of kb_screen_result records
+        (see ``records``); asynchronous on the current stream."""
+        K = len(cands)
+        N = ref.numel()
+        code = DTYPE_CODE.get(ref.dtype, -1)
+        for c in cands:
+            if c.dtype != ref.dtype or c.numel() != N or not c.is_cuda or not c.is_contiguous():
+                raise KbError(1, "kb_screen", "candidates must be contiguous CUDA tensors with the "
+                                              "reference's dtype and element count")
+        if not ref.is_cuda or not ref.is_contiguous():
+            raise KbError(1, "kb_screen", "reference must be a contiguous CUDA tensor")
+        if out is None:
+            out = torch.empty((K, RESULT_BYTES), dtype=torch.uint8, device=ref.device)
+        ptrs = (ctypes.c_void_p * max(K, 1))(*[c.data_ptr() for c in cands])
+        rc = load().kb_screen(self._h, ref.data_ptr(), ptrs, K, N, code, float(atol), float(rtol),
+                              mask._h if mask is not None else None, out.data_ptr(),
+                              _stream_ptr(ref.device))
+        self._check(rc, "kb_screen")
+        return out
+
+    def screen_host(self, ref: torch.Tensor, cands: Sequence[torch.Tensor], atol: float,
+                    rtol: float, mask: Optional[Mask] = None) -> np.ndarray:
+        """kb_screen_host: all tensors in host memory; returns K records (synchronous)."""
+        K = len(cands)
+        N = ref.numel()
+        code = DTYPE_CODE.get(ref.dtype, -1)
+        for c in list(cands) + [ref]:
+            if c.is_cuda or not c.is_contiguous() or c.dtype != ref.dtype or c.numel() != N:
+                raise KbError(1, "kb_screen_host", "tensors must be contiguous host tensors of one "
+                                                   "dtype and element count")
+        out = np.zeros(K, dtype=RESULT_DTYPE)
+        ptrs = (ctypes.c_void_p * max(K, 1))(*[c.data_ptr() for c in cands])
+        rc = load().kb_screen_host(self._h, ref.data_ptr(), ptrs, K, N, code, float(atol),
+                                   float(rtol), mask._h if mask is not None else None,
+                                   out.ctypes.data, _stream_ptr(self.device))
+        self._check(rc, "kb_screen_host")
+        return out
+
+    def adjudicate(self, timings: torch.Tensor, want_wins: bool = True):
+        """kb_adjudicate on a CUDA float32 tensor [K, S] -> (median[K], iqr[K], wins[K,K] or None).
+        wins is int32 storage holding uint32 counts (values < 2^31 for S < 32768)."""
+        if timings.dtype != torch.float32 or timings.dim() != 2 or not timings.is_cuda \
+                or not timings.is_contiguous():
+            raise KbError(1, "kb_adjudicate", "timings must be a contiguous CUDA float32 [K, S] tensor")
+        K, S = timings.shape
+        med = torch.empty(K, dtype=torch.float32, device=timings.device)
+        iqr = torch.empty(K, dtype=torch.float32, device=timings.device)
+        wins = torch.empty((K, K), dtype=torch.int32, device=timings.device) if want_wins else None
+        rc = load().kb_adjudicate(self._h, timings.data_ptr(), K, S, med.data_ptr(), iqr.data_ptr(),
+                                  wins.data_ptr() if want_wins else None,
+                                  _stream_ptr(timings.device))
+        self._check(rc, "kb_adjudicate")
+        return med, iqr, wins
+
+    def select(self, screen_out: torch.Tensor, median: torch.Tensor, policy: int, budget: int):
+        """kb_select -> (survivors int32 [budget] in rank order, n int32 [1]) on the device."""
+        K = median.numel()
+        surv = torch.empty(budget, dtype=torch.int32, device=median.device)
+        n = torch.empty(1, dtype=torch.int32, device=median.device)
+        rc = load().kb_select(self._h, screen_out.data_ptr(), median.data_ptr(), K, int(policy),
+                              int(budget), surv.data_ptr(), n.data_ptr(), _stream_ptr(median.device))
+        self._check(rc, "kb_select")
+        return surv, n
+
+
+def records(screen_out: torch.Tensor) -> np.ndarray:
+    """Copy a [K, 48] uint8 result tensor to the host as K numpy records (synchronises)."""
+    return screen_out.cpu().numpy().view(RESULT_DTYPE).reshape(-1)

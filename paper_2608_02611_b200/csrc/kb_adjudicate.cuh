@@ -1,0 +1,172 @@
+// Stability adjudication kernels (Algorithm 1 "adjudicated latency"; Sec. 1
+// contribution 1; Appendix "Relative Variability Metrics").
+//
+// rows_kernel         one CTA per candidate: sort its S timings in shared
+//                     memory (bitonic), take the type-7 quartiles with the
+//                     operation order fixed, write median and IQR.
+// wins_kernel         pairwise doubled Mann-Whitney counts.  A CTA takes a
+//                     block of 8 "a" rows x 8 "b" rows and a chunk of samples
+//                     of each; the a-chunk is staged in shared memory, each
+//                     warp owns one b row and each lane keeps up to 8 of its
+//                     samples in registers.  Per sample pair the work is two
+//                     compares that yield 0 / -1 and one three-input add.
+//                     Partial counts are merged with integer atomics.
+// wins_mirror_kernel  W[b][a] = 2*S*S - W[a][b] for the block-lower triangle.
+#pragma once
+
+#include "kb_common.cuh"
+
+namespace kb {
+
+constexpr int kRowsThreads = 256;
+
+__global__ void __launch_bounds__(kRowsThreads) rows_kernel(const float* __restrict__ timings,
+                                                            unsigned int S, unsigned int P /*pow2 >= S*/,
+                                                            float* __restrict__ median,
+                                                            float* __restrict__ iqr,
+                                                            unsigned int* status) {
+  extern __shared__ float xs[];
+  const unsigned int k = blockIdx.x;
+  const float* row = timings + (size_t)k * S;
+  const float inf = __uint_as_float(0x7F800000u);
+  bool nonfinite = false;
+  for (unsigned int i = threadIdx.x; i < P; i += kRowsThreads) {
+    float v = inf;   // padding sorts to the end
+    if (i < S) {
+      v = row[i];
+      if (!(fabsf(v) <= 3.402823466e38f)) nonfinite = true;
+    }
+    xs[i] = v;
+  }
+  if (nonfinite) set_status(status, (unsigned int)KB_ERR_NONFINITE);
+  __syncthreads();
+  for (unsigned int size = 2; size <= P; size <<= 1) {
+    for (unsigned int stride = size >> 1; stride > 0; stride >>= 1) {
+      for (unsigned int t = threadIdx.x; t < (P >> 1); t += kRowsThreads) {
+        const unsigned int lo = 2 * t - (t & (stride - 1));
+        const unsigned int hi = lo + stride;
+        const bool up = (lo & size) == 0;
+        const float a = xs[lo], b = xs[hi];
+        if ((a > b) == up) {
+          xs[lo] = b;
+          xs[hi] = a;
+        }
+      }
+      __syncthreads();
+    }
+  }
+  if (threadIdx.x == 0) {
+    float q[4];
+#pragma unroll
+    for (unsigned int j = 1; j <= 3; ++j) {
+      const unsigned long long pos = (unsigned long long)j * (S - 1);
+      const unsigned int lo = (unsigned int)(pos >> 2);
+      const unsigned int rem = (unsigned int)(pos & 3ull);
+      const unsigned int hi = (lo + 1 < S) ? lo + 1 : S - 1;
+      if (rem == 0) {
+        q[j] = xs[lo];
+      } else {
+        const float w = (float)rem * 0.25f;
+        q[j] = __fadd_rn(xs[lo], __fmul_rn(w, __fsub_rn(xs[hi], xs[lo])));
+      }
+    }
+    if (median) median[k] = q[2];
+    if (iqr) iqr[k] = __fsub_rn(q[3], q[1]);
+  }
+}
+
+// ---------------------------------------------------------------------------
+constexpr int kWinsThreads = 256;
+constexpr int kWinsRowsPerBlock = 8;    // a rows per CTA = b rows per CTA = warps
+constexpr int kWinsMaxR = 8;            // b samples per lane
+
+struct WinsParams {
+  const float* timings;
+  unsigned int* wins;
+  unsigned int K, S;
+  unsigned int KB;      // ceil(K / 8)
+  unsigned int npairs;  // KB*(KB+1)/2 block pairs, diagonal included
+  unsigned int nj, JC;  // b-sample chunks and their length (JC = 32*R)
+  unsigned int ni, IC;  // a-sample chunks and their length (multiple of 4)
+};
+
+// cnt += [a < b] + [a <= b]  (= 2*[a<b] + [a==b]); NaN padding compares false.
+__device__ __forceinline__ void count_pair(unsigned int& cnt, float a, float b) {
+  unsigned int s1, s2;
+  asm("set.lt.u32.f32 %0, %1, %2;" : "=r"(s1) : "f"(a), "f"(b));
+  asm("set.le.u32.f32 %0, %1, %2;" : "=r"(s2) : "f"(a), "f"(b));
+  cnt = cnt - s1 - s2;   // set yields 0xFFFFFFFF when true
+}
+
+template <int R>
+__global__ void __launch_bounds__(kWinsThreads) wins_kernel(const WinsParams p) {
+  extern __shared__ float as[];   // [8][IC]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  unsigned int item = blockIdx.x;
+  const unsigned int ic = item % p.ni;
+  item /= p.ni;
+  const unsigned int jc = item % p.nj;
+  const unsigned int pair = item / p.nj;
+  // block pair index -> (Ab <= Bb): row-major upper triangle
+  unsigned int Ab = 0, rem = pair;
+  while (rem >= p.KB - Ab) {
+    rem -= p.KB - Ab;
+    ++Ab;
+  }
+  const unsigned int Bb = Ab + rem;
+  const float qnan = __uint_as_float(0x7FC00000u);
+
+  // stage the a-chunk: rows Ab*8 .. Ab*8+7, samples ic*IC .. +IC
+  const unsigned int i0 = ic * p.IC;
+  for (unsigned int t = threadIdx.x; t < kWinsRowsPerBlock * p.IC; t += kWinsThreads) {
+    const unsigned int rr = t / p.IC, ii = t % p.IC;
+    const unsigned int a = Ab * kWinsRowsPerBlock + rr, i = i0 + ii;
+    as[t] = (a < p.K && i < p.S) ? p.timings[(size_t)a * p.S + i] : qnan;
+  }
+  // this warp's b row, this lane's samples
+  const unsigned int b = Bb * kWinsRowsPerBlock + warp;
+  float bv[R];
+#pragma unroll
+  for (int m = 0; m < R; ++m) {
+    const unsigned int j = jc * p.JC + lane + 32 * m;
+    bv[m] = (b < p.K && j < p.S) ? p.timings[(size_t)b * p.S + j] : qnan;
+  }
+  __syncthreads();
+  if (b >= p.K) return;
+
+  for (int rr = 0; rr < kWinsRowsPerBlock; ++rr) {
+    const unsigned int a = Ab * kWinsRowsPerBlock + rr;
+    if (a >= p.K) break;
+    unsigned int cnt[R];
+#pragma unroll
+    for (int m = 0; m < R; ++m) cnt[m] = 0u;
+    const float4* arow = reinterpret_cast<const float4*>(as + (size_t)rr * p.IC);
+    const unsigned int n4 = p.IC >> 2;
+#pragma unroll 2
+    for (unsigned int i = 0; i < n4; ++i) {
+      const float4 a4 = arow[i];
+#pragma unroll
+      for (int m = 0; m < R; ++m) {
+        count_pair(cnt[m], a4.x, bv[m]);
+        count_pair(cnt[m], a4.y, bv[m]);
+        count_pair(cnt[m], a4.z, bv[m]);
+        count_pair(cnt[m], a4.w, bv[m]);
+      }
+    }
+    unsigned int total = 0u;
+#pragma unroll
+    for (int m = 0; m < R; ++m) total += cnt[m];
+    total = warp_add_u32(total);
+    if (lane == 0 && total != 0u) atomicAdd(&p.wins[(size_t)a * p.K + b], total);
+  }
+}
+
+__global__ void wins_mirror_kernel(unsigned int* __restrict__ wins, unsigned int K, unsigned int S) {
+  const unsigned int b = blockIdx.x * blockDim.x + threadIdx.x;   // column
+  const unsigned int a = blockIdx.y;                              // row
+  if (a >= K || b >= K) return;
+  if ((a / kWinsRowsPerBlock) > (b / kWinsRowsPerBlock))
+    wins[(size_t)a * K + b] = 2u * S * S - wins[(size_t)b * K + a];
+}
+
+}  // namespace kb

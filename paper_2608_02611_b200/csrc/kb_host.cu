@@ -1,0 +1,633 @@
+// Host side of the kb C ABI: argument validation (the shape/dtype part of
+// the policy check, Sec. 3.2), workspace management and kernel dispatch.
+// Declarations and their contracts are in include/kb.h.
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <cmath>
+#include <new>
+#include <vector>
+
+#include "kb_adjudicate.cuh"
+#include "kb_common.cuh"
+#include "kb_screen.cuh"
+#include "kb_select.cuh"
+
+using namespace kb;
+
+struct kb_ctx {
+  int device = 0;
+  int sm_count = 0;
+  unsigned char* ws = nullptr;      // [acc K*40 | pad | pointer table K*8]
+  size_t ws_bytes = 0;
+  unsigned int* d_status = nullptr;
+  uint32_t forced_grid = 0;
+  char err[512] = {0};
+  // staging owned for kb_screen_host
+  unsigned char* st_ref = nullptr;
+  size_t st_ref_bytes = 0;
+  unsigned char* st_batch[2] = {nullptr, nullptr};
+  size_t st_batch_bytes = 0;
+  kb_screen_result* st_out = nullptr;
+  size_t st_out_bytes = 0;
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t ev_copied[2] = {nullptr, nullptr};
+  cudaEvent_t ev_done[2] = {nullptr, nullptr};
+};
+
+struct kb_mask {
+  kb_ctx* ctx = nullptr;
+  uint64_t N = 0;
+  uint32_t log2_tile = 0;
+  int kind = 0;                    // 1 strided, 2 bitmap
+  uint32_t stride = 1, phase = 0;
+  unsigned long long* d_bits = nullptr;
+  uint32_t* d_tiles = nullptr;     // selected FULL kernel tiles (log2_tile >= 12 only)
+  uint32_t n_tiles = 0;
+  bool coarse = false;             // log2_tile >= 12: the streaming kernel can skip tiles
+  uint64_t n_selected = 0;
+};
+
+namespace {
+
+thread_local char g_create_err[256] = {0};
+
+kb_status fail(kb_ctx* ctx, kb_status st, const char* fmt, ...) {
+  if (ctx) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(ctx->err, sizeof ctx->err, fmt, ap);
+    va_end(ap);
+  }
+  return st;
+}
+
+struct DeviceGuard {
+  int prev = -1;
+  bool changed = false;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) changed = cudaSetDevice(dev) == cudaSuccess;
+  }
+  ~DeviceGuard() {
+    if (changed) cudaSetDevice(prev);
+  }
+};
+
+#define KB_CUDA(ctx, call)                                                              \
+  do {                                                                                  \
+    cudaError_t e_ = (call);                                                            \
+    if (e_ != cudaSuccess)                                                              \
+      return fail((ctx), KB_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e_));  \
+  } while (0)
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline int elem_bytes(kb_dtype dt) { return dt == KB_F32 ? 4 : 2; }
+
+kb_status ensure_ws(kb_ctx* ctx, uint32_t K) {
+  const size_t need = round_up((size_t)K * sizeof(Acc), 256) + (size_t)K * sizeof(void*);
+  if (need <= ctx->ws_bytes) return KB_OK;
+  if (ctx->ws) cudaFree(ctx->ws);   // waits for enqueued work that still uses it
+  ctx->ws = nullptr;
+  ctx->ws_bytes = 0;
+  const size_t grow = round_up(need * 2, 4096);
+  if (cudaMalloc(&ctx->ws, grow) != cudaSuccess) {
+    cudaGetLastError();
+    return fail(ctx, KB_ERR_WORKSPACE, "cannot allocate %zu bytes of device workspace", grow);
+  }
+  ctx->ws_bytes = grow;
+  return KB_OK;
+}
+
+template <typename T>
+kb_status ensure_buf(kb_ctx* ctx, T** buf, size_t* have, size_t need) {
+  if (need <= *have) return KB_OK;
+  if (*buf) cudaFree(*buf);
+  *buf = nullptr;
+  *have = 0;
+  if (cudaMalloc(reinterpret_cast<void**>(buf), need) != cudaSuccess) {
+    cudaGetLastError();
+    return fail(ctx, KB_ERR_WORKSPACE, "cannot allocate %zu bytes of device staging", need);
+  }
+  *have = need;
+  return KB_OK;
+}
+
+template <int DT>
+kb_status launch_stream(kb_ctx* ctx, StreamParams& sp, cudaStream_t st) {
+  const uint32_t tile_bytes = kTile * Elem<DT>::kBytes;
+  sp.stages = (tile_bytes == 8192) ? 10 : 6;
+  const size_t smem = stream_smem_bytes(sp.stages, tile_bytes);
+  const unsigned long long nitems = (unsigned long long)sp.nchunks * sp.ntiles;
+  unsigned long long grid = ctx->forced_grid ? ctx->forced_grid : 2ull * ctx->sm_count;
+  if (grid > nitems) grid = nitems;
+  screen_stream_kernel<DT><<<(unsigned int)grid, kStreamThreads, smem, st>>>(sp);
+  KB_CUDA(ctx, cudaGetLastError());
+  return KB_OK;
+}
+
+template <int DT>
+kb_status launch_generic(kb_ctx* ctx, const void* ref, const void* const* tab, Acc* acc, uint32_t K,
+                         uint64_t e0, uint64_t e1, float atol, float rtol, const MaskDev& md,
+                         cudaStream_t st) {
+  if (e1 <= e0) return KB_OK;
+  const uint64_t len = e1 - e0;
+  uint64_t bx = (len + 255) / 256;
+  const uint64_t cap = (uint64_t)ctx->sm_count * 8;
+  if (bx > cap) bx = cap;
+  dim3 grid((unsigned int)bx, K);
+  screen_generic_kernel<DT><<<grid, 256, 0, st>>>(ref, tab, acc, e0, e1, atol, rtol, md);
+  KB_CUDA(ctx, cudaGetLastError());
+  return KB_OK;
+}
+
+template <int DT>
+kb_status set_stream_attr(kb_ctx* ctx) {
+  const uint32_t tile_bytes = kTile * Elem<DT>::kBytes;
+  const size_t smem = stream_smem_bytes(tile_bytes == 8192 ? 10 : 6, tile_bytes);
+  KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT>,
+                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  return KB_OK;
+}
+
+template <int R>
+void launch_wins(const WinsParams& wp, unsigned int grid, size_t smem, cudaStream_t st) {
+  wins_kernel<R><<<grid, kWinsThreads, smem, st>>>(wp);
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------
+// context
+// ---------------------------------------------------------------------------
+
+extern "C" kb_status kb_ctx_create(int device, kb_ctx** out) {
+  if (!out) {
+    snprintf(g_create_err, sizeof g_create_err, "kb_ctx_create: out is NULL");
+    return KB_ERR_INVALID_ARG;
+  }
+  *out = nullptr;
+  int ndev = 0;
+  cudaError_t e = cudaGetDeviceCount(&ndev);
+  if (e != cudaSuccess || device < 0 || device >= ndev) {
+    snprintf(g_create_err, sizeof g_create_err, "kb_ctx_create: no CUDA device %d (%s)", device,
+             e != cudaSuccess ? cudaGetErrorString(e) : "out of range");
+    cudaGetLastError();
+    return e != cudaSuccess ? KB_ERR_CUDA : KB_ERR_INVALID_ARG;
+  }
+  kb_ctx* ctx = new (std::nothrow) kb_ctx();
+  if (!ctx) return KB_ERR_WORKSPACE;
+  ctx->device = device;
+  DeviceGuard g(device);
+  cudaDeviceProp prop;
+  kb_status st = KB_OK;
+  auto bail = [&](kb_status s) {
+    snprintf(g_create_err, sizeof g_create_err, "kb_ctx_create: %s", ctx->err);
+    kb_ctx_destroy(ctx);
+    return s;
+  };
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) {
+    fail(ctx, KB_ERR_CUDA, "cudaGetDeviceProperties failed");
+    return bail(KB_ERR_CUDA);
+  }
+  ctx->sm_count = prop.multiProcessorCount;
+  if (cudaMalloc(&ctx->d_status, 256) != cudaSuccess || cudaMemset(ctx->d_status, 0, 256) != cudaSuccess) {
+    fail(ctx, KB_ERR_WORKSPACE, "cannot allocate the device status word");
+    return bail(KB_ERR_WORKSPACE);
+  }
+  if ((st = set_stream_attr<KB_F32>(ctx)) != KB_OK) return bail(st);
+  if ((st = set_stream_attr<KB_F16>(ctx)) != KB_OK) return bail(st);
+  if ((st = set_stream_attr<KB_BF16>(ctx)) != KB_OK) return bail(st);
+  if (cudaFuncSetAttribute(rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)(KB_MAX_S * sizeof(float))) != cudaSuccess) {
+    fail(ctx, KB_ERR_CUDA, "cannot raise the shared-memory limit of the row kernel");
+    return bail(KB_ERR_CUDA);
+  }
+  *out = ctx;
+  return KB_OK;
+}
+
+extern "C" kb_status kb_ctx_destroy(kb_ctx* ctx) {
+  if (!ctx) return KB_OK;
+  DeviceGuard g(ctx->device);
+  cudaDeviceSynchronize();
+  if (ctx->ws) cudaFree(ctx->ws);
+  if (ctx->d_status) cudaFree(ctx->d_status);
+  if (ctx->st_ref) cudaFree(ctx->st_ref);
+  for (int i = 0; i < 2; ++i) {
+    if (ctx->st_batch[i]) cudaFree(ctx->st_batch[i]);
+    if (ctx->ev_copied[i]) cudaEventDestroy(ctx->ev_copied[i]);
+    if (ctx->ev_done[i]) cudaEventDestroy(ctx->ev_done[i]);
+  }
+  if (ctx->st_out) cudaFree(ctx->st_out);
+  if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
+  cudaGetLastError();
+  delete ctx;
+  return KB_OK;
+}
+
+extern "C" const char* kb_last_error(const kb_ctx* ctx) { return ctx ? ctx->err : g_create_err; }
+
+extern "C" kb_status kb_ctx_poll(kb_ctx* ctx, void* stream, kb_status* device_status) {
+  if (!ctx || !device_status) return KB_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  unsigned int word = 0;
+  KB_CUDA(ctx, cudaMemcpyAsync(&word, ctx->d_status, sizeof word, cudaMemcpyDeviceToHost, st));
+  KB_CUDA(ctx, cudaMemsetAsync(ctx->d_status, 0, sizeof word, st));
+  KB_CUDA(ctx, cudaStreamSynchronize(st));
+  *device_status = (kb_status)word;
+  return KB_OK;
+}
+
+extern "C" kb_status kb_ctx_set_grid(kb_ctx* ctx, uint32_t blocks) {
+  if (!ctx) return KB_ERR_INVALID_ARG;
+  ctx->forced_grid = blocks;
+  return KB_OK;
+}
+
+// ---------------------------------------------------------------------------
+// masks
+// ---------------------------------------------------------------------------
+
+namespace {
+
+kb_status mask_finish(kb_ctx* ctx, kb_mask* m, const uint64_t* host_bits, kb_mask** out) {
+  const uint64_t tile = 1ull << m->log2_tile;
+  const uint64_t nt = (m->N + tile - 1) >> m->log2_tile;
+  auto sel = [&](uint64_t t) -> bool {
+    if (m->kind == 1) return (t % m->stride) == m->phase;
+    return (host_bits[t >> 6] >> (t & 63)) & 1ull;
+  };
+  auto tile_len = [&](uint64_t t) -> uint64_t {
+    const uint64_t b = t << m->log2_tile;
+    return (m->N - b < tile) ? m->N - b : tile;
+  };
+  m->coarse = m->log2_tile >= 12;
+  uint64_t nsel = 0;
+  if (m->kind == 1) {
+    const uint64_t cnt = nt > m->phase ? (nt - 1 - m->phase) / m->stride + 1 : 0;
+    nsel = cnt * tile;
+    if (cnt && sel(nt - 1)) nsel -= tile - tile_len(nt - 1);
+  } else {
+    for (uint64_t t = 0; t < nt; ++t)
+      if (sel(t)) nsel += tile_len(t);
+  }
+  m->n_selected = nsel;
+  DeviceGuard g(ctx->device);
+  if (m->kind == 2) {
+    const size_t words = (size_t)((nt + 63) / 64);
+    if (cudaMalloc(&m->d_bits, words * 8) != cudaSuccess) {
+      cudaGetLastError();
+      delete m;
+      return fail(ctx, KB_ERR_WORKSPACE, "cannot allocate the mask bitmap");
+    }
+    if (cudaMemcpy(m->d_bits, host_bits, words * 8, cudaMemcpyHostToDevice) != cudaSuccess) {
+      cudaFree(m->d_bits);
+      delete m;
+      return fail(ctx, KB_ERR_CUDA, "mask bitmap upload failed");
+    }
+  }
+  if (m->coarse) {
+    // list of selected FULL kernel tiles, ascending (the ragged tail goes to the generic kernel)
+    const uint32_t per = 1u << (m->log2_tile - 12);
+    const uint64_t nfull = m->N / kTile;
+    std::vector<uint32_t> tiles;
+    for (uint64_t t = 0; t < nt; ++t) {
+      if (!sel(t)) continue;
+      for (uint32_t w = 0; w < per; ++w) {
+        const uint64_t kt = t * per + w;
+        if (kt < nfull) tiles.push_back((uint32_t)kt);
+      }
+    }
+    m->n_tiles = (uint32_t)tiles.size();
+    if (m->n_tiles) {
+      if (cudaMalloc(&m->d_tiles, tiles.size() * 4) != cudaSuccess ||
+          cudaMemcpy(m->d_tiles, tiles.data(), tiles.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess) {
+        cudaGetLastError();
+        if (m->d_tiles) cudaFree(m->d_tiles);
+        if (m->d_bits) cudaFree(m->d_bits);
+        delete m;
+        return fail(ctx, KB_ERR_WORKSPACE, "cannot build the mask tile list");
+      }
+    }
+  }
+  *out = m;
+  return KB_OK;
+}
+
+}  // namespace
+
+extern "C" kb_status kb_mask_create_strided(kb_ctx* ctx, uint64_t N, uint32_t log2_tile,
+                                            uint32_t stride, uint32_t phase, kb_mask** out) {
+  if (!ctx || !out) return KB_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (N == 0 || N > KB_MAX_N || log2_tile > 31 || stride == 0 || phase >= stride)
+    return fail(ctx, KB_ERR_INVALID_ARG, "kb_mask_create_strided: bad N, log2_tile, stride or phase");
+  kb_mask* m = new (std::nothrow) kb_mask();
+  if (!m) return fail(ctx, KB_ERR_WORKSPACE, "out of host memory");
+  m->ctx = ctx;
+  m->N = N;
+  m->log2_tile = log2_tile;
+  m->kind = 1;
+  m->stride = stride;
+  m->phase = phase;
+  return mask_finish(ctx, m, nullptr, out);
+}
+
+extern "C" kb_status kb_mask_create_bitmap(kb_ctx* ctx, uint64_t N, uint32_t log2_tile,
+                                           const uint64_t* host_bits, kb_mask** out) {
+  if (!ctx || !out) return KB_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (N == 0 || N > KB_MAX_N || log2_tile > 31 || !host_bits)
+    return fail(ctx, KB_ERR_INVALID_ARG, "kb_mask_create_bitmap: bad N, log2_tile or bitmap");
+  kb_mask* m = new (std::nothrow) kb_mask();
+  if (!m) return fail(ctx, KB_ERR_WORKSPACE, "out of host memory");
+  m->ctx = ctx;
+  m->N = N;
+  m->log2_tile = log2_tile;
+  m->kind = 2;
+  return mask_finish(ctx, m, host_bits, out);
+}
+
+extern "C" kb_status kb_mask_count(const kb_mask* mask, uint64_t* n_selected) {
+  if (!mask || !n_selected) return KB_ERR_INVALID_ARG;
+  *n_selected = mask->n_selected;
+  return KB_OK;
+}
+
+extern "C" kb_status kb_mask_destroy(kb_mask* m) {
+  if (!m) return KB_OK;
+  DeviceGuard g(m->ctx->device);
+  if (m->d_bits) cudaFree(m->d_bits);
+  if (m->d_tiles) cudaFree(m->d_tiles);
+  cudaGetLastError();
+  delete m;
+  return KB_OK;
+}
+
+// ---------------------------------------------------------------------------
+// kb_screen
+// ---------------------------------------------------------------------------
+
+namespace {
+
+kb_status validate_screen(kb_ctx* ctx, const void* ref, const void* const* cands, uint32_t K,
+                          uint64_t N, kb_dtype dtype, float atol, float rtol, const kb_mask* mask,
+                          const void* out, bool device_ptrs) {
+  if (!ctx) return KB_ERR_INVALID_ARG;
+  if (!ref || !cands || !out) return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen: null pointer");
+  if (K == 0 || K > KB_MAX_K) return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen: K=%u outside [1, %u]", K, KB_MAX_K);
+  if (N == 0 || N > KB_MAX_N) return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen: N outside [1, 2^32]");
+  if (dtype != KB_F32 && dtype != KB_F16 && dtype != KB_BF16)
+    return fail(ctx, KB_ERR_UNSUPPORTED, "kb_screen: unknown dtype %d", (int)dtype);
+  if (!(atol >= 0.0f) || !(rtol >= 0.0f) || std::isinf(atol) || std::isinf(rtol))
+    return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen: atol and rtol must be finite and >= 0");
+  if (mask && (mask->N != N || mask->ctx != ctx))
+    return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen: the mask was created for another N or context");
+  if (device_ptrs) {
+    if (!aligned16(ref)) return fail(ctx, KB_ERR_ALIGNMENT, "kb_screen: reference not 16-byte aligned");
+    if ((reinterpret_cast<uintptr_t>(out) & 7u) != 0)
+      return fail(ctx, KB_ERR_ALIGNMENT, "kb_screen: output not 8-byte aligned");
+  }
+  for (uint32_t k = 0; k < K; ++k) {
+    if (!cands[k]) return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen: candidate %u is NULL", k);
+    if (device_ptrs && !aligned16(cands[k]))
+      return fail(ctx, KB_ERR_ALIGNMENT, "kb_screen: candidate %u not 16-byte aligned", k);
+  }
+  return KB_OK;
+}
+
+template <int DT>
+kb_status screen_impl(kb_ctx* ctx, const void* d_ref, const void* const* h_cands, uint32_t K,
+                      uint64_t N, float atol, float rtol, const kb_mask* mask,
+                      kb_screen_result* d_out, cudaStream_t st) {
+  kb_status rc = ensure_ws(ctx, K);
+  if (rc != KB_OK) return rc;
+  Acc* acc = reinterpret_cast<Acc*>(ctx->ws);
+  const void** table = reinterpret_cast<const void**>(ctx->ws + round_up((size_t)K * sizeof(Acc), 256));
+
+  for (uint32_t off = 0; off < K; off += kPtrsPerLaunch) {
+    PtrChunk ch;
+    const uint32_t cnt = (K - off < (uint32_t)kPtrsPerLaunch) ? K - off : (uint32_t)kPtrsPerLaunch;
+    memcpy(ch.p, h_cands + off, cnt * sizeof(void*));
+    upload_ptrs_kernel<<<(cnt + 127) / 128, 128, 0, st>>>(ch, table, off, cnt);
+    KB_CUDA(ctx, cudaGetLastError());
+  }
+  KB_CUDA(ctx, cudaMemsetAsync(acc, 0, (size_t)K * sizeof(Acc), st));
+
+  MaskDev md;
+  md.kind = mask ? mask->kind : 0;
+  md.log2_tile = mask ? mask->log2_tile : 0;
+  md.stride = mask ? mask->stride : 1;
+  md.phase = mask ? mask->phase : 0;
+  md.bits = mask ? mask->d_bits : nullptr;
+
+  if (mask && !mask->coarse) {
+    // finer than a kernel tile: every sector is touched anyway
+    rc = launch_generic<DT>(ctx, d_ref, table, acc, K, 0, N, atol, rtol, md, st);
+    if (rc != KB_OK) return rc;
+  } else {
+    const uint64_t nfull = N / kTile;
+    StreamParams sp;
+    sp.ref = d_ref;
+    sp.cands = table;
+    sp.acc = acc;
+    sp.tile_list = mask ? mask->d_tiles : nullptr;
+    sp.ntiles = mask ? mask->n_tiles : (uint32_t)nfull;
+    sp.K = K;
+    sp.atol = atol;
+    sp.rtol = rtol;
+    sp.status = ctx->d_status;
+    if (sp.ntiles) {
+      // chunk the candidates: shared-memory accumulators hold kMaxKC of them, and
+      // small tensors need more, smaller items to fill the machine
+      uint32_t nchunks = (K + kMaxKC - 1) / kMaxKC;
+      const uint64_t grid = ctx->forced_grid ? ctx->forced_grid : 2ull * ctx->sm_count;
+      const uint64_t want_items = 8 * grid;
+      if ((uint64_t)nchunks * sp.ntiles < want_items) {
+        uint64_t nc = (want_items + sp.ntiles - 1) / sp.ntiles;
+        const uint64_t max_nc = (K + 7) / 8;           // at least 8 candidates per chunk
+        if (nc > max_nc) nc = max_nc;
+        if (nc > nchunks) nchunks = (uint32_t)nc;
+      }
+      sp.KC = (K + nchunks - 1) / nchunks;
+      sp.nchunks = (K + sp.KC - 1) / sp.KC;
+      rc = launch_stream<DT>(ctx, sp, st);
+      if (rc != KB_OK) return rc;
+    }
+    // ragged tail (elements past the last full kernel tile)
+    rc = launch_generic<DT>(ctx, d_ref, table, acc, K, nfull * kTile, N, atol, rtol, md, st);
+    if (rc != KB_OK) return rc;
+  }
+  screen_finalize_kernel<<<(K + 127) / 128, 128, 0, st>>>(acc, d_out, K);
+  KB_CUDA(ctx, cudaGetLastError());
+  return KB_OK;
+}
+
+kb_status screen_dispatch(kb_ctx* ctx, const void* d_ref, const void* const* h_cands, uint32_t K,
+                          uint64_t N, kb_dtype dtype, float atol, float rtol, const kb_mask* mask,
+                          kb_screen_result* d_out, cudaStream_t st) {
+  switch (dtype) {
+    case KB_F32: return screen_impl<KB_F32>(ctx, d_ref, h_cands, K, N, atol, rtol, mask, d_out, st);
+    case KB_F16: return screen_impl<KB_F16>(ctx, d_ref, h_cands, K, N, atol, rtol, mask, d_out, st);
+    default: return screen_impl<KB_BF16>(ctx, d_ref, h_cands, K, N, atol, rtol, mask, d_out, st);
+  }
+}
+
+}  // namespace
+
+extern "C" kb_status kb_screen(kb_ctx* ctx, const void* d_ref, const void* const* h_cands, uint32_t K,
+                               uint64_t N, kb_dtype dtype, float atol, float rtol,
+                               const kb_mask* mask, kb_screen_result* d_out, void* stream) {
+  kb_status rc = validate_screen(ctx, d_ref, h_cands, K, N, dtype, atol, rtol, mask, d_out, true);
+  if (rc != KB_OK) return rc;
+  DeviceGuard g(ctx->device);
+  return screen_dispatch(ctx, d_ref, h_cands, K, N, dtype, atol, rtol, mask, d_out,
+                         reinterpret_cast<cudaStream_t>(stream));
+}
+
+extern "C" kb_status kb_screen_host(kb_ctx* ctx, const void* h_ref, const void* const* h_cands_host,
+                                    uint32_t K, uint64_t N, kb_dtype dtype, float atol, float rtol,
+                                    const kb_mask* mask, kb_screen_result* h_out, void* stream) {
+  kb_status rc = validate_screen(ctx, h_ref, h_cands_host, K, N, dtype, atol, rtol, mask, h_out, false);
+  if (rc != KB_OK) return rc;
+  DeviceGuard g(ctx->device);
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const size_t bytes = (size_t)N * elem_bytes(dtype);
+  const size_t pitch = round_up(bytes, 256);
+  // batch size: about 512 MiB of candidates per batch, two batches in flight
+  uint32_t B = (uint32_t)((512ull << 20) / pitch);
+  if (B < 1) B = 1;
+  if (B > K) B = K;
+  if (!ctx->copy_stream) {
+    KB_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
+    for (int i = 0; i < 2; ++i) {
+      KB_CUDA(ctx, cudaEventCreateWithFlags(&ctx->ev_copied[i], cudaEventDisableTiming));
+      KB_CUDA(ctx, cudaEventCreateWithFlags(&ctx->ev_done[i], cudaEventDisableTiming));
+    }
+  }
+  if ((rc = ensure_buf(ctx, &ctx->st_ref, &ctx->st_ref_bytes, pitch)) != KB_OK) return rc;
+  if ((size_t)B * pitch > ctx->st_batch_bytes) {
+    size_t have0 = ctx->st_batch_bytes, have1 = ctx->st_batch_bytes;
+    if ((rc = ensure_buf(ctx, &ctx->st_batch[0], &have0, (size_t)B * pitch)) != KB_OK) return rc;
+    if ((rc = ensure_buf(ctx, &ctx->st_batch[1], &have1, (size_t)B * pitch)) != KB_OK) return rc;
+    ctx->st_batch_bytes = (size_t)B * pitch;
+  }
+  if ((rc = ensure_buf(ctx, &ctx->st_out, &ctx->st_out_bytes, (size_t)K * sizeof(kb_screen_result))) != KB_OK)
+    return rc;
+
+  // order the copy stream after work already enqueued on the caller's stream
+  KB_CUDA(ctx, cudaEventRecord(ctx->ev_done[0], st));
+  KB_CUDA(ctx, cudaEventRecord(ctx->ev_done[1], st));
+  KB_CUDA(ctx, cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_done[0], 0));
+  KB_CUDA(ctx, cudaMemcpyAsync(ctx->st_ref, h_ref, bytes, cudaMemcpyHostToDevice, ctx->copy_stream));
+  std::vector<const void*> ptrs(B);
+  int buf = 0;
+  for (uint32_t k0 = 0; k0 < K; k0 += B, buf ^= 1) {
+    const uint32_t nb = (K - k0 < B) ? K - k0 : B;
+    KB_CUDA(ctx, cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_done[buf], 0));
+    for (uint32_t i = 0; i < nb; ++i) {
+      unsigned char* dst = ctx->st_batch[buf] + (size_t)i * pitch;
+      KB_CUDA(ctx, cudaMemcpyAsync(dst, h_cands_host[k0 + i], bytes, cudaMemcpyHostToDevice, ctx->copy_stream));
+      ptrs[i] = dst;
+    }
+    KB_CUDA(ctx, cudaEventRecord(ctx->ev_copied[buf], ctx->copy_stream));
+    KB_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_copied[buf], 0));
+    rc = screen_dispatch(ctx, ctx->st_ref, ptrs.data(), nb, N, dtype, atol, rtol, mask, ctx->st_out + k0, st);
+    if (rc != KB_OK) return rc;
+    KB_CUDA(ctx, cudaEventRecord(ctx->ev_done[buf], st));
+  }
+  KB_CUDA(ctx, cudaMemcpyAsync(h_out, ctx->st_out, (size_t)K * sizeof(kb_screen_result),
+                               cudaMemcpyDeviceToHost, st));
+  KB_CUDA(ctx, cudaStreamSynchronize(st));
+  return KB_OK;
+}
+
+// ---------------------------------------------------------------------------
+// kb_adjudicate
+// ---------------------------------------------------------------------------
+
+extern "C" kb_status kb_adjudicate(kb_ctx* ctx, const float* d_timings, uint32_t K, uint32_t S,
+                                   float* d_median, float* d_iqr, uint32_t* d_wins, void* stream) {
+  if (!ctx) return KB_ERR_INVALID_ARG;
+  if (!d_timings) return fail(ctx, KB_ERR_INVALID_ARG, "kb_adjudicate: timings is NULL");
+  if (K == 0 || K > KB_MAX_K) return fail(ctx, KB_ERR_INVALID_ARG, "kb_adjudicate: K=%u outside [1, %u]", K, KB_MAX_K);
+  if (S == 0 || S > KB_MAX_S) return fail(ctx, KB_ERR_INVALID_ARG, "kb_adjudicate: S=%u outside [1, %u]", S, KB_MAX_S);
+  if ((reinterpret_cast<uintptr_t>(d_timings) & 3u) || (reinterpret_cast<uintptr_t>(d_median) & 3u) ||
+      (reinterpret_cast<uintptr_t>(d_iqr) & 3u) || (reinterpret_cast<uintptr_t>(d_wins) & 3u))
+    return fail(ctx, KB_ERR_ALIGNMENT, "kb_adjudicate: a pointer is not 4-byte aligned");
+  DeviceGuard g(ctx->device);
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+
+  // rows: sort + quartiles (also the place where non-finite timings are caught)
+  unsigned int P = 1;
+  while (P < S) P <<= 1;
+  rows_kernel<<<K, kRowsThreads, (size_t)P * sizeof(float), st>>>(d_timings, S, P, d_median, d_iqr,
+                                                                   ctx->d_status);
+  KB_CUDA(ctx, cudaGetLastError());
+  if (!d_wins) return KB_OK;
+
+  KB_CUDA(ctx, cudaMemsetAsync(d_wins, 0, (size_t)K * K * sizeof(uint32_t), st));
+  WinsParams wp;
+  wp.timings = d_timings;
+  wp.wins = d_wins;
+  wp.K = K;
+  wp.S = S;
+  wp.KB = (K + kWinsRowsPerBlock - 1) / kWinsRowsPerBlock;
+  const unsigned long long npairs = (unsigned long long)wp.KB * (wp.KB + 1) / 2;
+  wp.npairs = (unsigned int)npairs;
+  wp.nj = (S + 32 * kWinsMaxR - 1) / (32 * kWinsMaxR);
+  const unsigned int per_chunk = (S + wp.nj - 1) / wp.nj;
+  const int R = (int)((per_chunk + 31) / 32);
+  wp.JC = 32u * R;
+  wp.IC = (unsigned int)round_up(S < 1024 ? S : 1024, 4);
+  wp.ni = (S + wp.IC - 1) / wp.IC;
+  while (npairs * wp.nj * wp.ni < 2ull * ctx->sm_count && wp.IC > 64) {
+    wp.IC = (unsigned int)round_up((wp.IC + 1) / 2, 4);
+    wp.ni = (S + wp.IC - 1) / wp.IC;
+  }
+  const unsigned long long items = npairs * wp.nj * wp.ni;
+  if (items > 0x7FFFFFFFull) return fail(ctx, KB_ERR_UNSUPPORTED, "kb_adjudicate: K*S too large for one launch");
+  const size_t smem = (size_t)kWinsRowsPerBlock * wp.IC * sizeof(float);
+  const unsigned int grid = (unsigned int)items;
+  switch (R) {
+    case 1: launch_wins<1>(wp, grid, smem, st); break;
+    case 2: launch_wins<2>(wp, grid, smem, st); break;
+    case 3: launch_wins<3>(wp, grid, smem, st); break;
+    case 4: launch_wins<4>(wp, grid, smem, st); break;
+    case 5: launch_wins<5>(wp, grid, smem, st); break;
+    case 6: launch_wins<6>(wp, grid, smem, st); break;
+    case 7: launch_wins<7>(wp, grid, smem, st); break;
+    default: launch_wins<8>(wp, grid, smem, st); break;
+  }
+  KB_CUDA(ctx, cudaGetLastError());
+  if (wp.KB > 1) {
+    dim3 mg((K + 255) / 256, K);
+    wins_mirror_kernel<<<mg, 256, 0, st>>>(d_wins, K, S);
+    KB_CUDA(ctx, cudaGetLastError());
+  }
+  return KB_OK;
+}
+
+// ---------------------------------------------------------------------------
+// kb_select
+// ---------------------------------------------------------------------------
+
+extern "C" kb_status kb_select(kb_ctx* ctx, const kb_screen_result* d_screen, const float* d_median,
+                               uint32_t K, kb_select_policy policy, uint32_t budget,
+                               int32_t* d_survivors, uint32_t* d_n_survivors, void* stream) {
+  if (!ctx) return KB_ERR_INVALID_ARG;
+  if (!d_screen || !d_median || !d_survivors || !d_n_survivors)
+    return fail(ctx, KB_ERR_INVALID_ARG, "kb_select: null pointer");
+  if (K == 0 || K > KB_MAX_K) return fail(ctx, KB_ERR_INVALID_ARG, "kb_select: K=%u outside [1, %u]", K, KB_MAX_K);
+  if (budget == 0) return fail(ctx, KB_ERR_INVALID_ARG, "kb_select: budget must be >= 1");
+  if (policy != KB_SELECT_ERR_THEN_TIME && policy != KB_SELECT_TIME)
+    return fail(ctx, KB_ERR_UNSUPPORTED, "kb_select: unknown policy %d", (int)policy);
+  DeviceGuard g(ctx->device);
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  select_kernel<<<(K + kSelectThreads - 1) / kSelectThreads, kSelectThreads, 0, st>>>(
+      d_screen, d_median, K, (int)policy, budget, d_survivors, d_n_survivors);
+  KB_CUDA(ctx, cudaGetLastError());
+  return KB_OK;
+}

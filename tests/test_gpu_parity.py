@@ -1,0 +1,409 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle.
+
+Everything is compared bit for bit: counts, flags, indices, the bit patterns of
+max_abs_err / max_rel_err / median / IQR, the win counts and the survivor
+order.  Sizes span several 4096-element tiles plus ragged tails, all three
+dtypes, masks finer and coarser than a kernel tile, candidate counts around
+the chunk size of the streaming kernel, and several forced grid sizes (the
+result must not depend on the launch shape).
+"""
+import json
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2608_02611_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+FIELDS = ["mismatch_count", "nan_count", "inf_count", "argmax_idx", "pass", "reserved"]
+
+
+@pytest.fixture(scope="module")
+def kb():
+    from paper_2608_02611_b200 import binding
+    return binding
+
+
+@pytest.fixture(scope="module")
+def ctx(kb):
+    c = kb.Context(0)
+    yield c
+    c.close()
+
+
+def fbits(a):
+    return np.ascontiguousarray(a, dtype=np.float32).view(np.uint32)
+
+
+def assert_records_equal(got, want, label=""):
+    for f in FIELDS:
+        bad = np.nonzero(got[f] != want[f])[0]
+        assert bad.size == 0, f"{label} field {f} differs at candidates {bad[:8]}: " \
+                              f"got {got[f][bad[:8]]} want {want[f][bad[:8]]}"
+    for f in ("max_abs_err", "max_rel_err"):
+        bad = np.nonzero(fbits(got[f]) != fbits(want[f]))[0]
+        assert bad.size == 0, f"{label} field {f} differs at candidates {bad[:8]}: " \
+                              f"got {got[f][bad[:8]]} want {want[f][bad[:8]]}"
+
+
+def oracle_screen(case_dtype, ref_t, cand_ts, atol, rtol, mask_spec=None, threads=None):
+    threads = threads or max(1, len(os.sched_getaffinity(0)))
+    ref = synth.to_oracle_array(ref_t, case_dtype)
+    cands = [synth.to_oracle_array(c, case_dtype) for c in cand_ts]
+    return oracle.screen(ref, cands, case_dtype, atol, rtol, mask_spec, threads=threads)
+
+
+def awkward(n, dtype_code, rng, device):
+    """Random values with zeros, subnormals, huge values, NaN and Inf mixed in."""
+    x = rng.standard_normal(n) * np.exp(3 * rng.standard_normal(n))
+    x[rng.random(n) < 0.02] = 0.0
+    t = torch.from_numpy(x).to(synth.TORCH_DTYPE[dtype_code])
+    bits = synth._bits(t, dtype_code)
+    u = torch.from_numpy(rng.random(n))
+    inf_mag = synth._INF_MAG[dtype_code]
+    sign = synth._SIGN_BIT[dtype_code]
+    specials = [1, 2, inf_mag - 1, inf_mag, inf_mag | 1, sign | inf_mag, sign | 1, sign]
+    for j, pat in enumerate(specials):
+        bits = torch.where((u >= 0.004 * j) & (u < 0.004 * (j + 1)), torch.full_like(bits, pat), bits)
+    return synth._from_bits(bits, dtype_code).to(device)
+
+
+def perturbed(ref, dtype_code, rng, device, p_flip=0.3, p_big=0.01, p_special=0.003):
+    n = ref.numel()
+    step = torch.from_numpy(rng.integers(-2, 3, n)) * torch.from_numpy(rng.random(n) < p_flip)
+    c = synth.ulp_step(ref.cpu(), dtype_code, step.to(torch.int64))
+    big = torch.from_numpy(rng.random(n) < p_big)
+    c = torch.where(big, (c.float() * 1.5 + 0.25).to(c.dtype), c)
+    u = torch.from_numpy(rng.random(n))
+    c = torch.where(u < p_special, torch.full_like(c, float("nan")), c)
+    c = torch.where((u >= p_special) & (u < 2 * p_special), torch.full_like(c, float("inf")), c)
+    c = torch.where((u >= 2 * p_special) & (u < 3 * p_special), torch.full_like(c, float("-inf")), c)
+    return c.contiguous().to(device)
+
+
+def run_screen(ctx, kb, ref, cands, atol, rtol, mask_spec=None, N=None):
+    mask = None
+    if mask_spec is not None:
+        N = ref.numel()
+        if mask_spec[0] == "strided":
+            mask = ctx.mask_strided(N, mask_spec[1], mask_spec[2], mask_spec[3])
+        else:
+            mask = ctx.mask_bitmap(N, mask_spec[1], mask_spec[2])
+    out = ctx.screen(ref, cands, atol, rtol, mask)
+    rec = kb.records(out)
+    assert ctx.poll() == 0
+    if mask is not None:
+        mask.close()
+    return rec
+
+
+# --------------------------------------------------------------------------
+# stored + live oracle on the small seeded configurations
+# --------------------------------------------------------------------------
+
+def _golden():
+    with open(os.path.join(GOLD, "oracle_small_cases.json")) as f:
+        return json.load(f)
+
+
+def _check_against_stored(rec, med, iqr, wins, surv, n, stored):
+    for k, s in enumerate(stored["screen"]):
+        assert int(rec["mismatch_count"][k]) == s["mismatch_count"]
+        assert int(rec["nan_count"][k]) == s["nan_count"]
+        assert int(rec["inf_count"][k]) == s["inf_count"]
+        assert int(rec["argmax_idx"][k]) == s["argmax_idx"]
+        assert int(fbits(rec["max_abs_err"])[k]) == s["max_abs_err_bits"]
+        assert int(fbits(rec["max_rel_err"])[k]) == s["max_rel_err_bits"]
+        assert int(rec["pass"][k]) == s["passed"]
+    assert fbits(med).tolist() == stored["median_bits"]
+    assert fbits(iqr).tolist() == stored["iqr_bits"]
+    assert wins.astype(np.int64).tolist() == stored["wins"]
+    assert surv.tolist() == stored["survivors"] and n == stored["n_survivors"]
+
+
+SMALL = {
+    "config1": lambda dev: synth.config1(dev),
+    "config2_side512_K16": lambda dev: synth.config2(dev, side=512, K=16, n_bad=3),
+    "config3_small": lambda dev: synth.config3(dev, B=1, H=2, S=64, D=128, K=12, n_nan=2,
+                                               n_transposed=2, S_t=50),
+    "config4_small": lambda dev: synth.config4(dev, N=1 << 14, K=40, S_t=16),
+}
+
+
+@pytest.mark.parametrize("name", list(SMALL))
+def test_small_configs_whole_path(ctx, kb, name):
+    # inputs are built on the host so that the bytes are the ones the stored values came from
+    case, timings = SMALL[name]("cpu")
+    stored = _golden()[name]
+    dev = torch.device("cuda", 0)
+    ref = case.ref.to(dev)
+    cands_cpu = case.cands()
+    cands = [c.to(dev) for c in cands_cpu]
+    out = ctx.screen(ref, cands, case.atol, case.rtol)
+    t = torch.from_numpy(timings).to(dev)
+    med, iqr, wins = ctx.adjudicate(t)
+    surv, n = ctx.select(out, med, stored["policy"], stored["budget"])
+    assert ctx.poll() == 0
+    rec = kb.records(out)
+    want = oracle_screen(case.dtype, case.ref, cands_cpu, case.atol, case.rtol)
+    assert_records_equal(rec, want, name)
+    _check_against_stored(rec, med.cpu().numpy(), iqr.cpu().numpy(),
+                          wins.cpu().numpy().view(np.uint32), surv.cpu().numpy(), int(n.item()), stored)
+
+
+def test_config5_small_two_tier(ctx, kb):
+    c5 = synth.config5("cpu", N=1 << 20, K=32, budget=4, S1=20, S2=40)
+    case = c5["case"]
+    stored = _golden()["config5_small_tier1"]
+    dev = torch.device("cuda", 0)
+    ref = case.ref.to(dev)
+    cands_cpu = case.cands()
+    cands = [c.to(dev) for c in cands_cpu]
+    _, log2_tile, stride, phase = case.mask
+    mask = ctx.mask_strided(case.N, log2_tile, stride, phase)
+    assert mask.n_selected == case.N // stride
+    out1 = ctx.screen(ref, cands, case.atol, case.rtol, mask)
+    med1, iqr1, wins1 = ctx.adjudicate(torch.from_numpy(c5["timings1"]).to(dev))
+    surv, n = ctx.select(out1, med1, kb.KB_SELECT_ERR_THEN_TIME, c5["budget"])
+    assert ctx.poll() == 0
+    rec1 = kb.records(out1)
+    _check_against_stored(rec1, med1.cpu().numpy(), iqr1.cpu().numpy(),
+                          wins1.cpu().numpy().view(np.uint32), surv.cpu().numpy(), int(n.item()), stored)
+    # tier 2: the survivors on every element, chained from the device-side survivor list
+    s = surv.cpu().numpy()[: int(n.item())].tolist()
+    out2 = ctx.screen(ref, [cands[k] for k in s], case.atol, case.rtol)
+    rec2 = kb.records(out2)
+    want2 = oracle_screen(case.dtype, case.ref, [cands_cpu[k] for k in s], case.atol, case.rtol)
+    assert_records_equal(rec2, want2, "tier2")
+    t2 = c5["make_timings2"](s)
+    med2, iqr2, wins2 = ctx.adjudicate(torch.from_numpy(t2).to(dev))
+    omed, oiqr, owins = oracle.adjudicate(t2)
+    assert (fbits(med2.cpu().numpy()) == fbits(omed)).all()
+    assert (fbits(iqr2.cpu().numpy()) == fbits(oiqr)).all()
+    assert (wins2.cpu().numpy().view(np.uint32) == owins).all()
+    mask.close()
+
+
+# --------------------------------------------------------------------------
+# awkward values, ragged sizes, chunk boundaries, grid independence
+# --------------------------------------------------------------------------
+
+@pytest.mark.parametrize("dtype_code", [synth.F32, synth.F16, synth.BF16])
+@pytest.mark.parametrize("N", [1, 7, 8, 9, 4095, 4096, 4097, 3 * 4096 + 5, 20 * 4096 + 123])
+def test_awkward_values_and_ragged_sizes(ctx, kb, dtype_code, N):
+    rng = np.random.default_rng(N * 3 + dtype_code)
+    dev = torch.device("cuda", 0)
+    ref = awkward(N, dtype_code, rng, dev)
+    cands = [ref.clone(), perturbed(ref, dtype_code, rng, dev), awkward(N, dtype_code, rng, dev),
+             perturbed(ref, dtype_code, rng, dev, p_flip=0.01, p_big=0.0, p_special=0.0)]
+    for atol, rtol in [(1e-5, 1e-3), (0.0, 0.0), (1e-2, 1.6e-2)]:
+        got = run_screen(ctx, kb, ref, cands, atol, rtol)
+        want = oracle_screen(dtype_code, ref, cands, atol, rtol)
+        assert_records_equal(got, want, f"N={N} dtype={dtype_code} tol=({atol},{rtol})")
+
+
+@pytest.mark.parametrize("K", [1, 3, 33, 127, 128, 129, 300])
+def test_candidate_counts_around_chunk_size(ctx, kb, K):
+    rng = np.random.default_rng(K)
+    dev = torch.device("cuda", 0)
+    N = 6 * 4096 + 17
+    ref = awkward(N, synth.BF16, rng, dev)
+    base = [perturbed(ref, synth.BF16, rng, dev) for _ in range(5)]
+    cands = []
+    for k in range(K):
+        c = base[k % 5].clone()
+        c[(k * 977) % N] = float(k)            # make every candidate different
+        cands.append(c)
+    got = run_screen(ctx, kb, ref, cands, 1e-2, 1.6e-2)
+    want = oracle_screen(synth.BF16, ref, cands, 1e-2, 1.6e-2)
+    assert_records_equal(got, want, f"K={K}")
+
+
+@pytest.mark.parametrize("grid", [1, 2, 5, 37, 0])
+def test_result_does_not_depend_on_grid(ctx, kb, grid):
+    rng = np.random.default_rng(99)
+    dev = torch.device("cuda", 0)
+    N = 41 * 4096 + 1000
+    ref = awkward(N, synth.F16, rng, dev)
+    cands = [perturbed(ref, synth.F16, rng, dev) for _ in range(9)] + [ref.clone()]
+    want = oracle_screen(synth.F16, ref, cands, 1e-3, 1e-2)
+    try:
+        ctx.set_grid(grid)
+        got = run_screen(ctx, kb, ref, cands, 1e-3, 1e-2)
+    finally:
+        ctx.set_grid(0)
+    assert_records_equal(got, want, f"grid={grid}")
+
+
+def test_ties_on_max_abs_err_pick_lowest_index(ctx, kb):
+    dev = torch.device("cuda", 0)
+    N = 30 * 4096
+    ref = torch.zeros(N, dtype=torch.float32, device=dev)
+    c = ref.clone()
+    hits = [29 * 4096 + 5, 17 * 4096 + 4000, 3 * 4096 + 77, 3 * 4096 + 78]
+    c[hits] = 0.5                                  # equal errors in several tiles and threads
+    for grid in (0, 1, 3):
+        ctx.set_grid(grid)
+        rec = run_screen(ctx, kb, ref, [c, ref.clone()], 0.0, 0.0)
+        ctx.set_grid(0)
+        assert rec["argmax_idx"].tolist() == [3 * 4096 + 77, 0]
+        assert rec["max_abs_err"].tolist() == [0.5, 0.0]
+        assert rec["mismatch_count"].tolist() == [4, 0]
+        assert rec["max_rel_err"].tolist() == [0.0, 0.0]       # reference is zero everywhere
+
+
+MASKS = [("strided", 0, 3, 1), ("strided", 3, 2, 0), ("strided", 7, 5, 4), ("strided", 11, 2, 1),
+         ("strided", 12, 2, 1), ("strided", 12, 16, 5), ("strided", 13, 3, 0), ("strided", 14, 1, 0),
+         ("strided", 20, 1, 0)]
+
+
+@pytest.mark.parametrize("mask_spec", MASKS)
+@pytest.mark.parametrize("N", [50 * 4096, 50 * 4096 + 999])
+def test_masks(ctx, kb, mask_spec, N):
+    rng = np.random.default_rng(N + mask_spec[1])
+    dev = torch.device("cuda", 0)
+    ref = awkward(N, synth.BF16, rng, dev)
+    cands = [perturbed(ref, synth.BF16, rng, dev) for _ in range(3)] + [ref.clone()]
+    got = run_screen(ctx, kb, ref, cands, 1e-2, 1.6e-2, mask_spec)
+    want = oracle_screen(synth.BF16, ref, cands, 1e-2, 1.6e-2, mask_spec)
+    assert_records_equal(got, want, f"mask={mask_spec} N={N}")
+
+
+@pytest.mark.parametrize("log2_tile", [2, 9, 12, 13])
+def test_bitmap_masks_and_empty_selection(ctx, kb, log2_tile):
+    rng = np.random.default_rng(log2_tile)
+    dev = torch.device("cuda", 0)
+    N = 33 * 4096 + 77
+    nt = (N + (1 << log2_tile) - 1) >> log2_tile
+    ref = awkward(N, synth.F32, rng, dev)
+    cands = [perturbed(ref, synth.F32, rng, dev) for _ in range(3)]
+    for density in (0.0, 0.3, 1.0):
+        words = np.zeros((nt + 63) // 64, dtype=np.uint64)
+        for t in np.nonzero(rng.random(nt) < density)[0] if density < 1.0 else range(nt):
+            words[int(t) >> 6] |= np.uint64(1) << np.uint64(int(t) & 63)
+        spec = ("bitmap", log2_tile, words)
+        got = run_screen(ctx, kb, ref, cands, 1e-5, 1e-3, spec)
+        want = oracle_screen(synth.F32, ref, cands, 1e-5, 1e-3, spec)
+        assert_records_equal(got, want, f"bitmap log2_tile={log2_tile} density={density}")
+        if density == 0.0:
+            assert (got["argmax_idx"] == -1).all() and (got["pass"] == 1).all()
+
+
+def test_extreme_reference_magnitudes(ctx, kb):
+    """Tiny and huge |r| where the filter's products could underflow or overflow."""
+    dev = torch.device("cuda", 0)
+    vals = np.float32([1e-38, 3e-39, 1e-45, 2e-44, 1e38, 3e38, 1e-31, 1e31, 1.0, 0.0])
+    N = 5 * 4096
+    rng = np.random.default_rng(3)
+    ref_np = rng.choice(vals, N).astype(np.float32)
+    ref = torch.from_numpy(ref_np).to(dev)
+    cands = []
+    for scale in (1.0000001, 1.5, 0.5, 3.0):
+        c = (ref_np.astype(np.float64) * scale).astype(np.float32)
+        same = rng.random(N) < 0.5
+        c[same] = ref_np[same]
+        cands.append(torch.from_numpy(c).to(dev))
+    cands.append(torch.from_numpy(np.nextafter(ref_np, np.float32(np.inf))).to(dev))
+    got = run_screen(ctx, kb, ref, cands, 0.0, 1e-3)
+    want = oracle_screen(synth.F32, ref, cands, 0.0, 1e-3)
+    assert_records_equal(got, want, "extreme")
+
+
+# --------------------------------------------------------------------------
+# argument errors leave outputs untouched and never reach the device
+# --------------------------------------------------------------------------
+
+def test_argument_errors(ctx, kb):
+    dev = torch.device("cuda", 0)
+    ref = torch.zeros(64, dtype=torch.float32, device=dev)
+    out = torch.full((1, 48), 0xAB, dtype=torch.uint8, device=dev)
+    for atol, rtol in [(-1.0, 0.0), (0.0, float("inf")), (float("nan"), 0.0)]:
+        with pytest.raises(kb.KbError) as e:
+            ctx.screen(ref, [ref.clone()], atol, rtol, out=out)
+        assert e.value.status == 1
+    with pytest.raises(kb.KbError) as e:
+        ctx.screen(ref, [], 0.0, 0.0)
+    assert e.value.status == 1
+    with pytest.raises(kb.KbError) as e:                       # misaligned candidate view
+        big = torch.zeros(65, dtype=torch.float32, device=dev)
+        ctx.screen(ref, [big[1:]], 0.0, 0.0, out=out)
+    assert e.value.status == 2
+    with pytest.raises(kb.KbError) as e:                       # dtype constraint of the policy check
+        ctx.screen(ref.double(), [ref.double()], 0.0, 0.0, out=out)
+    assert e.value.status == 3
+    with pytest.raises(kb.KbError):
+        ctx.mask_strided(64, 3, 2, 2)
+    m = ctx.mask_strided(128, 3, 2, 1)
+    with pytest.raises(kb.KbError):                            # mask made for another N
+        ctx.screen(ref, [ref.clone()], 0.0, 0.0, m, out=out)
+    m.close()
+    assert (out.cpu() == 0xAB).all()
+    t = torch.ones((3, 4), dtype=torch.float32, device=dev)
+    with pytest.raises(kb.KbError):
+        ctx.select(out, t[0], 7, 1)
+    assert ctx.poll() == 0
+
+
+# --------------------------------------------------------------------------
+# adjudication and selection
+# --------------------------------------------------------------------------
+
+@pytest.mark.parametrize("K,S", [(1, 1), (2, 2), (3, 3), (4, 4), (5, 5), (21, 4), (21, 16), (21, 60),
+                                 (8, 31), (9, 32), (17, 33), (33, 64), (16, 100), (24, 200), (7, 256),
+                                 (6, 257), (5, 300), (12, 1000), (4, 2000), (3, 2049)])
+def test_adjudicate_matches_oracle(ctx, kb, K, S):
+    rng = np.random.default_rng(K * 10007 + S)
+    dev = torch.device("cuda", 0)
+    for ties in (False, True):
+        t = rng.lognormal(0, 0.1, (K, S))
+        if ties:
+            t = np.round(t, 2)
+        t = t.astype(np.float32)
+        med, iqr, wins = ctx.adjudicate(torch.from_numpy(t).to(dev))
+        assert ctx.poll() == 0
+        omed, oiqr, owins = oracle.adjudicate(t)
+        assert (fbits(med.cpu().numpy()) == fbits(omed)).all()
+        assert (fbits(iqr.cpu().numpy()) == fbits(oiqr)).all()
+        w = wins.cpu().numpy().view(np.uint32)
+        assert (w == owins).all(), np.argwhere(w != owins)[:5]
+
+
+def test_adjudicate_negative_and_zero_timings(ctx, kb):
+    dev = torch.device("cuda", 0)
+    t = np.float32([[0.0, -1.0, 2.0, 0.0, 1.0], [1.0, 0.0, -2.0, 5.0, 1.0], [3.0, 3.0, 3.0, 3.0, 3.0]])
+    med, iqr, wins = ctx.adjudicate(torch.from_numpy(t).to(dev))
+    omed, oiqr, owins = oracle.adjudicate(t)
+    assert (med.cpu().numpy() == omed).all() and (iqr.cpu().numpy() == oiqr).all()
+    assert (wins.cpu().numpy().view(np.uint32) == owins).all()
+
+
+def test_adjudicate_flags_nonfinite(ctx, kb):
+    dev = torch.device("cuda", 0)
+    for bad in (float("nan"), float("inf"), float("-inf")):
+        t = torch.ones((5, 40), dtype=torch.float32, device=dev)
+        t[3, 17] = bad
+        ctx.adjudicate(t)
+        assert ctx.poll() == 6          # KB_ERR_NONFINITE
+        assert ctx.poll() == 0          # the status word is cleared by the read
+
+
+@pytest.mark.parametrize("policy", [0, 1])
+@pytest.mark.parametrize("K,budget", [(1, 1), (7, 3), (33, 8), (64, 64), (40, 100), (300, 32), (1000, 7)])
+def test_select_matches_oracle(ctx, kb, policy, K, budget):
+    rng = np.random.default_rng(K * 31 + budget + policy)
+    dev = torch.device("cuda", 0)
+    rec = np.zeros(K, dtype=oracle.RESULT_DTYPE)
+    rec["pass"] = rng.random(K) < 0.6
+    rec["mismatch_count"] = 1 - rec["pass"]
+    rec["max_rel_err"] = rng.choice(np.float32([0.0, 2.0 ** -7, 2.0 ** -8, 0.01, np.inf]), K)
+    med = rng.choice(np.float32([0.9, 1.0, 1.0, 1.1, 0.0, -0.0]), K).astype(np.float32)
+    d_rec = torch.from_numpy(rec.view(np.uint8).reshape(K, 48).copy()).to(dev)
+    surv, n = ctx.select(d_rec, torch.from_numpy(med).to(dev), policy, budget)
+    osurv, on = oracle.select(rec, med, policy, budget)
+    assert int(n.item()) == on
+    assert surv.cpu().numpy().tolist() == osurv.tolist()

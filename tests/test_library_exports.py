@@ -1,0 +1,57 @@
+"""The C-ABI library builds, loads and exports every symbol the header declares (CPU only;
+no compute call is made without a GPU)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "kb.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(kb_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_header_declares_the_three_calls():
+    names = declared_functions()
+    for must in ("kb_screen", "kb_adjudicate", "kb_select", "kb_ctx_create", "kb_ctx_destroy"):
+        assert must in names
+
+
+def test_library_exports_every_declared_symbol():
+    from paper_2608_02611_b200 import build, binding
+    lib_path = build.build()
+    lib = ctypes.CDLL(lib_path)
+    for name in declared_functions():
+        assert hasattr(lib, name), f"{name} is declared in kb.h but not exported"
+    assert sorted(binding.EXPORTS) == declared_functions()
+    binding.load()
+
+
+def test_result_record_layout_matches_header():
+    from paper_2608_02611_b200 import binding
+    assert binding.RESULT_DTYPE.itemsize == 48
+    assert [binding.RESULT_DTYPE.fields[n][1] for n in binding.RESULT_DTYPE.names] == \
+        [0, 8, 16, 24, 32, 36, 40, 44]
+
+
+def test_no_device_is_a_clean_error():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a device is present")
+    from paper_2608_02611_b200 import binding
+    with pytest.raises(binding.KbError):
+        binding.Context(0)
+
+
+def test_product_does_not_import_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2608_02611_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert "import oracle" not in text and "from oracle" not in text, f
+                assert "kb_oracle" not in text, f
