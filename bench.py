@@ -1,0 +1,329 @@
+"""Benchmark of the whole hot path on synthetic config 2.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+A step is one pass of the path over one batch: kb_screen of K=64 bf16
+candidates of 4096x4096 against one reference, kb_adjudicate of timings
+[64][100], kb_select of the top 32.  Inputs are resident in HBM before the
+timed region; they total 2.18 GB per step, far above the 126 MB L2, so no cache
+flush is needed between steps.  One JSON line is printed by rank 0.
+
+With N > 1 (torchrun, one process per GPU) the candidates are independent, so
+every rank screens its own 64 candidates against its own replica of the
+reference (weak scaling, no data-path collective); the time is the maximum
+over ranks.
+
+`--impl reference` times the CPU oracle (test infrastructure, used as it
+stands) on the host cores on the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "candidate-elements screened/sec"
+UNIT = "elements/s"
+K_CANDS, SIDE, S_TIMINGS, BUDGET = 64, 4096, 100, 32
+# DRAM bytes moved per algorithmic byte by the streaming screen kernel, from the ncu capture
+# summarised in profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over (K+1)*N*2 bytes);
+# None until a capture exists.
+DRAM_BYTES_PER_ALGORITHMIC_BYTE = None
+
+WORKLOAD = ("config2: screen K=64 bf16 4096x4096 (atol=1e-2, rtol=1.6e-2) + adjudicate "
+            "timings[64][100] + select top 32")
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._halt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4),
+        }
+        while not self._halt.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for name, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._halt.wait(self.period)
+
+    def stop(self):
+        self._halt.set()
+        if self.is_alive():
+            self.join(timeout=2)
+        return {"sm_mhz": int(np.median(self.samples)) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def host_cores() -> int:
+    return max(1, len(os.sched_getaffinity(0)))
+
+
+def oracle_step(ref_np, cands_np, timings, n_cands, threads):
+    """One bounded sample of the workload on the CPU oracle; returns seconds."""
+    import oracle
+    t0 = time.perf_counter()
+    rec = oracle.screen(ref_np, cands_np[:n_cands], 2, 1e-2, 1.6e-2, threads=threads)
+    med, iqr, wins = oracle.adjudicate(timings, threads=threads)
+    oracle.select(rec, med[:n_cands], 0, min(BUDGET, n_cands))
+    return time.perf_counter() - t0
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle on the host cores, same config and metric."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import torch
+    from paper_2608_02611_b200 import synth
+    cores = host_cores()
+    n_sample = min(K_CANDS, max(8, cores))          # candidates per step (bounded sample)
+    case, timings = synth.config2("cpu", side=SIDE, K=K_CANDS)
+    ref_np = synth.to_oracle_array(case.ref, case.dtype)
+    cands_np = [synth.to_oracle_array(case.make_cand(k), case.dtype) for k in range(n_sample)]
+    for _ in range(min(args.warmup, 1)):
+        oracle_step(ref_np, cands_np, timings, n_sample, cores)
+    steps = max(1, min(args.steps, 5))
+    secs = [oracle_step(ref_np, cands_np, timings, n_sample, cores) for _ in range(steps)]
+    per_step = float(np.mean(secs))
+    value = n_sample * case.N / per_step
+    sample = (f"{n_sample} of {K_CANDS} candidates of 4096x4096 bf16 per step, full adjudication "
+              f"[64][100] and select; {steps} steps")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": per_step * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic", "config": {"workload": WORKLOAD, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--side", type=int, default=SIDE,
+                    help="tensor side; anything but 4096 is for profiler captures only and is "
+                         "not a benchmark configuration")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import torch.distributed as dist
+    from paper_2608_02611_b200 import binding, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    ctx = binding.Context(local_rank)
+
+    side = args.side
+    small = side != SIDE
+    steps = max(1, args.steps)
+    warmup = max(3, args.warmup)
+
+    # ---- inputs, resident in HBM (each rank: its own candidates, same reference) ----
+    case, timings = synth.config2(dev, side=side, K=K_CANDS)
+    N = case.N
+    cands = []
+    for k in range(K_CANDS):
+        cands.append(case.make_cand(k) if rank == 0 else
+                     synth._sparse_flips(case.ref, case.dtype, synth.MASTER_SEED + 2 + 1000 * rank, k, 100))
+    d_timings = torch.from_numpy(timings).to(dev)
+    out = torch.empty((K_CANDS, binding.RESULT_BYTES), dtype=torch.uint8, device=dev)
+    torch.cuda.synchronize()
+
+    def step():
+        ctx.screen(case.ref, cands, case.atol, case.rtol, out=out)
+        med, iqr, wins = ctx.adjudicate(d_timings)
+        return ctx.select(out, med, binding.KB_SELECT_ERR_THEN_TIME, BUDGET)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(warmup):
+        step()
+    barrier()
+    assert ctx.poll() == 0
+
+    # ---- timed region: exactly `steps` steps, CUDA events, clocks sampled meanwhile ----
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    ctx.enable_timing(True)
+    launches0 = ctx.launch_count
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(steps):
+        surv, n = step()
+    e1.record()
+    barrier()
+    clocks = sampler.stop()
+    elapsed_ms = e0.elapsed_time(e1)
+    launches = ctx.launch_count - launches0
+    stream_ms = ctx.read_timer(binding.KB_TIMER_SCREEN_STREAM)
+    wins_ms = ctx.read_timer(binding.KB_TIMER_WINS)
+    ctx.enable_timing(False)
+    if world > 1:
+        t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+    ms_per_step = elapsed_ms / steps
+    value = world * K_CANDS * N / (ms_per_step * 1e-3)
+
+    # ---- end to end through the C ABI with HOST buffers (pinned), copies inside the timing ----
+    e2e_steps = max(1, min(steps, 5))
+    if args.no_e2e:
+        e2e_steps = 0
+    h_ref = case.ref.cpu().pin_memory() if e2e_steps else None
+    h_cands = [c.cpu().pin_memory() for c in cands] if e2e_steps else []
+    h_timings = torch.from_numpy(timings).pin_memory()
+
+    def e2e_step():
+        rec = ctx.screen_host(h_ref, h_cands, case.atol, case.rtol)          # H2D + D2H inside
+        dt = h_timings.to(dev, non_blocking=True)
+        med, iqr, wins = ctx.adjudicate(dt)
+        d_rec = torch.from_numpy(rec.view(np.uint8).reshape(K_CANDS, binding.RESULT_BYTES)).to(dev)
+        surv, n = ctx.select(d_rec, med, binding.KB_SELECT_ERR_THEN_TIME, BUDGET)
+        return surv.cpu(), n.cpu(), med.cpu(), iqr.cpu(), wins.cpu()
+
+    if e2e_steps:
+        e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        res = e2e_step()
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    if world > 1:
+        t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    esz = synth.ELEM_SIZE[case.dtype]
+    h2d = (K_CANDS + 1) * N * esz + K_CANDS * S_TIMINGS * 4 + K_CANDS * binding.RESULT_BYTES
+    d2h = K_CANDS * binding.RESULT_BYTES + BUDGET * 4 + 4 + 2 * K_CANDS * 4 + K_CANDS * K_CANDS * 4
+    e2e_value = world * K_CANDS * N / (e2e_s / e2e_steps) if e2e_steps else None
+
+    if rank != 0:
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (streaming screen): algorithmic bytes / event time ----
+    peak, peak_src = peaks()
+    alg_bytes = (K_CANDS + 1) * N * esz                      # reference counted once
+    avg_stream_ms = float(np.mean(stream_ms)) if len(stream_ms) else float("nan")
+    achieved = alg_bytes / (avg_stream_ms * 1e-3) / 1e9
+    traffic = DRAM_BYTES_PER_ALGORITHMIC_BYTE * alg_bytes if DRAM_BYTES_PER_ALGORITHMIC_BYTE else None
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
+                "kernel": "screen_stream_kernel<bf16>", "launch_ms_avg": avg_stream_ms,
+                "launch_ms_min": float(np.min(stream_ms)) if len(stream_ms) else None,
+                "algorithmic_bytes_per_launch": alg_bytes, "launches_timed": int(len(stream_ms))}
+
+    # ---- CPU baseline: the oracle as it stands on a bounded sample (rank 0, N=1 only) ----
+    cpu_baseline = None
+    if world == 1 and not args.no_cpu_baseline:
+        cores = host_cores()
+        n_sample = K_CANDS
+        ref_np = synth.to_oracle_array(case.ref, case.dtype)
+        cands_np = [synth.to_oracle_array(c, case.dtype) for c in cands[:n_sample]]
+        secs = oracle_step(ref_np, cands_np, timings, n_sample, cores)
+        cpu_baseline = {"value": n_sample * N / secs, "unit": UNIT, "cores": cores, "kind": "oracle",
+                        "sample": f"one full step: {n_sample} candidates x {N} elements screened, "
+                                  f"adjudication [64][100], select; {secs:.2f} s wall on {cores} threads"}
+
+    S2 = S_TIMINGS * S_TIMINGS
+    avg_wins_ms = float(np.mean(wins_ms)) if len(wins_ms) else float("nan")
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
+        "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": WORKLOAD if not small else f"{side}x{side} variant (profiler capture only)",
+                   "K": K_CANDS, "N": N, "storage": "bf16", "S": S_TIMINGS, "budget": BUDGET,
+                   "l2": "inputs (2.18 GB per step) exceed the 126 MB L2; no flush between steps",
+                   "sharding": "candidates per rank, reference replicated, no collective"},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+                "ms_per_step": e2e_s / e2e_steps * 1e3 if e2e_steps else None},
+        "gpu_launches": int(launches),
+        "roofline": roofline,
+        "cpu_baseline": cpu_baseline,
+        "screen_gbs_whole_step": world * alg_bytes / (ms_per_step * 1e-3) / 1e9,
+        "pairwise_comparisons_per_s": K_CANDS * K_CANDS * S2 / (avg_wins_ms * 1e-3),
+        "wins_kernel_ms_avg": avg_wins_ms,
+        "n_survivors": int(n.item()),
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    ctx.close()
+
+
+if __name__ == "__main__":
+    main()

@@ -110,6 +110,24 @@ kb_status kb_ctx_poll(kb_ctx* ctx, void* stream, kb_status* device_status);
  * kernel (0 = automatic).  Results do not depend on it. */
 kb_status kb_ctx_set_grid(kb_ctx* ctx, uint32_t blocks);
 
+/* ---- instrumentation (used by the benchmark; no paper counterpart) ------- */
+
+typedef enum {
+  KB_TIMER_SCREEN_STREAM = 0, /* the streaming screen kernel */
+  KB_TIMER_WINS = 1           /* the pairwise win-count kernel */
+} kb_timer;
+
+/* With timing on, every launch of the two kernels above is bracketed by a pair
+ * of CUDA events recorded on the launching stream (taken from a ctx-owned
+ * pool of 256 pairs per timer; older launches are overwritten). */
+kb_status kb_ctx_enable_timing(kb_ctx* ctx, int on);
+/* Wait for the recorded launches of `which` since the last read, write their
+ * durations in milliseconds (oldest first, at most `cap`) to h_ms (HOST) and
+ * their number to *n (HOST); the record is then cleared. */
+kb_status kb_ctx_read_timer(kb_ctx* ctx, kb_timer which, float* h_ms, uint32_t cap, uint32_t* n);
+/* Number of kernels this context has launched since it was created (HOST out). */
+kb_status kb_ctx_launch_count(const kb_ctx* ctx, uint64_t* n);
+
 /* ---- fidelity masks (Sec. 3.2 "Fidelity level", rendered on elements) --- */
 
 /* A mask selects whole tiles of 2^log2_tile consecutive elements: element i is

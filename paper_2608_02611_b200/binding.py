@@ -23,6 +23,7 @@ STATUS_NAMES = {
 }
 KB_F32, KB_F16, KB_BF16 = 0, 1, 2
 KB_SELECT_ERR_THEN_TIME, KB_SELECT_TIME = 0, 1
+KB_TIMER_SCREEN_STREAM, KB_TIMER_WINS = 0, 1
 DTYPE_CODE = {torch.float32: KB_F32, torch.float16: KB_F16, torch.bfloat16: KB_BF16}
 
 # kb_screen_result as a numpy record (48 bytes)
@@ -34,6 +35,7 @@ RESULT_BYTES = 48
 
 EXPORTS = [
     "kb_ctx_create", "kb_ctx_destroy", "kb_last_error", "kb_ctx_poll", "kb_ctx_set_grid",
+    "kb_ctx_enable_timing", "kb_ctx_read_timer", "kb_ctx_launch_count",
     "kb_mask_create_strided", "kb_mask_create_bitmap", "kb_mask_count", "kb_mask_destroy",
     "kb_screen", "kb_screen_host", "kb_adjudicate", "kb_select",
 ]
@@ -67,6 +69,9 @@ def load() -> ctypes.CDLL:
     L.kb_last_error.restype = ctypes.c_char_p
     L.kb_ctx_poll.argtypes = [vp, vp, ctypes.POINTER(i32)]
     L.kb_ctx_set_grid.argtypes = [vp, u32]
+    L.kb_ctx_enable_timing.argtypes = [vp, i32]
+    L.kb_ctx_read_timer.argtypes = [vp, i32, vp, u32, ctypes.POINTER(u32)]
+    L.kb_ctx_launch_count.argtypes = [vp, ctypes.POINTER(u64)]
     L.kb_mask_create_strided.argtypes = [vp, u64, u32, u32, u32, pvp]
     L.kb_mask_create_bitmap.argtypes = [vp, u64, u32, vp, pvp]
     L.kb_mask_count.argtypes = [vp, ctypes.POINTER(u64)]
@@ -149,6 +154,23 @@ class Context:
 
     def set_grid(self, blocks: int):
         self._check(load().kb_ctx_set_grid(self._h, int(blocks)), "kb_ctx_set_grid")
+
+    def enable_timing(self, on: bool = True):
+        self._check(load().kb_ctx_enable_timing(self._h, 1 if on else 0), "kb_ctx_enable_timing")
+
+    def read_timer(self, which: int, cap: int = 256) -> np.ndarray:
+        """Durations (ms) of the instrumented kernel's launches since the last read."""
+        buf = np.zeros(cap, dtype=np.float32)
+        n = ctypes.c_uint32(0)
+        self._check(load().kb_ctx_read_timer(self._h, int(which), buf.ctypes.data, cap,
+                                             ctypes.byref(n)), "kb_ctx_read_timer")
+        return buf[: n.value].copy()
+
+    @property
+    def launch_count(self) -> int:
+        n = ctypes.c_uint64(0)
+        self._check(load().kb_ctx_launch_count(self._h, ctypes.byref(n)), "kb_ctx_launch_count")
+        return int(n.value)
 
     # -- masks --------------------------------------------------------------
     def mask_strided(self, N: int, log2_tile: int, stride: int, phase: int) -> Mask:

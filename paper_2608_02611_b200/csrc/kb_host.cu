@@ -33,6 +33,13 @@ struct kb_ctx {
   cudaStream_t copy_stream = nullptr;
   cudaEvent_t ev_copied[2] = {nullptr, nullptr};
   cudaEvent_t ev_done[2] = {nullptr, nullptr};
+  // instrumentation
+  uint64_t launches = 0;
+  bool timing = false;
+  static constexpr int kTimers = 2, kPool = 256;
+  cudaEvent_t tm_beg[kTimers][kPool] = {};
+  cudaEvent_t tm_end[kTimers][kPool] = {};
+  uint32_t tm_used[kTimers] = {0, 0};
 };
 
 struct kb_mask {
@@ -84,6 +91,23 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline int elem_bytes(kb_dtype dt) { return dt == KB_F32 ? 4 : 2; }
 
+// Event pair around one launch of an instrumented kernel (no-op unless timing is on).
+struct ScopedTimer {
+  kb_ctx* ctx;
+  cudaStream_t st;
+  int which, slot = -1;
+  ScopedTimer(kb_ctx* c, int w, cudaStream_t s) : ctx(c), st(s), which(w) {
+    if (!ctx->timing) return;
+    slot = (int)(ctx->tm_used[which] % kb_ctx::kPool);
+    cudaEventRecord(ctx->tm_beg[which][slot], st);
+  }
+  ~ScopedTimer() {
+    if (slot < 0) return;
+    cudaEventRecord(ctx->tm_end[which][slot], st);
+    ++ctx->tm_used[which];
+  }
+};
+
 kb_status ensure_ws(kb_ctx* ctx, uint32_t K) {
   const size_t need = round_up((size_t)K * sizeof(Acc), 256) + (size_t)K * sizeof(void*);
   if (need <= ctx->ws_bytes) return KB_OK;
@@ -121,7 +145,11 @@ kb_status launch_stream(kb_ctx* ctx, StreamParams& sp, cudaStream_t st) {
   const unsigned long long nitems = (unsigned long long)sp.nchunks * sp.ntiles;
   unsigned long long grid = ctx->forced_grid ? ctx->forced_grid : 2ull * ctx->sm_count;
   if (grid > nitems) grid = nitems;
-  screen_stream_kernel<DT><<<(unsigned int)grid, kStreamThreads, smem, st>>>(sp);
+  {
+    ScopedTimer tm(ctx, KB_TIMER_SCREEN_STREAM, st);
+    screen_stream_kernel<DT><<<(unsigned int)grid, kStreamThreads, smem, st>>>(sp);
+  }
+  ++ctx->launches;
   KB_CUDA(ctx, cudaGetLastError());
   return KB_OK;
 }
@@ -137,6 +165,7 @@ kb_status launch_generic(kb_ctx* ctx, const void* ref, const void* const* tab, A
   if (bx > cap) bx = cap;
   dim3 grid((unsigned int)bx, K);
   screen_generic_kernel<DT><<<grid, 256, 0, st>>>(ref, tab, acc, e0, e1, atol, rtol, md);
+  ++ctx->launches;
   KB_CUDA(ctx, cudaGetLastError());
   return KB_OK;
 }
@@ -147,6 +176,9 @@ kb_status set_stream_attr(kb_ctx* ctx) {
   const size_t smem = stream_smem_bytes(tile_bytes == 8192 ? 10 : 6, tile_bytes);
   KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT>,
                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT>,
+                                    cudaFuncAttributePreferredSharedMemoryCarveout,
+                                    (int)cudaSharedmemCarveoutMaxShared));
   return KB_OK;
 }
 
@@ -221,6 +253,11 @@ extern "C" kb_status kb_ctx_destroy(kb_ctx* ctx) {
   }
   if (ctx->st_out) cudaFree(ctx->st_out);
   if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
+  for (int t = 0; t < kb_ctx::kTimers; ++t)
+    for (int i = 0; i < kb_ctx::kPool; ++i) {
+      if (ctx->tm_beg[t][i]) cudaEventDestroy(ctx->tm_beg[t][i]);
+      if (ctx->tm_end[t][i]) cudaEventDestroy(ctx->tm_end[t][i]);
+    }
   cudaGetLastError();
   delete ctx;
   return KB_OK;
@@ -243,6 +280,44 @@ extern "C" kb_status kb_ctx_poll(kb_ctx* ctx, void* stream, kb_status* device_st
 extern "C" kb_status kb_ctx_set_grid(kb_ctx* ctx, uint32_t blocks) {
   if (!ctx) return KB_ERR_INVALID_ARG;
   ctx->forced_grid = blocks;
+  return KB_OK;
+}
+
+extern "C" kb_status kb_ctx_enable_timing(kb_ctx* ctx, int on) {
+  if (!ctx) return KB_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  if (on && !ctx->tm_beg[0][0]) {
+    for (int t = 0; t < kb_ctx::kTimers; ++t)
+      for (int i = 0; i < kb_ctx::kPool; ++i) {
+        KB_CUDA(ctx, cudaEventCreate(&ctx->tm_beg[t][i]));
+        KB_CUDA(ctx, cudaEventCreate(&ctx->tm_end[t][i]));
+      }
+  }
+  ctx->timing = on != 0;
+  ctx->tm_used[0] = ctx->tm_used[1] = 0;
+  return KB_OK;
+}
+
+extern "C" kb_status kb_ctx_read_timer(kb_ctx* ctx, kb_timer which, float* h_ms, uint32_t cap,
+                                       uint32_t* n) {
+  if (!ctx || !h_ms || !n || (int)which < 0 || (int)which >= kb_ctx::kTimers) return KB_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  const uint32_t used = ctx->tm_used[which];
+  uint32_t have = used < (uint32_t)kb_ctx::kPool ? used : (uint32_t)kb_ctx::kPool;
+  if (have > cap) have = cap;
+  for (uint32_t i = 0; i < have; ++i) {
+    const uint32_t slot = (used - have + i) % kb_ctx::kPool;
+    KB_CUDA(ctx, cudaEventSynchronize(ctx->tm_end[which][slot]));
+    KB_CUDA(ctx, cudaEventElapsedTime(&h_ms[i], ctx->tm_beg[which][slot], ctx->tm_end[which][slot]));
+  }
+  *n = have;
+  ctx->tm_used[which] = 0;
+  return KB_OK;
+}
+
+extern "C" kb_status kb_ctx_launch_count(const kb_ctx* ctx, uint64_t* n) {
+  if (!ctx || !n) return KB_ERR_INVALID_ARG;
+  *n = ctx->launches;
   return KB_OK;
 }
 
@@ -412,6 +487,7 @@ kb_status screen_impl(kb_ctx* ctx, const void* d_ref, const void* const* h_cands
     const uint32_t cnt = (K - off < (uint32_t)kPtrsPerLaunch) ? K - off : (uint32_t)kPtrsPerLaunch;
     memcpy(ch.p, h_cands + off, cnt * sizeof(void*));
     upload_ptrs_kernel<<<(cnt + 127) / 128, 128, 0, st>>>(ch, table, off, cnt);
+    ++ctx->launches;
     KB_CUDA(ctx, cudaGetLastError());
   }
   KB_CUDA(ctx, cudaMemsetAsync(acc, 0, (size_t)K * sizeof(Acc), st));
@@ -438,6 +514,13 @@ kb_status screen_impl(kb_ctx* ctx, const void* d_ref, const void* const* h_cands
     sp.K = K;
     sp.atol = atol;
     sp.rtol = rtol;
+    sp.rtol_lean = -1.0f;
+    if (rtol >= 9.5367431640625e-07f) {   // 2^-20
+      const double v = (double)rtol * (1.0 - 9.5367431640625e-07);
+      float f = (float)v;
+      if ((double)f > v) f = std::nextafterf(f, 0.0f);
+      sp.rtol_lean = f;
+    }
     sp.status = ctx->d_status;
     if (sp.ntiles) {
       // chunk the candidates: shared-memory accumulators hold kMaxKC of them, and
@@ -461,6 +544,7 @@ kb_status screen_impl(kb_ctx* ctx, const void* d_ref, const void* const* h_cands
     if (rc != KB_OK) return rc;
   }
   screen_finalize_kernel<<<(K + 127) / 128, 128, 0, st>>>(acc, d_out, K);
+  ++ctx->launches;
   KB_CUDA(ctx, cudaGetLastError());
   return KB_OK;
 }
@@ -565,6 +649,7 @@ extern "C" kb_status kb_adjudicate(kb_ctx* ctx, const float* d_timings, uint32_t
   while (P < S) P <<= 1;
   rows_kernel<<<K, kRowsThreads, (size_t)P * sizeof(float), st>>>(d_timings, S, P, d_median, d_iqr,
                                                                    ctx->d_status);
+  ++ctx->launches;
   KB_CUDA(ctx, cudaGetLastError());
   if (!d_wins) return KB_OK;
 
@@ -591,6 +676,8 @@ extern "C" kb_status kb_adjudicate(kb_ctx* ctx, const float* d_timings, uint32_t
   if (items > 0x7FFFFFFFull) return fail(ctx, KB_ERR_UNSUPPORTED, "kb_adjudicate: K*S too large for one launch");
   const size_t smem = (size_t)kWinsRowsPerBlock * wp.IC * sizeof(float);
   const unsigned int grid = (unsigned int)items;
+  {
+  ScopedTimer tm(ctx, KB_TIMER_WINS, st);
   switch (R) {
     case 1: launch_wins<1>(wp, grid, smem, st); break;
     case 2: launch_wins<2>(wp, grid, smem, st); break;
@@ -601,10 +688,13 @@ extern "C" kb_status kb_adjudicate(kb_ctx* ctx, const float* d_timings, uint32_t
     case 7: launch_wins<7>(wp, grid, smem, st); break;
     default: launch_wins<8>(wp, grid, smem, st); break;
   }
+  }
+  ++ctx->launches;
   KB_CUDA(ctx, cudaGetLastError());
   if (wp.KB > 1) {
     dim3 mg((K + 255) / 256, K);
     wins_mirror_kernel<<<mg, 256, 0, st>>>(d_wins, K, S);
+    ++ctx->launches;
     KB_CUDA(ctx, cudaGetLastError());
   }
   return KB_OK;
@@ -628,6 +718,7 @@ extern "C" kb_status kb_select(kb_ctx* ctx, const kb_screen_result* d_screen, co
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   select_kernel<<<(K + kSelectThreads - 1) / kSelectThreads, kSelectThreads, 0, st>>>(
       d_screen, d_median, K, (int)policy, budget, d_survivors, d_n_survivors);
+  ++ctx->launches;
   KB_CUDA(ctx, cudaGetLastError());
   return KB_OK;
 }

@@ -35,6 +35,7 @@ struct StreamParams {
   uint32_t K, KC, nchunks;
   uint32_t stages;
   float atol, rtol;
+  float rtol_lean;              // rtol*(1-2^-20) rounded down, or -1: see the lean filter below
   unsigned int* status;
 };
 
@@ -55,6 +56,23 @@ __device__ __forceinline__ void consumers_sync() {
   asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory");
 }
 
+// three-input maxima (one instruction on sm_100); the .NaN form returns NaN if any input is NaN
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ float max3_nan(float a, float b, float c) {
+  float d;
+  asm("max.NaN.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ float max2_nan(float a, float b) {
+  float d;
+  asm("max.NaN.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+  return d;
+}
+
 // Shared-memory carve-up (dynamic): stage buffers first (128-byte aligned).
 struct StreamSmem {
   unsigned char* buf;
@@ -62,26 +80,41 @@ struct StreamSmem {
   uint64_t* empty;
   unsigned long long* cnt;   // [3][kMaxKC] mism, nan, inf
   unsigned long long* key;   // [kMaxKC]
-  unsigned int* rel;         // [kMaxKC]
-  float2* thr;               // [kMaxKC][kWarps]: (abs threshold, rel threshold) per warp
+  const void** ptrs;         // [kMaxKC] candidate pointers of the current chunk (producer only)
+  unsigned int* rel;         // [kMaxKC] bits of the running max relative error (CTA-wide)
+  float* thr;                // [kMaxKC][kWarps] running max |c-r| seen by each warp (-1: none)
   volatile unsigned int* abort_flag;
 };
 
 __host__ __device__ inline size_t stream_smem_bytes(uint32_t stages, uint32_t tile_bytes) {
   size_t b = (size_t)stages * tile_bytes;
   b += 2 * (size_t)stages * 8;
-  b += 3 * (size_t)kMaxKC * 8 + (size_t)kMaxKC * 8 + (size_t)kMaxKC * 4;
-  b += (size_t)kMaxKC * kWarps * 8;
+  b += 3 * (size_t)kMaxKC * 8 + (size_t)kMaxKC * 8 + (size_t)kMaxKC * 8 + (size_t)kMaxKC * 4;
+  b += (size_t)kMaxKC * kWarps * 4;
   b += 16;
   return b + 128;  // alignment slack
 }
 
+// The filter.  Per (tile, candidate) step a thread looks at its 16 elements and
+// decides, without branches, whether anything about them could change the
+// candidate's record; only then does its warp take the exact path.  With
+//   ad = |c - r|,  rel = the CTA's running max of ad/|r|,  th = the warp's running max of ad,
+// nothing can change if for every element
+//   (b) ad <= th                          (an equal error in a later tile loses the index tie)
+//   (c) ad - rel*|r| <= 0 as a real number (then ad/|r| cannot round above rel)
+//   (a) ad <= atol + rtol*|r|              (match)
+// and no NaN is involved.  (c) is one fused multiply-add, whose single rounding
+// keeps the sign; a NaN-propagating max carries any NaN (a NaN or Inf candidate,
+// Inf - Inf) to the decision.  While rel <= rtol*(1-2^-20), (c) implies (a) and
+// the "lean" form drops the tolerance test: ad <= rel*|r| <= RN(rtol*|r|) <= tol.
 template <int DT>
-__global__ void __maxnreg__(112) screen_stream_kernel(const StreamParams p) {
+__global__ void __maxnreg__(96) screen_stream_kernel(const StreamParams p) {
   using E = Elem<DT>;
   constexpr int VEC = E::kVec;
   constexpr int NV = kEPT / VEC;
   constexpr uint32_t TILE_BYTES = kTile * E::kBytes;
+  const float kInf = __uint_as_float(0x7F800000u);
+  const float kFltMax = 3.402823466e38f;
 
   extern __shared__ unsigned char smem_raw[];
   StreamSmem s;
@@ -98,8 +131,10 @@ __global__ void __maxnreg__(112) screen_stream_kernel(const StreamParams p) {
     q += 3 * (size_t)kMaxKC * 8;
     s.key = reinterpret_cast<unsigned long long*>(q);
     q += (size_t)kMaxKC * 8;
-    s.thr = reinterpret_cast<float2*>(q);
-    q += (size_t)kMaxKC * kWarps * 8;
+    s.ptrs = reinterpret_cast<const void**>(q);
+    q += (size_t)kMaxKC * 8;
+    s.thr = reinterpret_cast<float*>(q);
+    q += (size_t)kMaxKC * kWarps * 4;
     s.rel = reinterpret_cast<unsigned int*>(q);
     q += (size_t)kMaxKC * 4;
     s.abort_flag = reinterpret_cast<volatile unsigned int*>(q);
@@ -125,53 +160,60 @@ __global__ void __maxnreg__(112) screen_stream_kernel(const StreamParams p) {
     s.key[i] = 0ull;
     s.rel[i] = 0u;
   }
-  for (int i = tid; i < kMaxKC * kWarps; i += kStreamThreads) s.thr[i] = make_float2(-1.0f, 0.0f);
+  for (int i = tid; i < kMaxKC * kWarps; i += kStreamThreads) s.thr[i] = -1.0f;
   __syncthreads();
 
   const unsigned long long nitems = (unsigned long long)p.nchunks * p.ntiles;
 
   if (warp == kWarps) {
     // ------------------------------ producer ------------------------------
-    if (lane == 0) {
-      const uint64_t pol_first = l2_policy_evict_first();
-      const uint64_t pol_last = l2_policy_evict_last();
-      uint32_t stage = 0, phase = 0;   // phase of the ring pass being filled
-      unsigned long long issued = 0;
-      bool ok = true;
-      for (unsigned long long item = blockIdx.x; ok && item < nitems; item += gridDim.x) {
-        const uint32_t chunk = (uint32_t)(item / p.ntiles);
-        const uint32_t slot = (uint32_t)(item % p.ntiles);
-        const uint32_t tile = p.tile_list ? p.tile_list[slot] : slot;
-        const uint32_t k0 = chunk * p.KC;
-        const int kc = (int)min(p.KC, p.K - k0);
-        const size_t off = (size_t)tile * TILE_BYTES;
-        for (int kk = -1; kk < kc; ++kk) {
-          if (!mbar_wait_bounded(&s.empty[stage], phase ^ 1u, s.abort_flag, p.status)) {
-            ok = false;
-            break;
-          }
-          const unsigned char* src =
-              reinterpret_cast<const unsigned char*>(kk < 0 ? p.ref : p.cands[k0 + kk]) + off;
-          mbar_arrive_expect_tx(&s.full[stage], TILE_BYTES);
-          bulk_g2s(s.buf + (size_t)stage * TILE_BYTES, src, TILE_BYTES, &s.full[stage],
-                   (kk < 0 && p.nchunks > 1) ? pol_last : pol_first);
-          ++issued;
-          if (++stage == stages) {
-            stage = 0;
-            phase ^= 1u;
-          }
+    const uint64_t pol_first = l2_policy_evict_first();
+    const uint64_t pol_last = l2_policy_evict_last();
+    uint32_t stage = 0, phase = 0;   // phase of the ring pass being filled
+    unsigned long long issued = 0;
+    bool ok = true;
+    int cur_chunk = -1;
+    for (unsigned long long item = blockIdx.x; item < nitems; item += gridDim.x) {
+      const uint32_t chunk = (uint32_t)(item / p.ntiles);
+      const uint32_t slot = (uint32_t)(item % p.ntiles);
+      const uint32_t k0 = chunk * p.KC;
+      const int kc = (int)min(p.KC, p.K - k0);
+      if ((int)chunk != cur_chunk) {
+        // the chunk's candidate pointers go to shared memory once (whole warp)
+        cur_chunk = (int)chunk;
+        __syncwarp();
+        for (int i = lane; i < kc; i += 32) s.ptrs[i] = p.cands[k0 + i];
+        __syncwarp();
+      }
+      if (lane != 0 || !ok) continue;
+      const uint32_t tile = p.tile_list ? p.tile_list[slot] : slot;
+      const size_t off = (size_t)tile * TILE_BYTES;
+      for (int kk = -1; kk < kc; ++kk) {
+        if (!mbar_wait_bounded(&s.empty[stage], phase ^ 1u, s.abort_flag, p.status)) {
+          ok = false;
+          break;
+        }
+        const unsigned char* src =
+            reinterpret_cast<const unsigned char*>(kk < 0 ? p.ref : s.ptrs[kk]) + off;
+        mbar_arrive_expect_tx(&s.full[stage], TILE_BYTES);
+        bulk_g2s(s.buf + (size_t)stage * TILE_BYTES, src, TILE_BYTES, &s.full[stage],
+                 (kk < 0 && p.nchunks > 1) ? pol_last : pol_first);
+        ++issued;
+        if (++stage == stages) {
+          stage = 0;
+          phase ^= 1u;
         }
       }
-      if (!ok) {
-        // Gave up: let every copy already issued land before the CTA may exit.
-        const unsigned long long back = issued < stages ? issued : stages;
-        for (unsigned long long m = issued - back; m < issued; ++m) {
-          uint64_t* bar = &s.full[m % stages];
-          const uint32_t par = (uint32_t)((m / stages) & 1ull);
-          const unsigned long long t0 = global_ns();
-          while (!mbar_try_wait(bar, par)) {
-            if (global_ns() - t0 > 1000000000ull) break;
-          }
+    }
+    if (lane == 0 && !ok) {
+      // Gave up: let every copy already issued land before the CTA may exit.
+      const unsigned long long back = issued < stages ? issued : stages;
+      for (unsigned long long m = issued - back; m < issued; ++m) {
+        uint64_t* bar = &s.full[m % stages];
+        const uint32_t par = (uint32_t)((m / stages) & 1ull);
+        const unsigned long long t0 = global_ns();
+        while (!mbar_try_wait(bar, par)) {
+          if (global_ns() - t0 > 1000000000ull) break;
         }
       }
     }
@@ -202,7 +244,7 @@ __global__ void __maxnreg__(112) screen_stream_kernel(const StreamParams p) {
         s.key[i] = 0ull;
         s.rel[i] = 0u;
       }
-      for (int i = tid; i < kMaxKC * kWarps; i += kConsumers) s.thr[i] = make_float2(-1.0f, 0.0f);
+      for (int i = tid; i < kMaxKC * kWarps; i += kConsumers) s.thr[i] = -1.0f;
       consumers_sync();
     };
 
@@ -220,9 +262,9 @@ __global__ void __maxnreg__(112) screen_stream_kernel(const StreamParams p) {
       const unsigned long long tile_base = (unsigned long long)tile * kTile;
 
       // ---- reference tile: 16 elements per thread stay in registers ----
-      float r[kEPT], tolc[kEPT];
-      bool extreme = false;   // a reference magnitude so small or large that the filter's
-                              // product could underflow: such threads always go exact
+      float r[kEPT];
+      bool extreme = false;   // 0 < |r| < 2^-100: the fused multiply-add of the filter could
+                              // underflow to zero and lose its sign; such threads go exact
       {
         if (!mbar_wait_bounded(&s.full[stage], phase, s.abort_flag, p.status)) {
           ok = false;
@@ -243,14 +285,14 @@ __global__ void __maxnreg__(112) screen_stream_kernel(const StreamParams p) {
 #pragma unroll
         for (int e = 0; e < kEPT; ++e) {
           const float ar = fabsf(r[e]);
-          tolc[e] = tol_clamped(r[e], p.atol, p.rtol);
-          extreme |= (ar > 0.0f && ar < 7.888609052e-31f) || (ar > 1.267650600e30f && ar <= 3.402823466e38f);
+          extreme |= (ar > 0.0f && ar < 7.888609052e-31f);
         }
       }
 
       // ---- the candidates of this chunk against the tile in registers ----
       for (int kk = 0; kk < cur_kc; ++kk) {
-        const float2 th = s.thr[kk * kWarps + warp];
+        const float rel = __uint_as_float(*reinterpret_cast<volatile unsigned int*>(&s.rel[kk]));
+        const float th = s.thr[kk * kWarps + warp];
         if (!mbar_wait_bounded(&s.full[stage], phase, s.abort_flag, p.status)) {
           ok = false;
           break;
@@ -270,97 +312,76 @@ __global__ void __maxnreg__(112) screen_stream_kernel(const StreamParams p) {
 #pragma unroll
         for (int j = 0; j < NV; ++j) E::decode(w[j], &c[j * VEC]);
 
-        // Filter: three running quantities per thread, no branches.
         bool bad = false;
         float mabs = 0.0f, mrel = 0.0f;
+        if (rel <= p.rtol_lean) {
+          // lean filter: (b) and (c); (a) is implied
 #pragma unroll
-        for (int e = 0; e < kEPT; ++e) {
-          const float ad = fabsf(__fsub_rn(c[e], r[e]));
-          bad |= !(ad <= tolc[e]);                    // also true for NaN / Inf differences
-          mabs = fmaxf(mabs, ad);                     // fmaxf drops NaN operands
-          // sign of (ad - thr*|r|): positive iff ad/|r| may exceed the running maximum
-          mrel = fmaxf(mrel, fmaf(-th.y, fabsf(r[e]), ad));
+          for (int e = 0; e < kEPT; e += 2) {
+            const float ad0 = fabsf(__fsub_rn(c[e], r[e]));
+            const float ad1 = fabsf(__fsub_rn(c[e + 1], r[e + 1]));
+            const float t0 = fmaf(-rel, fabsf(r[e]), ad0);
+            const float t1 = fmaf(-rel, fabsf(r[e + 1]), ad1);
+            mabs = max3(mabs, ad0, ad1);
+            mrel = max3_nan(mrel, t0, t1);
+          }
+        } else {
+#pragma unroll
+          for (int e = 0; e < kEPT; ++e) {
+            const float ad = fabsf(__fsub_rn(c[e], r[e]));
+            const float tol = __fadd_rn(p.atol, __fmul_rn(p.rtol, fabsf(r[e])));
+            bad |= !(ad <= tol);      // an infinite ad with an infinite tol is caught by (b)
+            mabs = fmaxf(mabs, ad);
+            mrel = max2_nan(mrel, fmaf(-rel, fabsf(r[e]), ad));
+          }
         }
-        const bool trig_b = mabs > th.x;
-        const bool trig_c = (mrel > 0.0f) || extreme;
-        const unsigned int any_a = __ballot_sync(0xFFFFFFFFu, bad);
-        const unsigned int any_b = __ballot_sync(0xFFFFFFFFu, trig_b);
-        const unsigned int any_c = __ballot_sync(0xFFFFFFFFu, trig_c);
-        if ((any_a | any_b | any_c) == 0u) continue;
+        const bool trig = bad || (mabs > th) || !(mrel <= 0.0f) || extreme;
+        if (!__any_sync(0xFFFFFFFFu, trig)) continue;
 
-        // ---- exact slow path (warp-uniform entry) ----
-        if (any_a) {
-          unsigned int n_mis = 0, n_nan = 0, n_inf = 0;
-          if (bad) {
+        // ---- exact path: every element of a triggered thread by the definition ----
+        unsigned int n_mis = 0, n_nan = 0, n_inf = 0, qb = 0u;
+        unsigned long long best = 0ull;
+        if (trig) {
 #pragma unroll
-            for (int e = 0; e < kEPT; ++e) {
-              const float ad = fabsf(__fsub_rn(c[e], r[e]));
-              const bool match = (c[e] == r[e]) || (ad <= tolc[e]);
-              n_mis += match ? 0u : 1u;
-              n_nan += (c[e] != c[e]) ? 1u : 0u;
-              n_inf += (fabsf(c[e]) == __uint_as_float(0x7F800000u)) ? 1u : 0u;
-            }
-          }
-          n_mis = warp_add_u32(n_mis);
-          n_nan = warp_add_u32(n_nan);
-          n_inf = warp_add_u32(n_inf);
-          if (lane == 0) {
-            if (n_mis) atomicAdd(&s.cnt[kk], (unsigned long long)n_mis);
-            if (n_nan) atomicAdd(&s.cnt[kMaxKC + kk], (unsigned long long)n_nan);
-            if (n_inf) atomicAdd(&s.cnt[2 * kMaxKC + kk], (unsigned long long)n_inf);
-          }
-        }
-        float2 nth = th;
-        if (any_b) {
-          unsigned long long best = 0ull;
-          if (trig_b) {
-#pragma unroll
-            for (int e = 0; e < kEPT; ++e) {
-              const float ad = fabsf(__fsub_rn(c[e], r[e]));
-              if (is_finite_nonneg(ad)) {
+          for (int e = 0; e < kEPT; ++e) {
+            const float ad = fabsf(__fsub_rn(c[e], r[e]));
+            const float ar = fabsf(r[e]);
+            const float tol = __fadd_rn(p.atol, __fmul_rn(p.rtol, ar));
+            const bool fin = ad <= kFltMax;
+            const bool match = (c[e] == r[e]) || (fin && ad <= tol);
+            n_mis += match ? 0u : 1u;
+            n_nan += (c[e] != c[e]) ? 1u : 0u;
+            n_inf += (fabsf(c[e]) == kInf) ? 1u : 0u;
+            if (fin) {
+              if (ad > th) {
                 const unsigned long long idx =
                     tile_base + (unsigned long long)((tid + kConsumers * (e / VEC)) * VEC + (e % VEC));
                 const unsigned long long kv = pack_key(ad, idx);
                 best = kv > best ? kv : best;
               }
-            }
-          }
-          best = warp_max_u64(best);
-          if (best != 0ull) {
-            if (lane == 0) atomicMax(&s.key[kk], best);
-            nth.x = fmaxf(nth.x, __uint_as_float((unsigned int)((best - 1ull) >> 32)));
-          }
-        }
-        if (any_c) {
-          unsigned int qb = 0u;
-          if (trig_c) {
-#pragma unroll
-            for (int e = 0; e < kEPT; ++e) {
-              const float ad = fabsf(__fsub_rn(c[e], r[e]));
-              const float ar = fabsf(r[e]);
-              if ((extreme || fmaf(-th.y, ar, ad) > 0.0f) && is_finite_nonneg(ad) && ar > 0.0f &&
-                  is_finite_nonneg(ar)) {
+              if (ar > 0.0f && ar <= kFltMax && (extreme || fmaf(-rel, ar, ad) > 0.0f)) {
                 const unsigned int q = __float_as_uint(__fdiv_rn(ad, ar));
                 qb = q > qb ? q : qb;
               }
             }
           }
-          qb = warp_max_u32(qb);
-          if (qb != 0u) {
-            unsigned int cur = qb;
-            if (lane == 0) {
-              const unsigned int old = atomicMax(&s.rel[kk], qb);
-              cur = old > qb ? old : qb;
-            }
-            cur = __shfl_sync(0xFFFFFFFFu, cur, 0);
-            // The running maximum itself is the threshold: a quotient that rounds
-            // above it is above it as a real number, so ad - thr*|r| > 0 exactly
-            // (the fused multiply-add rounds once and keeps the sign); an exact
-            // tie gives 0 and does not fire.
-            nth.y = fmaxf(nth.y, __uint_as_float(cur));
-          }
         }
-        if (lane == 0) s.thr[kk * kWarps + warp] = nth;
+        n_mis = warp_add_u32(n_mis);
+        n_nan = warp_add_u32(n_nan);
+        n_inf = warp_add_u32(n_inf);
+        best = warp_max_u64(best);
+        qb = warp_max_u32(qb);
+        if (lane == 0) {
+          if (n_mis) atomicAdd(&s.cnt[kk], (unsigned long long)n_mis);
+          if (n_nan) atomicAdd(&s.cnt[kMaxKC + kk], (unsigned long long)n_nan);
+          if (n_inf) atomicAdd(&s.cnt[2 * kMaxKC + kk], (unsigned long long)n_inf);
+          if (best != 0ull) {
+            atomicMax(&s.key[kk], best);
+            // everything this warp meets in later tiles with an error <= this one loses
+            s.thr[kk * kWarps + warp] = fmaxf(th, __uint_as_float((unsigned int)((best - 1ull) >> 32)));
+          }
+          if (qb > __float_as_uint(rel)) atomicMax(&s.rel[kk], qb);
+        }
         __syncwarp();
       }
     }
