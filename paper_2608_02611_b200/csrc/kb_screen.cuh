@@ -83,6 +83,7 @@ struct StreamSmem {
   const void** ptrs;         // [kMaxKC] candidate pointers of the current chunk (producer only)
   unsigned int* rel;         // [kMaxKC] bits of the running max relative error (CTA-wide)
   float* thr;                // [kMaxKC][kWarps] running max |c-r| seen by each warp (-1: none)
+  float* gth;                // [kMaxKC] a value strictly below an error some CTA has recorded (-1: none)
   volatile unsigned int* abort_flag;
 };
 
@@ -90,7 +91,7 @@ __host__ __device__ inline size_t stream_smem_bytes(uint32_t stages, uint32_t ti
   size_t b = (size_t)stages * tile_bytes;
   b += 2 * (size_t)stages * 8;
   b += 3 * (size_t)kMaxKC * 8 + (size_t)kMaxKC * 8 + (size_t)kMaxKC * 8 + (size_t)kMaxKC * 4;
-  b += (size_t)kMaxKC * kWarps * 4;
+  b += (size_t)kMaxKC * kWarps * 4 + (size_t)kMaxKC * 4;
   b += 16;
   return b + 128;  // alignment slack
 }
@@ -135,6 +136,8 @@ __global__ void __maxnreg__(96) screen_stream_kernel(const StreamParams p) {
     q += (size_t)kMaxKC * 8;
     s.thr = reinterpret_cast<float*>(q);
     q += (size_t)kMaxKC * kWarps * 4;
+    s.gth = reinterpret_cast<float*>(q);
+    q += (size_t)kMaxKC * 4;
     s.rel = reinterpret_cast<unsigned int*>(q);
     q += (size_t)kMaxKC * 4;
     s.abort_flag = reinterpret_cast<volatile unsigned int*>(q);
@@ -159,6 +162,7 @@ __global__ void __maxnreg__(96) screen_stream_kernel(const StreamParams p) {
     s.cnt[2 * kMaxKC + i] = 0ull;
     s.key[i] = 0ull;
     s.rel[i] = 0u;
+    s.gth[i] = -1.0f;
   }
   for (int i = tid; i < kMaxKC * kWarps; i += kStreamThreads) s.thr[i] = -1.0f;
   __syncthreads();
@@ -244,6 +248,7 @@ __global__ void __maxnreg__(96) screen_stream_kernel(const StreamParams p) {
         s.key[i] = 0ull;
         s.rel[i] = 0u;
       }
+      for (int i = tid; i < kMaxKC; i += kConsumers) s.gth[i] = -1.0f;
       for (int i = tid; i < kMaxKC * kWarps; i += kConsumers) s.thr[i] = -1.0f;
       consumers_sync();
     };
@@ -260,6 +265,19 @@ __global__ void __maxnreg__(96) screen_stream_kernel(const StreamParams p) {
       }
       if (!ok) continue;
       const unsigned long long tile_base = (unsigned long long)tile * kTile;
+
+      // ---- exchange running maxima with the other CTAs (all merges are maxima, so this
+      // needs no ordering): push this CTA's, pull everyone's; applied after the tile load ----
+      const int xkk = warp + kWarps * lane;          // each candidate of the chunk has one owner lane
+      unsigned long long xmine_k = 0ull, xold_k = 0ull;
+      unsigned int xmine_r = 0u, xold_r = 0u;
+      if (xkk < cur_kc) {
+        xmine_k = *reinterpret_cast<volatile unsigned long long*>(&s.key[xkk]);
+        xmine_r = *reinterpret_cast<volatile unsigned int*>(&s.rel[xkk]);
+        Acc* a = &p.acc[cur_k0 + xkk];
+        xold_k = atomicMax(&a->key, xmine_k);
+        xold_r = atomicMax(&a->rel, xmine_r);
+      }
 
       // ---- reference tile: 16 elements per thread stay in registers ----
       float r[kEPT];
@@ -288,11 +306,22 @@ __global__ void __maxnreg__(96) screen_stream_kernel(const StreamParams p) {
           extreme |= (ar > 0.0f && ar < 7.888609052e-31f);
         }
       }
+      if (xkk < cur_kc) {
+        if (xold_r > xmine_r) atomicMax(&s.rel[xkk], xold_r);
+        const unsigned long long gk = xold_k > xmine_k ? xold_k : xmine_k;
+        if (gk != 0ull) {
+          // an error strictly below a recorded one can never become the maximum
+          const unsigned int db = (unsigned int)((gk - 1ull) >> 32);
+          s.gth[xkk] = db ? __uint_as_float(db - 1u) : -1.0f;
+        }
+      }
+      __syncwarp();
 
       // ---- the candidates of this chunk against the tile in registers ----
       for (int kk = 0; kk < cur_kc; ++kk) {
         const float rel = __uint_as_float(*reinterpret_cast<volatile unsigned int*>(&s.rel[kk]));
-        const float th = s.thr[kk * kWarps + warp];
+        const float th_own = s.thr[kk * kWarps + warp];
+        const float th = fmaxf(th_own, *reinterpret_cast<volatile float*>(&s.gth[kk]));
         if (!mbar_wait_bounded(&s.full[stage], phase, s.abort_flag, p.status)) {
           ok = false;
           break;
@@ -338,7 +367,9 @@ __global__ void __maxnreg__(96) screen_stream_kernel(const StreamParams p) {
         const bool trig = bad || (mabs > th) || !(mrel <= 0.0f) || extreme;
         if (!__any_sync(0xFFFFFFFFu, trig)) continue;
 
-        // ---- exact path: every element of a triggered thread by the definition ----
+        // ---- exact path.  A triggered thread re-tests each of its elements and
+        // evaluates by the definition those that could matter ("hot"). ----
+        const bool lean = rel <= p.rtol_lean;
         unsigned int n_mis = 0, n_nan = 0, n_inf = 0, qb = 0u;
         unsigned long long best = 0ull;
         if (trig) {
@@ -346,22 +377,27 @@ __global__ void __maxnreg__(96) screen_stream_kernel(const StreamParams p) {
           for (int e = 0; e < kEPT; ++e) {
             const float ad = fabsf(__fsub_rn(c[e], r[e]));
             const float ar = fabsf(r[e]);
-            const float tol = __fadd_rn(p.atol, __fmul_rn(p.rtol, ar));
-            const bool fin = ad <= kFltMax;
-            const bool match = (c[e] == r[e]) || (fin && ad <= tol);
-            n_mis += match ? 0u : 1u;
-            n_nan += (c[e] != c[e]) ? 1u : 0u;
-            n_inf += (fabsf(c[e]) == kInf) ? 1u : 0u;
-            if (fin) {
-              if (ad > th) {
-                const unsigned long long idx =
-                    tile_base + (unsigned long long)((tid + kConsumers * (e / VEC)) * VEC + (e % VEC));
-                const unsigned long long kv = pack_key(ad, idx);
-                best = kv > best ? kv : best;
-              }
-              if (ar > 0.0f && ar <= kFltMax && (extreme || fmaf(-rel, ar, ad) > 0.0f)) {
-                const unsigned int q = __float_as_uint(__fdiv_rn(ad, ar));
-                qb = q > qb ? q : qb;
+            const float t = fmaf(-rel, ar, ad);
+            bool hot = !(ad <= th) || !(t <= 0.0f) || extreme;
+            if (!lean) hot = hot || !(ad <= __fadd_rn(p.atol, __fmul_rn(p.rtol, ar)));
+            if (hot) {
+              const float tol = __fadd_rn(p.atol, __fmul_rn(p.rtol, ar));
+              const bool fin = ad <= kFltMax;
+              const bool match = (c[e] == r[e]) || (fin && ad <= tol);
+              n_mis += match ? 0u : 1u;
+              n_nan += (c[e] != c[e]) ? 1u : 0u;
+              n_inf += (fabsf(c[e]) == kInf) ? 1u : 0u;
+              if (fin) {
+                if (ad > th) {
+                  const unsigned long long idx =
+                      tile_base + (unsigned long long)((tid + kConsumers * (e / VEC)) * VEC + (e % VEC));
+                  const unsigned long long kv = pack_key(ad, idx);
+                  best = kv > best ? kv : best;
+                }
+                if (ar > 0.0f && ar <= kFltMax && (extreme || t > 0.0f)) {
+                  const unsigned int q = __float_as_uint(__fdiv_rn(ad, ar));
+                  qb = q > qb ? q : qb;
+                }
               }
             }
           }
@@ -378,7 +414,7 @@ __global__ void __maxnreg__(96) screen_stream_kernel(const StreamParams p) {
           if (best != 0ull) {
             atomicMax(&s.key[kk], best);
             // everything this warp meets in later tiles with an error <= this one loses
-            s.thr[kk * kWarps + warp] = fmaxf(th, __uint_as_float((unsigned int)((best - 1ull) >> 32)));
+            s.thr[kk * kWarps + warp] = fmaxf(th_own, __uint_as_float((unsigned int)((best - 1ull) >> 32)));
           }
           if (qb > __float_as_uint(rel)) atomicMax(&s.rel[kk], qb);
         }
