@@ -312,7 +312,7 @@ __global__ void __maxnreg__(96) screen_stream_kernel(const StreamParams p) {
         if (gk != 0ull) {
           // an error strictly below a recorded one can never become the maximum
           const unsigned int db = (unsigned int)((gk - 1ull) >> 32);
-          s.gth[xkk] = db ? __uint_as_float(db - 1u) : -1.0f;
+          if (db) atomicMax(reinterpret_cast<int*>(&s.gth[xkk]), (int)(db - 1u));
         }
       }
       __syncwarp();
@@ -367,39 +367,43 @@ __global__ void __maxnreg__(96) screen_stream_kernel(const StreamParams p) {
         const bool trig = bad || (mabs > th) || !(mrel <= 0.0f) || extreme;
         if (!__any_sync(0xFFFFFFFFu, trig)) continue;
 
-        // ---- exact path.  A triggered thread re-tests each of its elements and
-        // evaluates by the definition those that could matter ("hot"). ----
+        // ---- exact path.  A triggered thread finds its largest finite error (first
+        // index on ties) with a running compare, and evaluates by the definition the
+        // elements that fail the tolerance / relative-error filter or are not finite. ----
         const bool lean = rel <= p.rtol_lean;
         unsigned int n_mis = 0, n_nan = 0, n_inf = 0, qb = 0u;
         unsigned long long best = 0ull;
         if (trig) {
+          float m = -1.0f;
+          int mi = 0;
 #pragma unroll
           for (int e = 0; e < kEPT; ++e) {
             const float ad = fabsf(__fsub_rn(c[e], r[e]));
             const float ar = fabsf(r[e]);
             const float t = fmaf(-rel, ar, ad);
-            bool hot = !(ad <= th) || !(t <= 0.0f) || extreme;
+            const bool fin = ad <= kFltMax;
+            if (fin && ad > m) {
+              m = ad;
+              mi = e;
+            }
+            bool hot = !(t <= 0.0f) || !fin || extreme;
             if (!lean) hot = hot || !(ad <= __fadd_rn(p.atol, __fmul_rn(p.rtol, ar)));
             if (hot) {
               const float tol = __fadd_rn(p.atol, __fmul_rn(p.rtol, ar));
-              const bool fin = ad <= kFltMax;
               const bool match = (c[e] == r[e]) || (fin && ad <= tol);
               n_mis += match ? 0u : 1u;
               n_nan += (c[e] != c[e]) ? 1u : 0u;
               n_inf += (fabsf(c[e]) == kInf) ? 1u : 0u;
-              if (fin) {
-                if (ad > th) {
-                  const unsigned long long idx =
-                      tile_base + (unsigned long long)((tid + kConsumers * (e / VEC)) * VEC + (e % VEC));
-                  const unsigned long long kv = pack_key(ad, idx);
-                  best = kv > best ? kv : best;
-                }
-                if (ar > 0.0f && ar <= kFltMax && (extreme || t > 0.0f)) {
-                  const unsigned int q = __float_as_uint(__fdiv_rn(ad, ar));
-                  qb = q > qb ? q : qb;
-                }
+              if (fin && ar > 0.0f && ar <= kFltMax && (extreme || t > 0.0f)) {
+                const unsigned int q = __float_as_uint(__fdiv_rn(ad, ar));
+                qb = q > qb ? q : qb;
               }
             }
+          }
+          if (m > th) {
+            const unsigned long long idx =
+                tile_base + (unsigned long long)((tid + kConsumers * (mi / VEC)) * VEC + (mi % VEC));
+            best = pack_key(m, idx);
           }
         }
         n_mis = warp_add_u32(n_mis);
@@ -413,8 +417,11 @@ __global__ void __maxnreg__(96) screen_stream_kernel(const StreamParams p) {
           if (n_inf) atomicAdd(&s.cnt[2 * kMaxKC + kk], (unsigned long long)n_inf);
           if (best != 0ull) {
             atomicMax(&s.key[kk], best);
-            // everything this warp meets in later tiles with an error <= this one loses
-            s.thr[kk * kWarps + warp] = fmaxf(th_own, __uint_as_float((unsigned int)((best - 1ull) >> 32)));
+            // everything this warp meets in later tiles with an error <= this one loses ...
+            const unsigned int db = (unsigned int)((best - 1ull) >> 32);
+            s.thr[kk * kWarps + warp] = fmaxf(th_own, __uint_as_float(db));
+            // ... and anything strictly below it loses for every warp
+            if (db) atomicMax(reinterpret_cast<int*>(&s.gth[kk]), (int)(db - 1u));
           }
           if (qb > __float_as_uint(rel)) atomicMax(&s.rel[kk], qb);
         }
