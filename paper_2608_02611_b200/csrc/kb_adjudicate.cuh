@@ -10,8 +10,11 @@
 //                     warp owns one b row and each lane keeps up to 8 of its
 //                     samples in registers.  Per sample pair the work is two
 //                     compares that yield 0 / -1 and one three-input add.
-//                     Partial counts are merged with integer atomics.
-// wins_mirror_kernel  W[b][a] = 2*S*S - W[a][b] for the block-lower triangle.
+//                     When a pair's samples fit one chunk each entry has a
+//                     single writer (plain stores); otherwise partial counts
+//                     are merged with integer atomics into a zeroed matrix.
+//                     The mirrored entry W[b][a] = 2*S*S - W[a][b] is written by
+//                     the same warp (the complement is additive over chunks).
 #pragma once
 
 #include "kb_common.cuh"
@@ -84,10 +87,12 @@ struct WinsParams {
   const float* timings;
   unsigned int* wins;
   unsigned int K, S;
-  unsigned int KB;      // ceil(K / 8)
+  unsigned int KB;      // ceil(K / 8) blocks of 8 rows
   unsigned int npairs;  // KB*(KB+1)/2 block pairs, diagonal included
+  unsigned int TA;      // a rows per CTA (1, 2, 4 or 8); 8/TA CTAs share one block pair
   unsigned int nj, JC;  // b-sample chunks and their length (JC = 32*R)
   unsigned int ni, IC;  // a-sample chunks and their length (multiple of 4)
+  unsigned int direct;  // 1: each entry has one writer (ni == nj == 1): plain stores, no zeroing
 };
 
 // cnt += [a < b] + [a <= b]  (= 2*[a<b] + [a==b]); NaN padding compares false.
@@ -100,13 +105,16 @@ __device__ __forceinline__ void count_pair(unsigned int& cnt, float a, float b) 
 
 template <int R>
 __global__ void __launch_bounds__(kWinsThreads) wins_kernel(const WinsParams p) {
-  extern __shared__ float as[];   // [8][IC]
+  extern __shared__ float as[];   // [TA][IC]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   unsigned int item = blockIdx.x;
   const unsigned int ic = item % p.ni;
   item /= p.ni;
   const unsigned int jc = item % p.nj;
-  const unsigned int pair = item / p.nj;
+  item /= p.nj;
+  const unsigned int nsub = kWinsRowsPerBlock / p.TA;
+  const unsigned int sub = item % nsub;
+  const unsigned int pair = item / nsub;
   // block pair index -> (Ab <= Bb): row-major upper triangle
   unsigned int Ab = 0, rem = pair;
   while (rem >= p.KB - Ab) {
@@ -116,26 +124,30 @@ __global__ void __launch_bounds__(kWinsThreads) wins_kernel(const WinsParams p) 
   const unsigned int Bb = Ab + rem;
   const float qnan = __uint_as_float(0x7FC00000u);
 
-  // stage the a-chunk: rows Ab*8 .. Ab*8+7, samples ic*IC .. +IC
+  // stage the a-chunk: TA rows from Ab*8 + sub*TA, samples ic*IC .. +IC
+  const unsigned int a0 = Ab * kWinsRowsPerBlock + sub * p.TA;
   const unsigned int i0 = ic * p.IC;
-  for (unsigned int t = threadIdx.x; t < kWinsRowsPerBlock * p.IC; t += kWinsThreads) {
+  for (unsigned int t = threadIdx.x; t < p.TA * p.IC; t += kWinsThreads) {
     const unsigned int rr = t / p.IC, ii = t % p.IC;
-    const unsigned int a = Ab * kWinsRowsPerBlock + rr, i = i0 + ii;
+    const unsigned int a = a0 + rr, i = i0 + ii;
     as[t] = (a < p.K && i < p.S) ? p.timings[(size_t)a * p.S + i] : qnan;
   }
   // this warp's b row, this lane's samples
   const unsigned int b = Bb * kWinsRowsPerBlock + warp;
+  const unsigned int j0 = jc * p.JC;
   float bv[R];
 #pragma unroll
   for (int m = 0; m < R; ++m) {
-    const unsigned int j = jc * p.JC + lane + 32 * m;
+    const unsigned int j = j0 + lane + 32 * m;
     bv[m] = (b < p.K && j < p.S) ? p.timings[(size_t)b * p.S + j] : qnan;
   }
   __syncthreads();
   if (b >= p.K) return;
+  const unsigned int ilen = min(p.IC, p.S - i0);
+  const unsigned int jlen = min(p.JC, p.S - j0);
 
-  for (int rr = 0; rr < kWinsRowsPerBlock; ++rr) {
-    const unsigned int a = Ab * kWinsRowsPerBlock + rr;
+  for (unsigned int rr = 0; rr < p.TA; ++rr) {
+    const unsigned int a = a0 + rr;
     if (a >= p.K) break;
     unsigned int cnt[R];
 #pragma unroll
@@ -157,16 +169,20 @@ __global__ void __launch_bounds__(kWinsThreads) wins_kernel(const WinsParams p) 
 #pragma unroll
     for (int m = 0; m < R; ++m) total += cnt[m];
     total = warp_add_u32(total);
-    if (lane == 0 && total != 0u) atomicAdd(&p.wins[(size_t)a * p.K + b], total);
+    if (lane == 0) {
+      // W[b][a] = 2*S*S - W[a][b]; over chunks the complement is additive as well
+      const unsigned int mirror = 2u * ilen * jlen - total;
+      unsigned int* wab = &p.wins[(size_t)a * p.K + b];
+      unsigned int* wba = &p.wins[(size_t)b * p.K + a];
+      if (p.direct) {
+        *wab = total;
+        if (Ab != Bb) *wba = mirror;
+      } else {
+        if (total) atomicAdd(wab, total);
+        if (Ab != Bb && mirror) atomicAdd(wba, mirror);
+      }
+    }
   }
-}
-
-__global__ void wins_mirror_kernel(unsigned int* __restrict__ wins, unsigned int K, unsigned int S) {
-  const unsigned int b = blockIdx.x * blockDim.x + threadIdx.x;   // column
-  const unsigned int a = blockIdx.y;                              // row
-  if (a >= K || b >= K) return;
-  if ((a / kWinsRowsPerBlock) > (b / kWinsRowsPerBlock))
-    wins[(size_t)a * K + b] = 2u * S * S - wins[(size_t)b * K + a];
 }
 
 }  // namespace kb

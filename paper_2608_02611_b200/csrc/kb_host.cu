@@ -486,11 +486,10 @@ kb_status screen_impl(kb_ctx* ctx, const void* d_ref, const void* const* h_cands
     PtrChunk ch;
     const uint32_t cnt = (K - off < (uint32_t)kPtrsPerLaunch) ? K - off : (uint32_t)kPtrsPerLaunch;
     memcpy(ch.p, h_cands + off, cnt * sizeof(void*));
-    upload_ptrs_kernel<<<(cnt + 127) / 128, 128, 0, st>>>(ch, table, off, cnt);
+    screen_prep_kernel<<<(cnt + 127) / 128, 128, 0, st>>>(ch, table, acc, ctx->d_status + 1, off, cnt);
     ++ctx->launches;
     KB_CUDA(ctx, cudaGetLastError());
   }
-  KB_CUDA(ctx, cudaMemsetAsync(acc, 0, (size_t)K * sizeof(Acc), st));
 
   MaskDev md;
   md.kind = mask ? mask->kind : 0;
@@ -522,6 +521,24 @@ kb_status screen_impl(kb_ctx* ctx, const void* d_ref, const void* const* h_cands
       sp.rtol_lean = f;
     }
     sp.status = ctx->d_status;
+    // Scout a few leading tiles exactly (about 1% of the work at most); the streaming
+    // kernel starts behind them with its thresholds seeded.
+    uint32_t nscout = 0;
+    if (sp.ntiles >= 2) {
+      nscout = sp.ntiles / 128;
+      if (nscout < 1) nscout = 1;
+      if (nscout > 8) nscout = 8;
+      dim3 sg(nscout * (kTile / 256), K);
+      screen_scout_kernel<DT><<<sg, 256, 0, st>>>(d_ref, table, acc, sp.tile_list, atol, rtol);
+      ++ctx->launches;
+      KB_CUDA(ctx, cudaGetLastError());
+    }
+    sp.slot0 = nscout;
+    sp.ntiles -= nscout;
+    // ragged tail (elements past the last full kernel tile), before the streaming
+    // kernel so that its last CTA can unpack the finished records
+    rc = launch_generic<DT>(ctx, d_ref, table, acc, K, nfull * kTile, N, atol, rtol, md, st);
+    if (rc != KB_OK) return rc;
     if (sp.ntiles) {
       // chunk the candidates: shared-memory accumulators hold kMaxKC of them, and
       // small tensors need more, smaller items to fill the machine
@@ -536,12 +553,10 @@ kb_status screen_impl(kb_ctx* ctx, const void* d_ref, const void* const* h_cands
       }
       sp.KC = (K + nchunks - 1) / nchunks;
       sp.nchunks = (K + sp.KC - 1) / sp.KC;
-      rc = launch_stream<DT>(ctx, sp, st);
-      if (rc != KB_OK) return rc;
+      sp.done = ctx->d_status + 1;
+      sp.out = d_out;
+      return launch_stream<DT>(ctx, sp, st);
     }
-    // ragged tail (elements past the last full kernel tile)
-    rc = launch_generic<DT>(ctx, d_ref, table, acc, K, nfull * kTile, N, atol, rtol, md, st);
-    if (rc != KB_OK) return rc;
   }
   screen_finalize_kernel<<<(K + 127) / 128, 128, 0, st>>>(acc, d_out, K);
   ++ctx->launches;
@@ -653,7 +668,6 @@ extern "C" kb_status kb_adjudicate(kb_ctx* ctx, const float* d_timings, uint32_t
   KB_CUDA(ctx, cudaGetLastError());
   if (!d_wins) return KB_OK;
 
-  KB_CUDA(ctx, cudaMemsetAsync(d_wins, 0, (size_t)K * K * sizeof(uint32_t), st));
   WinsParams wp;
   wp.timings = d_timings;
   wp.wins = d_wins;
@@ -668,35 +682,34 @@ extern "C" kb_status kb_adjudicate(kb_ctx* ctx, const float* d_timings, uint32_t
   wp.JC = 32u * R;
   wp.IC = (unsigned int)round_up(S < 1024 ? S : 1024, 4);
   wp.ni = (S + wp.IC - 1) / wp.IC;
-  while (npairs * wp.nj * wp.ni < 2ull * ctx->sm_count && wp.IC > 64) {
+  // small problems: fewer a rows per CTA, then shorter a chunks, until the machine is filled
+  wp.TA = kWinsRowsPerBlock;
+  auto items = [&]() { return npairs * (kWinsRowsPerBlock / wp.TA) * wp.nj * wp.ni; };
+  while (items() < 2ull * ctx->sm_count && wp.TA > 1) wp.TA /= 2;
+  while (items() < (unsigned long long)ctx->sm_count && wp.IC > 256) {
     wp.IC = (unsigned int)round_up((wp.IC + 1) / 2, 4);
     wp.ni = (S + wp.IC - 1) / wp.IC;
   }
-  const unsigned long long items = npairs * wp.nj * wp.ni;
-  if (items > 0x7FFFFFFFull) return fail(ctx, KB_ERR_UNSUPPORTED, "kb_adjudicate: K*S too large for one launch");
-  const size_t smem = (size_t)kWinsRowsPerBlock * wp.IC * sizeof(float);
-  const unsigned int grid = (unsigned int)items;
+  wp.direct = (wp.ni == 1 && wp.nj == 1) ? 1u : 0u;
+  if (items() > 0x7FFFFFFFull) return fail(ctx, KB_ERR_UNSUPPORTED, "kb_adjudicate: K*S too large for one launch");
+  if (!wp.direct) KB_CUDA(ctx, cudaMemsetAsync(d_wins, 0, (size_t)K * K * sizeof(uint32_t), st));
+  const size_t smem = (size_t)wp.TA * wp.IC * sizeof(float);
+  const unsigned int grid = (unsigned int)items();
   {
-  ScopedTimer tm(ctx, KB_TIMER_WINS, st);
-  switch (R) {
-    case 1: launch_wins<1>(wp, grid, smem, st); break;
-    case 2: launch_wins<2>(wp, grid, smem, st); break;
-    case 3: launch_wins<3>(wp, grid, smem, st); break;
-    case 4: launch_wins<4>(wp, grid, smem, st); break;
-    case 5: launch_wins<5>(wp, grid, smem, st); break;
-    case 6: launch_wins<6>(wp, grid, smem, st); break;
-    case 7: launch_wins<7>(wp, grid, smem, st); break;
-    default: launch_wins<8>(wp, grid, smem, st); break;
-  }
+    ScopedTimer tm(ctx, KB_TIMER_WINS, st);
+    switch (R) {
+      case 1: launch_wins<1>(wp, grid, smem, st); break;
+      case 2: launch_wins<2>(wp, grid, smem, st); break;
+      case 3: launch_wins<3>(wp, grid, smem, st); break;
+      case 4: launch_wins<4>(wp, grid, smem, st); break;
+      case 5: launch_wins<5>(wp, grid, smem, st); break;
+      case 6: launch_wins<6>(wp, grid, smem, st); break;
+      case 7: launch_wins<7>(wp, grid, smem, st); break;
+      default: launch_wins<8>(wp, grid, smem, st); break;
+    }
   }
   ++ctx->launches;
   KB_CUDA(ctx, cudaGetLastError());
-  if (wp.KB > 1) {
-    dim3 mg((K + 255) / 256, K);
-    wins_mirror_kernel<<<mg, 256, 0, st>>>(d_wins, K, S);
-    ++ctx->launches;
-    KB_CUDA(ctx, cudaGetLastError());
-  }
   return KB_OK;
 }
 

@@ -32,11 +32,14 @@ struct StreamParams {
   Acc* acc;                     // [K], zeroed by the caller
   const uint32_t* tile_list;    // selected full tiles, ascending; NULL: tile = slot
   uint32_t ntiles;              // number of full tiles to visit
+  uint32_t slot0;               // first slot of the tile list / first tile (earlier ones were scouted)
   uint32_t K, KC, nchunks;
   uint32_t stages;
   float atol, rtol;
   float rtol_lean;              // rtol*(1-2^-20) rounded down, or -1: see the lean filter below
   unsigned int* status;
+  unsigned int* done;           // zeroed ticket counter: the last CTA to finish unpacks the records
+  kb_screen_result* out;        // [K]
 };
 
 struct MaskDev {
@@ -54,6 +57,26 @@ __device__ __forceinline__ bool mask_selected(const MaskDev& m, unsigned long lo
 
 __device__ __forceinline__ void consumers_sync() {
   asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory");
+}
+
+// accumulator -> public record
+__device__ __forceinline__ void unpack_record(const Acc& a, kb_screen_result* dst) {
+  kb_screen_result r;
+  r.mismatch_count = a.mism;
+  r.nan_count = a.nan;
+  r.inf_count = a.inf;
+  if (a.key == 0ull) {
+    r.argmax_idx = -1;
+    r.max_abs_err = 0.0f;
+  } else {
+    const unsigned long long kv = a.key - 1ull;
+    r.max_abs_err = __uint_as_float((unsigned int)(kv >> 32));
+    r.argmax_idx = (int64_t)(0xFFFFFFFFu - (unsigned int)kv);
+  }
+  r.max_rel_err = __uint_as_float(a.rel);
+  r.pass = a.mism == 0ull ? 1u : 0u;
+  r.reserved = 0u;
+  *dst = r;
 }
 
 // three-input maxima (one instruction on sm_100); the .NaN form returns NaN if any input is NaN
@@ -167,7 +190,12 @@ __global__ void __maxnreg__(96) screen_stream_kernel(const StreamParams p) {
   for (int i = tid; i < kMaxKC * kWarps; i += kStreamThreads) s.thr[i] = -1.0f;
   __syncthreads();
 
+  // Work items (chunk, tile), chunk-major; each CTA takes one contiguous run of them, so
+  // that it stays with one chunk (warm thresholds) and walks tiles in ascending order.
   const unsigned long long nitems = (unsigned long long)p.nchunks * p.ntiles;
+  const unsigned long long per_cta = (nitems + gridDim.x - 1) / gridDim.x;
+  const unsigned long long item_lo = per_cta * blockIdx.x < nitems ? per_cta * blockIdx.x : nitems;
+  const unsigned long long item_hi = item_lo + per_cta < nitems ? item_lo + per_cta : nitems;
 
   if (warp == kWarps) {
     // ------------------------------ producer ------------------------------
@@ -177,9 +205,9 @@ __global__ void __maxnreg__(96) screen_stream_kernel(const StreamParams p) {
     unsigned long long issued = 0;
     bool ok = true;
     int cur_chunk = -1;
-    for (unsigned long long item = blockIdx.x; item < nitems; item += gridDim.x) {
+    for (unsigned long long item = item_lo; item < item_hi; ++item) {
       const uint32_t chunk = (uint32_t)(item / p.ntiles);
-      const uint32_t slot = (uint32_t)(item % p.ntiles);
+      const uint32_t slot = p.slot0 + (uint32_t)(item % p.ntiles);
       const uint32_t k0 = chunk * p.KC;
       const int kc = (int)min(p.KC, p.K - k0);
       if ((int)chunk != cur_chunk) {
@@ -253,9 +281,9 @@ __global__ void __maxnreg__(96) screen_stream_kernel(const StreamParams p) {
       consumers_sync();
     };
 
-    for (unsigned long long item = blockIdx.x; item < nitems; item += gridDim.x) {
+    for (unsigned long long item = item_lo; item < item_hi; ++item) {
       const uint32_t chunk = (uint32_t)(item / p.ntiles);
-      const uint32_t slot = (uint32_t)(item % p.ntiles);
+      const uint32_t slot = p.slot0 + (uint32_t)(item % p.ntiles);
       const uint32_t tile = p.tile_list ? p.tile_list[slot] : slot;
       if ((int)chunk != cur_chunk) {
         if (cur_chunk >= 0) flush();
@@ -310,9 +338,14 @@ __global__ void __maxnreg__(96) screen_stream_kernel(const StreamParams p) {
         if (xold_r > xmine_r) atomicMax(&s.rel[xkk], xold_r);
         const unsigned long long gk = xold_k > xmine_k ? xold_k : xmine_k;
         if (gk != 0ull) {
-          // an error strictly below a recorded one can never become the maximum
+          // An error equal to one recorded at a lower index, or strictly below one
+          // recorded anywhere, can never become the maximum.
           const unsigned int db = (unsigned int)((gk - 1ull) >> 32);
-          if (db) atomicMax(reinterpret_cast<int*>(&s.gth[xkk]), (int)(db - 1u));
+          const unsigned long long gidx = 0xFFFFFFFFull - ((gk - 1ull) & 0xFFFFFFFFull);
+          if (gidx < tile_base)
+            atomicMax(reinterpret_cast<int*>(&s.gth[xkk]), (int)db);
+          else if (db)
+            atomicMax(reinterpret_cast<int*>(&s.gth[xkk]), (int)(db - 1u));
         }
       }
       __syncwarp();
@@ -430,32 +463,34 @@ __global__ void __maxnreg__(96) screen_stream_kernel(const StreamParams p) {
     }
     if (cur_chunk >= 0) flush();
   }
+  // ---- the last CTA to get here unpacks all K records (saves a launch) ----
+  __shared__ unsigned int s_ticket;
+  __threadfence();
   __syncthreads();
+  if (tid == 0) s_ticket = atomicAdd(p.done, 1u);
+  __syncthreads();
+  if (s_ticket == gridDim.x - 1) {
+    __threadfence();
+    for (unsigned int k = tid; k < p.K; k += kStreamThreads) {
+      Acc a;
+      a.mism = __ldcg(&p.acc[k].mism);
+      a.nan = __ldcg(&p.acc[k].nan);
+      a.inf = __ldcg(&p.acc[k].inf);
+      a.key = __ldcg(&p.acc[k].key);
+      a.rel = __ldcg(&p.acc[k].rel);
+      unpack_record(a, &p.out[k]);
+    }
+  }
 }
 
 // ---------------------------------------------------------------------------
-// Generic path: elements [e0, e1) of every candidate, plain loads, exact
-// classification of each selected element.  grid = (blocks, K).
+// Plain-load kernels: every selected element classified by the definition.
 // ---------------------------------------------------------------------------
-template <int DT>
-__global__ void __launch_bounds__(256) screen_generic_kernel(const void* __restrict__ ref,
-                                                             const void* const* __restrict__ cands,
-                                                             Acc* __restrict__ acc,
-                                                             unsigned long long e0,
-                                                             unsigned long long e1, float atol,
-                                                             float rtol, MaskDev mask) {
-  using E = Elem<DT>;
-  const unsigned int k = blockIdx.y;
-  const void* cand = cands[k];
-  unsigned int n_mis = 0, n_nan = 0, n_inf = 0;
+struct ExactAcc {
+  unsigned int n_mis = 0, n_nan = 0, n_inf = 0, qb = 0;
   unsigned long long best = 0ull;
-  unsigned int qb = 0u;
-  const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
-  for (unsigned long long i = e0 + (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < e1;
-       i += stride) {
-    if (!mask_selected(mask, i)) continue;
-    const float r = E::load(ref, i);
-    const float c = E::load(cand, i);
+
+  __device__ __forceinline__ void add(float r, float c, unsigned long long i, float atol, float rtol) {
     const float ad = fabsf(__fsub_rn(c, r));
     const float tolc = tol_clamped(r, atol, rtol);
     const bool match = (c == r) || (ad <= tolc);
@@ -472,42 +507,71 @@ __global__ void __launch_bounds__(256) screen_generic_kernel(const void* __restr
       }
     }
   }
-  n_mis = warp_add_u32(n_mis);   // a warp sees < 2^32 elements of one launch slice
-  n_nan = warp_add_u32(n_nan);
-  n_inf = warp_add_u32(n_inf);
-  best = warp_max_u64(best);
-  qb = warp_max_u32(qb);
-  if ((threadIdx.x & 31) == 0) {
-    Acc* a = &acc[k];
-    if (n_mis) atomicAdd(&a->mism, (unsigned long long)n_mis);
-    if (n_nan) atomicAdd(&a->nan, (unsigned long long)n_nan);
-    if (n_inf) atomicAdd(&a->inf, (unsigned long long)n_inf);
-    if (best) atomicMax(&a->key, best);
-    if (qb) atomicMax(&a->rel, qb);
+  // warp-level merge, then one set of atomics per warp (a warp sees < 2^32 elements)
+  __device__ __forceinline__ void commit(Acc* a) {
+    n_mis = warp_add_u32(n_mis);
+    n_nan = warp_add_u32(n_nan);
+    n_inf = warp_add_u32(n_inf);
+    best = warp_max_u64(best);
+    qb = warp_max_u32(qb);
+    if ((threadIdx.x & 31) == 0) {
+      if (n_mis) atomicAdd(&a->mism, (unsigned long long)n_mis);
+      if (n_nan) atomicAdd(&a->nan, (unsigned long long)n_nan);
+      if (n_inf) atomicAdd(&a->inf, (unsigned long long)n_inf);
+      if (best) atomicMax(&a->key, best);
+      if (qb) atomicMax(&a->rel, qb);
+    }
   }
+};
+
+// Elements [e0, e1) of every candidate under an arbitrary mask.  grid = (blocks, K).
+// Used for the ragged tail and for masks finer than a kernel tile.
+template <int DT>
+__global__ void __launch_bounds__(256) screen_generic_kernel(const void* __restrict__ ref,
+                                                             const void* const* __restrict__ cands,
+                                                             Acc* __restrict__ acc,
+                                                             unsigned long long e0,
+                                                             unsigned long long e1, float atol,
+                                                             float rtol, MaskDev mask) {
+  using E = Elem<DT>;
+  const unsigned int k = blockIdx.y;
+  const void* cand = cands[k];
+  ExactAcc x;
+  const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
+  for (unsigned long long i = e0 + (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < e1;
+       i += stride) {
+    if (!mask_selected(mask, i)) continue;
+    x.add(E::load(ref, i), E::load(cand, i), i, atol, rtol);
+  }
+  x.commit(&acc[k]);
+}
+
+// Scout: the first `nscout` full tiles (of the list, or tiles 0..nscout-1) of every
+// candidate, classified exactly before the streaming kernel starts.  Their maxima
+// seed the streaming kernel's thresholds, so that its first tile does not have to
+// discover them.  grid = (nscout * kTile / 256, K).
+template <int DT>
+__global__ void __launch_bounds__(256) screen_scout_kernel(const void* __restrict__ ref,
+                                                           const void* const* __restrict__ cands,
+                                                           Acc* __restrict__ acc,
+                                                           const uint32_t* __restrict__ tile_list,
+                                                           float atol, float rtol) {
+  using E = Elem<DT>;
+  constexpr unsigned int kBlocksPerTile = kTile / 256;
+  const unsigned int k = blockIdx.y;
+  const unsigned int slot = blockIdx.x / kBlocksPerTile;
+  const unsigned long long tile = tile_list ? tile_list[slot] : slot;
+  const unsigned long long i = tile * kTile + (blockIdx.x % kBlocksPerTile) * 256 + threadIdx.x;
+  ExactAcc x;
+  x.add(E::load(ref, i), E::load(cands[k], i), i, atol, rtol);
+  x.commit(&acc[k]);
 }
 
 __global__ void screen_finalize_kernel(const Acc* __restrict__ acc, kb_screen_result* __restrict__ out,
                                        unsigned int K) {
   const unsigned int k = blockIdx.x * blockDim.x + threadIdx.x;
   if (k >= K) return;
-  const Acc a = acc[k];
-  kb_screen_result r;
-  r.mismatch_count = a.mism;
-  r.nan_count = a.nan;
-  r.inf_count = a.inf;
-  if (a.key == 0ull) {
-    r.argmax_idx = -1;
-    r.max_abs_err = 0.0f;
-  } else {
-    const unsigned long long kv = a.key - 1ull;
-    r.max_abs_err = __uint_as_float((unsigned int)(kv >> 32));
-    r.argmax_idx = (int64_t)(0xFFFFFFFFu - (unsigned int)kv);
-  }
-  r.max_rel_err = __uint_as_float(a.rel);
-  r.pass = a.mism == 0ull ? 1u : 0u;
-  r.reserved = 0u;
-  out[k] = r;
+  unpack_record(acc[k], &out[k]);
 }
 
 // K pointers travel to the device table through kernel arguments (no staging
@@ -516,10 +580,18 @@ constexpr int kPtrsPerLaunch = 480;
 struct PtrChunk {
   const void* p[kPtrsPerLaunch];
 };
-__global__ void upload_ptrs_kernel(const PtrChunk chunk, const void** table, unsigned int offset,
-                                   unsigned int count) {
+// Also zeroes the accumulators of the same candidates and the ticket counter.
+__global__ void screen_prep_kernel(const PtrChunk chunk, const void** table, Acc* acc,
+                                   unsigned int* done, unsigned int offset, unsigned int count) {
   const unsigned int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < count) table[offset + i] = chunk.p[i];
+  if (i < count) {
+    table[offset + i] = chunk.p[i];
+    Acc z;
+    z.mism = z.nan = z.inf = z.key = 0ull;
+    z.rel = z.pad = 0u;
+    acc[offset + i] = z;
+  }
+  if (i == 0) *done = 0u;
 }
 
 }  // namespace kb
