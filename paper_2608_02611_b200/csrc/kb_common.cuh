@@ -44,6 +44,12 @@ template <> struct Elem<KB_F32> {
   __device__ __forceinline__ static float load(const void* p, unsigned long long i) {
     return reinterpret_cast<const float*>(p)[i];
   }
+  // d0 = c[e] - r0, d1 = c[e+1] - r1 for the even element e of a thread's raw words
+  __device__ __forceinline__ static void pair_diff(const unsigned int* words, int e, float r0, float r1,
+                                                   float& d0, float& d1) {
+    d0 = __fsub_rn(__uint_as_float(words[e]), r0);
+    d1 = __fsub_rn(__uint_as_float(words[e + 1]), r1);
+  }
 };
 template <> struct Elem<KB_BF16> {
   static constexpr int kBytes = 2;
@@ -61,6 +67,15 @@ template <> struct Elem<KB_BF16> {
   __device__ __forceinline__ static float load(const void* p, unsigned long long i) {
     return __uint_as_float((unsigned int)reinterpret_cast<const unsigned short*>(p)[i] << 16);
   }
+  // Mixed-precision subtract: the bf16 operand is widened exactly and the
+  // difference rounded once, i.e. the same value as decode + fp32 subtract,
+  // without a separate decode instruction.
+  __device__ __forceinline__ static void pair_diff(const unsigned int* words, int e, float r0, float r1,
+                                                   float& d0, float& d1) {
+    asm("{\n.reg .b16 lo, hi;\nmov.b32 {lo, hi}, %2;\nsub.rn.f32.bf16 %0, lo, %3;\nsub.rn.f32.bf16 %1, hi, %4;\n}"
+        : "=f"(d0), "=f"(d1)
+        : "r"(words[e >> 1]), "f"(r0), "f"(r1));
+  }
 };
 template <> struct Elem<KB_F16> {
   static constexpr int kBytes = 2;
@@ -76,6 +91,12 @@ template <> struct Elem<KB_F16> {
   }
   __device__ __forceinline__ static float load(const void* p, unsigned long long i) {
     return __half2float(reinterpret_cast<const __half*>(p)[i]);
+  }
+  __device__ __forceinline__ static void pair_diff(const unsigned int* words, int e, float r0, float r1,
+                                                   float& d0, float& d1) {
+    asm("{\n.reg .b16 lo, hi;\nmov.b32 {lo, hi}, %2;\nsub.rn.f32.f16 %0, lo, %3;\nsub.rn.f32.f16 %1, hi, %4;\n}"
+        : "=f"(d0), "=f"(d1)
+        : "r"(words[e >> 1]), "f"(r0), "f"(r1));
   }
 };
 

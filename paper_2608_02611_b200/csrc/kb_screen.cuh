@@ -105,8 +105,8 @@ struct StreamSmem {
   unsigned long long* key;   // [kMaxKC]
   const void** ptrs;         // [kMaxKC] candidate pointers of the current chunk (producer only)
   unsigned int* rel;         // [kMaxKC] bits of the running max relative error (CTA-wide)
-  float* thr;                // [kMaxKC][kWarps] running max |c-r| seen by each warp (-1: none)
-  float* gth;                // [kMaxKC] a value strictly below an error some CTA has recorded (-1: none)
+  float2* thr2;              // [kMaxKC][kWarps] per warp: x = errors <= x cannot become the maximum
+                             // (-1: none), y = the running max relative error (copy of rel)
   volatile unsigned int* abort_flag;
 };
 
@@ -114,7 +114,7 @@ __host__ __device__ inline size_t stream_smem_bytes(uint32_t stages, uint32_t ti
   size_t b = (size_t)stages * tile_bytes;
   b += 2 * (size_t)stages * 8;
   b += 3 * (size_t)kMaxKC * 8 + (size_t)kMaxKC * 8 + (size_t)kMaxKC * 8 + (size_t)kMaxKC * 4;
-  b += (size_t)kMaxKC * kWarps * 4 + (size_t)kMaxKC * 4;
+  b += (size_t)kMaxKC * kWarps * 8;
   b += 16;
   return b + 128;  // alignment slack
 }
@@ -157,10 +157,8 @@ __global__ void __maxnreg__(96) screen_stream_kernel(const StreamParams p) {
     q += (size_t)kMaxKC * 8;
     s.ptrs = reinterpret_cast<const void**>(q);
     q += (size_t)kMaxKC * 8;
-    s.thr = reinterpret_cast<float*>(q);
-    q += (size_t)kMaxKC * kWarps * 4;
-    s.gth = reinterpret_cast<float*>(q);
-    q += (size_t)kMaxKC * 4;
+    s.thr2 = reinterpret_cast<float2*>(q);
+    q += (size_t)kMaxKC * kWarps * 8;
     s.rel = reinterpret_cast<unsigned int*>(q);
     q += (size_t)kMaxKC * 4;
     s.abort_flag = reinterpret_cast<volatile unsigned int*>(q);
@@ -185,9 +183,8 @@ __global__ void __maxnreg__(96) screen_stream_kernel(const StreamParams p) {
     s.cnt[2 * kMaxKC + i] = 0ull;
     s.key[i] = 0ull;
     s.rel[i] = 0u;
-    s.gth[i] = -1.0f;
   }
-  for (int i = tid; i < kMaxKC * kWarps; i += kStreamThreads) s.thr[i] = -1.0f;
+  for (int i = tid; i < kMaxKC * kWarps; i += kStreamThreads) s.thr2[i] = make_float2(-1.0f, 0.0f);
   __syncthreads();
 
   // Work items (chunk, tile), chunk-major; each CTA takes one contiguous run of them, so
@@ -276,8 +273,7 @@ __global__ void __maxnreg__(96) screen_stream_kernel(const StreamParams p) {
         s.key[i] = 0ull;
         s.rel[i] = 0u;
       }
-      for (int i = tid; i < kMaxKC; i += kConsumers) s.gth[i] = -1.0f;
-      for (int i = tid; i < kMaxKC * kWarps; i += kConsumers) s.thr[i] = -1.0f;
+      for (int i = tid; i < kMaxKC * kWarps; i += kConsumers) s.thr2[i] = make_float2(-1.0f, 0.0f);
       consumers_sync();
     };
 
@@ -335,26 +331,33 @@ __global__ void __maxnreg__(96) screen_stream_kernel(const StreamParams p) {
         }
       }
       if (xkk < cur_kc) {
-        if (xold_r > xmine_r) atomicMax(&s.rel[xkk], xold_r);
+        int* row = reinterpret_cast<int*>(&s.thr2[xkk * kWarps]);
+        if (xold_r > xmine_r) {
+          atomicMax(&s.rel[xkk], xold_r);
+#pragma unroll
+          for (int w2 = 0; w2 < kWarps; ++w2) atomicMax(row + 2 * w2 + 1, (int)xold_r);
+        }
         const unsigned long long gk = xold_k > xmine_k ? xold_k : xmine_k;
         if (gk != 0ull) {
           // An error equal to one recorded at a lower index, or strictly below one
           // recorded anywhere, can never become the maximum.
           const unsigned int db = (unsigned int)((gk - 1ull) >> 32);
           const unsigned long long gidx = 0xFFFFFFFFull - ((gk - 1ull) & 0xFFFFFFFFull);
-          if (gidx < tile_base)
-            atomicMax(reinterpret_cast<int*>(&s.gth[xkk]), (int)db);
-          else if (db)
-            atomicMax(reinterpret_cast<int*>(&s.gth[xkk]), (int)(db - 1u));
+          const int lim = gidx < tile_base ? (int)db : (int)db - 1;   // db == 0: -1 is below every float >= -1
+          if (lim >= 0) {
+#pragma unroll
+            for (int w2 = 0; w2 < kWarps; ++w2) atomicMax(row + 2 * w2, lim);
+          }
         }
       }
       __syncwarp();
 
       // ---- the candidates of this chunk against the tile in registers ----
       for (int kk = 0; kk < cur_kc; ++kk) {
-        const float rel = __uint_as_float(*reinterpret_cast<volatile unsigned int*>(&s.rel[kk]));
-        const float th_own = s.thr[kk * kWarps + warp];
-        const float th = fmaxf(th_own, *reinterpret_cast<volatile float*>(&s.gth[kk]));
+        const unsigned long long trw =
+            *reinterpret_cast<volatile unsigned long long*>(&s.thr2[kk * kWarps + warp]);
+        const float th = __uint_as_float((unsigned int)trw);
+        const float rel = __uint_as_float((unsigned int)(trw >> 32));
         if (!mbar_wait_bounded(&s.full[stage], phase, s.abort_flag, p.status)) {
           ok = false;
           break;
@@ -369,32 +372,33 @@ __global__ void __maxnreg__(96) screen_stream_kernel(const StreamParams p) {
           stage = 0;
           phase ^= 1u;
         }
-
-        float c[kEPT];
-#pragma unroll
-        for (int j = 0; j < NV; ++j) E::decode(w[j], &c[j * VEC]);
+        const unsigned int* words = reinterpret_cast<const unsigned int*>(w);
 
         bool bad = false;
         float mabs = 0.0f, mrel = 0.0f;
-        if (rel <= p.rtol_lean) {
+        const bool lean = rel <= p.rtol_lean;
+        if (lean) {
           // lean filter: (b) and (c); (a) is implied
 #pragma unroll
           for (int e = 0; e < kEPT; e += 2) {
-            const float ad0 = fabsf(__fsub_rn(c[e], r[e]));
-            const float ad1 = fabsf(__fsub_rn(c[e + 1], r[e + 1]));
-            const float t0 = fmaf(-rel, fabsf(r[e]), ad0);
-            const float t1 = fmaf(-rel, fabsf(r[e + 1]), ad1);
-            mabs = max3(mabs, ad0, ad1);
+            float d0, d1;
+            E::pair_diff(words, e, r[e], r[e + 1], d0, d1);
+            const float t0 = fmaf(-rel, fabsf(r[e]), fabsf(d0));
+            const float t1 = fmaf(-rel, fabsf(r[e + 1]), fabsf(d1));
+            mabs = max3(mabs, fabsf(d0), fabsf(d1));
             mrel = max3_nan(mrel, t0, t1);
           }
         } else {
 #pragma unroll
-          for (int e = 0; e < kEPT; ++e) {
-            const float ad = fabsf(__fsub_rn(c[e], r[e]));
-            const float tol = __fadd_rn(p.atol, __fmul_rn(p.rtol, fabsf(r[e])));
-            bad |= !(ad <= tol);      // an infinite ad with an infinite tol is caught by (b)
-            mabs = fmaxf(mabs, ad);
-            mrel = max2_nan(mrel, fmaf(-rel, fabsf(r[e]), ad));
+          for (int e = 0; e < kEPT; e += 2) {
+            float d0, d1;
+            E::pair_diff(words, e, r[e], r[e + 1], d0, d1);
+            const float a0 = fabsf(d0), a1 = fabsf(d1);
+            const float tol0 = __fadd_rn(p.atol, __fmul_rn(p.rtol, fabsf(r[e])));
+            const float tol1 = __fadd_rn(p.atol, __fmul_rn(p.rtol, fabsf(r[e + 1])));
+            bad |= !(a0 <= tol0) || !(a1 <= tol1);   // an infinite error under an infinite tol is caught by (b)
+            mabs = max3(mabs, a0, a1);
+            mrel = max3_nan(mrel, fmaf(-rel, fabsf(r[e]), a0), fmaf(-rel, fabsf(r[e + 1]), a1));
           }
         }
         const bool trig = bad || (mabs > th) || !(mrel <= 0.0f) || extreme;
@@ -403,10 +407,12 @@ __global__ void __maxnreg__(96) screen_stream_kernel(const StreamParams p) {
         // ---- exact path.  A triggered thread finds its largest finite error (first
         // index on ties) with a running compare, and evaluates by the definition the
         // elements that fail the tolerance / relative-error filter or are not finite. ----
-        const bool lean = rel <= p.rtol_lean;
         unsigned int n_mis = 0, n_nan = 0, n_inf = 0, qb = 0u;
         unsigned long long best = 0ull;
         if (trig) {
+          float c[kEPT];
+#pragma unroll
+          for (int j = 0; j < NV; ++j) E::decode(w[j], &c[j * VEC]);
           float m = -1.0f;
           int mi = 0;
 #pragma unroll
@@ -448,15 +454,23 @@ __global__ void __maxnreg__(96) screen_stream_kernel(const StreamParams p) {
           if (n_mis) atomicAdd(&s.cnt[kk], (unsigned long long)n_mis);
           if (n_nan) atomicAdd(&s.cnt[kMaxKC + kk], (unsigned long long)n_nan);
           if (n_inf) atomicAdd(&s.cnt[2 * kMaxKC + kk], (unsigned long long)n_inf);
+          int* row = reinterpret_cast<int*>(&s.thr2[kk * kWarps]);
           if (best != 0ull) {
             atomicMax(&s.key[kk], best);
-            // everything this warp meets in later tiles with an error <= this one loses ...
-            const unsigned int db = (unsigned int)((best - 1ull) >> 32);
-            s.thr[kk * kWarps + warp] = fmaxf(th_own, __uint_as_float(db));
-            // ... and anything strictly below it loses for every warp
-            if (db) atomicMax(reinterpret_cast<int*>(&s.gth[kk]), (int)(db - 1u));
+            // what this warp meets in later tiles with an error <= this one loses the index
+            // tie; for the other warps (same tile, other indices) only strictly smaller errors do
+            const int db = (int)(unsigned int)((best - 1ull) >> 32);
+#pragma unroll
+            for (int w2 = 0; w2 < kWarps; ++w2) {
+              const int lim = (w2 == warp) ? db : db - 1;
+              if (lim >= 0) atomicMax(row + 2 * w2, lim);
+            }
           }
-          if (qb > __float_as_uint(rel)) atomicMax(&s.rel[kk], qb);
+          if (qb > __float_as_uint(rel)) {
+            atomicMax(&s.rel[kk], qb);
+#pragma unroll
+            for (int w2 = 0; w2 < kWarps; ++w2) atomicMax(row + 2 * w2 + 1, (int)qb);
+          }
         }
         __syncwarp();
       }
