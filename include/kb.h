@@ -172,6 +172,40 @@ kb_status kb_screen_host(kb_ctx* ctx, const void* h_ref, const void* const* h_ca
                          uint32_t K, uint64_t N, kb_dtype dtype, float atol, float rtol,
                          const kb_mask* mask, kb_screen_result* h_out, void* stream);
 
+/* ---- the same gate for callers that must not allocate ----------------------
+ * (The paper has no counterpart; this entry point exists for integration.)
+ *
+ * Some hosts of this library cannot let it call cudaMalloc: a serving loop that
+ * has promised its users no allocation after start-up; a framework whose own
+ * allocator has already claimed nearly all device memory, so that a driver
+ * allocation from a third party may simply fail; a process whose allocations
+ * are all audited and pre-approved.  kb_screen_static does what kb_screen does
+ * with mask == NULL, but creates no context and allocates nothing, neither on
+ * the device nor through any library: the per-candidate accumulators and the
+ * candidate pointer table live in a fixed array inside the library's device
+ * image (KB_STATIC_SCRATCH_BYTES, held by every GPU that loads the library
+ * until the process exits).
+ *
+ *   - The call works on the CURRENT device; `stream` must belong to it.
+ *   - 1 <= K <= KB_STATIC_MAX_K; larger K is refused with KB_ERR_WORKSPACE and
+ *     a message readable through kb_last_error(NULL).  Other argument rules are
+ *     those of kb_screen; there is no fidelity mask.
+ *   - The first call on a device looks up the address of the array and sets
+ *     kernel attributes.  Make that first call before any stream capture
+ *     begins.
+ *   - All calls on one device share the one array, which keeps what the last
+ *     call left in it; each call clears the part it uses before use.  Two
+ *     calls that overlap on the GPU (different streams, or one stream and a
+ *     graph replay) race on it and give wrong records: order them.
+ *   - Asynchronous like kb_screen; d_out is valid after `stream` synchronises.
+ *     A device-side wait that ran out cannot be polled through this entry point
+ *     (there is no context); use kb_screen + kb_ctx_poll where that matters. */
+#define KB_STATIC_MAX_K 1024u
+#define KB_STATIC_SCRATCH_BYTES (256u + 1024u * 40u + 1024u * 8u)
+kb_status kb_screen_static(const void* d_ref, const void* const* h_cands, uint32_t K, uint64_t N,
+                           kb_dtype dtype, float atol, float rtol, kb_screen_result* d_out,
+                           void* stream);
+
 /* ---- stability adjudication (Algorithm 1 "adjudicated latency"; Sec. 1
  *      contribution 1; Appendix "Relative Variability Metrics") ------------ */
 

@@ -37,7 +37,7 @@ EXPORTS = [
     "kb_ctx_create", "kb_ctx_destroy", "kb_last_error", "kb_ctx_poll", "kb_ctx_set_grid",
     "kb_ctx_enable_timing", "kb_ctx_read_timer", "kb_ctx_launch_count",
     "kb_mask_create_strided", "kb_mask_create_bitmap", "kb_mask_count", "kb_mask_destroy",
-    "kb_screen", "kb_screen_host", "kb_adjudicate", "kb_select",
+    "kb_screen", "kb_screen_host", "kb_screen_static", "kb_adjudicate", "kb_select",
 ]
 
 
@@ -78,6 +78,7 @@ def load() -> ctypes.CDLL:
     L.kb_mask_destroy.argtypes = [vp]
     L.kb_screen.argtypes = [vp, vp, vp, u32, u64, i32, f32, f32, vp, vp, vp]
     L.kb_screen_host.argtypes = [vp, vp, vp, u32, u64, i32, f32, f32, vp, vp, vp]
+    L.kb_screen_static.argtypes = [vp, vp, u32, u64, i32, f32, f32, vp, vp]
     L.kb_adjudicate.argtypes = [vp, vp, u32, u32, vp, vp, vp, vp]
     L.kb_select.argtypes = [vp, vp, vp, u32, i32, u32, vp, vp, vp]
     for name in EXPORTS:
@@ -252,6 +253,32 @@ class Context:
                               int(budget), surv.data_ptr(), n.data_ptr(), _stream_ptr(median.device))
         self._check(rc, "kb_select")
         return surv, n
+
+
+KB_STATIC_MAX_K = 1024
+
+
+def screen_static(ref: torch.Tensor, cands: Sequence[torch.Tensor], atol: float, rtol: float,
+                  out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """kb_screen_static: the gate for hosts that forbid allocation by third parties.
+
+    Needs no Context and makes the library allocate nothing; its scratch is a fixed array
+    inside the library (at most KB_STATIC_MAX_K candidates, no mask).  Pass ``out`` (a uint8
+    CUDA tensor [K, 48]) to keep torch from allocating as well.  Calls share the array: do
+    not let two of them overlap on the GPU.  Works on the current device and stream.
+    """
+    K = len(cands)
+    N = ref.numel()
+    code = DTYPE_CODE.get(ref.dtype, -1)
+    if out is None:
+        out = torch.empty((K, RESULT_BYTES), dtype=torch.uint8, device=ref.device)
+    ptrs = (ctypes.c_void_p * max(K, 1))(*[c.data_ptr() for c in cands])
+    with torch.cuda.device(ref.device):
+        rc = load().kb_screen_static(ref.data_ptr(), ptrs, K, N, code, float(atol), float(rtol),
+                                     out.data_ptr(), _stream_ptr(ref.device))
+    if rc != KB_OK:
+        raise KbError(rc, "kb_screen_static", (load().kb_last_error(None) or b"").decode())
+    return out
 
 
 def records(screen_out: torch.Tensor) -> np.ndarray:

@@ -5,6 +5,7 @@
 #include <cstdio>
 #include <cstring>
 #include <cmath>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -584,6 +585,78 @@ extern "C" kb_status kb_screen(kb_ctx* ctx, const void* d_ref, const void* const
   DeviceGuard g(ctx->device);
   return screen_dispatch(ctx, d_ref, h_cands, K, N, dtype, atol, rtol, mask, d_out,
                          reinterpret_cast<cudaStream_t>(stream));
+}
+
+// ---------------------------------------------------------------------------
+// kb_screen_static: the gate without any allocation
+// ---------------------------------------------------------------------------
+
+// Scratch of the allocation-free entry point: [status words 256 B | accumulators | pointer
+// table].  In host code this name is only a handle for cudaGetSymbolAddress; it is not a
+// device address and must never be passed to a kernel as it stands.
+static __device__ __align__(256) unsigned char g_static_scratch[KB_STATIC_SCRATCH_BYTES];
+
+namespace {
+
+constexpr int kStaticMaxDevices = 64;
+struct StaticSlot {
+  bool ready = false;
+  kb_ctx ctx;   // a host-side view over the static array; owns nothing, is never destroyed
+};
+StaticSlot g_static_slot[kStaticMaxDevices];
+std::mutex g_static_mutex;
+
+// Once per device, with that device current: resolve the array's device address, read the
+// SM count, raise the kernels' shared-memory limits.  None of these allocates.
+kb_status static_setup(int device, kb_ctx** out) {
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  StaticSlot& slot = g_static_slot[device];
+  if (!slot.ready) {
+    kb_ctx* ctx = &slot.ctx;
+    ctx->device = device;
+    unsigned char* base = nullptr;
+    KB_CUDA(ctx, cudaGetSymbolAddress(reinterpret_cast<void**>(&base), g_static_scratch));
+    int sms = 0;
+    KB_CUDA(ctx, cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
+    ctx->sm_count = sms;
+    ctx->d_status = reinterpret_cast<unsigned int*>(base);
+    ctx->ws = base + 256;
+    ctx->ws_bytes = KB_STATIC_SCRATCH_BYTES - 256;   // ensure_ws never grows it: K is capped
+    kb_status st;
+    if ((st = set_stream_attr<KB_F32>(ctx)) != KB_OK) return st;
+    if ((st = set_stream_attr<KB_F16>(ctx)) != KB_OK) return st;
+    if ((st = set_stream_attr<KB_BF16>(ctx)) != KB_OK) return st;
+    slot.ready = true;
+  }
+  *out = &slot.ctx;
+  return KB_OK;
+}
+
+}  // namespace
+
+extern "C" kb_status kb_screen_static(const void* d_ref, const void* const* h_cands, uint32_t K,
+                                      uint64_t N, kb_dtype dtype, float atol, float rtol,
+                                      kb_screen_result* d_out, void* stream) {
+  int device = -1;
+  if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= kStaticMaxDevices) {
+    cudaGetLastError();
+    snprintf(g_create_err, sizeof g_create_err, "kb_screen_static: no usable current CUDA device");
+    return KB_ERR_CUDA;
+  }
+  if (K > KB_STATIC_MAX_K) {
+    snprintf(g_create_err, sizeof g_create_err,
+             "kb_screen_static: K=%u exceeds the %u candidates the static scratch holds "
+             "(use kb_screen, which may allocate)", K, KB_STATIC_MAX_K);
+    return KB_ERR_WORKSPACE;
+  }
+  kb_ctx* ctx = nullptr;
+  kb_status rc = static_setup(device, &ctx);
+  if (rc == KB_OK) rc = validate_screen(ctx, d_ref, h_cands, K, N, dtype, atol, rtol, nullptr, d_out, true);
+  if (rc == KB_OK)
+    rc = screen_dispatch(ctx, d_ref, h_cands, K, N, dtype, atol, rtol, nullptr, d_out,
+                         reinterpret_cast<cudaStream_t>(stream));
+  if (rc != KB_OK) snprintf(g_create_err, sizeof g_create_err, "%.250s", g_static_slot[device].ctx.err);
+  return rc;
 }
 
 extern "C" kb_status kb_screen_host(kb_ctx* ctx, const void* h_ref, const void* const* h_cands_host,
