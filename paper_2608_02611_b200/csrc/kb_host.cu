@@ -141,10 +141,10 @@ kb_status ensure_buf(kb_ctx* ctx, T** buf, size_t* have, size_t need) {
 template <int DT>
 kb_status launch_stream(kb_ctx* ctx, StreamParams& sp, cudaStream_t st) {
   const uint32_t tile_bytes = kTile * Elem<DT>::kBytes;
-  sp.stages = (tile_bytes == 8192) ? 10 : 6;
+  sp.stages = (tile_bytes == 8192) ? 7 : 3;
   const size_t smem = stream_smem_bytes(sp.stages, tile_bytes);
   const unsigned long long nitems = (unsigned long long)sp.nchunks * sp.ntiles;
-  unsigned long long grid = ctx->forced_grid ? ctx->forced_grid : 2ull * ctx->sm_count;
+  unsigned long long grid = ctx->forced_grid ? ctx->forced_grid : 3ull * ctx->sm_count;
   if (grid > nitems) grid = nitems;
   {
     ScopedTimer tm(ctx, KB_TIMER_SCREEN_STREAM, st);
@@ -174,7 +174,7 @@ kb_status launch_generic(kb_ctx* ctx, const void* ref, const void* const* tab, A
 template <int DT>
 kb_status set_stream_attr(kb_ctx* ctx) {
   const uint32_t tile_bytes = kTile * Elem<DT>::kBytes;
-  const size_t smem = stream_smem_bytes(tile_bytes == 8192 ? 10 : 6, tile_bytes);
+  const size_t smem = stream_smem_bytes(tile_bytes == 8192 ? 7 : 3, tile_bytes);
   KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT>,
                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT>,
@@ -544,7 +544,7 @@ kb_status screen_impl(kb_ctx* ctx, const void* d_ref, const void* const* h_cands
       // chunk the candidates: shared-memory accumulators hold kMaxKC of them, and
       // small tensors need more, smaller items to fill the machine
       uint32_t nchunks = (K + kMaxKC - 1) / kMaxKC;
-      const uint64_t grid = ctx->forced_grid ? ctx->forced_grid : 2ull * ctx->sm_count;
+      const uint64_t grid = ctx->forced_grid ? ctx->forced_grid : 3ull * ctx->sm_count;
       const uint64_t want_items = 8 * grid;
       if ((uint64_t)nchunks * sp.ntiles < want_items) {
         uint64_t nc = (want_items + sp.ntiles - 1) / sp.ntiles;

@@ -132,7 +132,7 @@ __host__ __device__ inline size_t stream_smem_bytes(uint32_t stages, uint32_t ti
 // Inf - Inf) to the decision.  While rel <= rtol*(1-2^-20), (c) implies (a) and
 // the "lean" form drops the tolerance test: ad <= rel*|r| <= RN(rtol*|r|) <= tol.
 template <int DT>
-__global__ void __maxnreg__(96) screen_stream_kernel(const StreamParams p) {
+__global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
   using E = Elem<DT>;
   constexpr int VEC = E::kVec;
   constexpr int NV = kEPT / VEC;
@@ -277,11 +277,55 @@ __global__ void __maxnreg__(96) screen_stream_kernel(const StreamParams p) {
       consumers_sync();
     };
 
+    // Exchange of running maxima with the other CTAs.  Every merge is a maximum, so the
+    // exchange needs no ordering: lane (warp, lane) owns candidate warp + 8*lane of the
+    // chunk, pushes this CTA's maxima with atomicMax and gets everyone's back.  The values
+    // that come back are applied one tile later (the round trip to L2 is then hidden),
+    // except on a chunk's first tile, where the scout's seeds are wanted at once.
+    const int xkk = warp + kWarps * lane;
+    unsigned long long xmine_k = 0ull, xold_k = 0ull;
+    unsigned int xmine_r = 0u, xold_r = 0u;
+    bool xpending = false;
+    auto exchange_issue = [&]() {
+      if (xkk < cur_kc) {
+        xmine_k = *reinterpret_cast<volatile unsigned long long*>(&s.key[xkk]);
+        xmine_r = *reinterpret_cast<volatile unsigned int*>(&s.rel[xkk]);
+        Acc* a = &p.acc[cur_k0 + xkk];
+        xold_k = atomicMax(&a->key, xmine_k);
+        xold_r = atomicMax(&a->rel, xmine_r);
+      }
+    };
+    auto exchange_apply = [&](unsigned long long tile_base) {
+      if (xkk < cur_kc) {
+        int* row = reinterpret_cast<int*>(&s.thr2[xkk * kWarps]);
+        if (xold_r > xmine_r) {
+          atomicMax(&s.rel[xkk], xold_r);
+#pragma unroll
+          for (int w2 = 0; w2 < kWarps; ++w2) atomicMax(row + 2 * w2 + 1, (int)xold_r);
+        }
+        const unsigned long long gk = xold_k > xmine_k ? xold_k : xmine_k;
+        if (gk != 0ull) {
+          // An error equal to one recorded at a lower index, or strictly below one
+          // recorded anywhere, can never become the maximum.
+          const unsigned int db = (unsigned int)((gk - 1ull) >> 32);
+          const unsigned long long gidx = 0xFFFFFFFFull - ((gk - 1ull) & 0xFFFFFFFFull);
+          const int lim = gidx < tile_base ? (int)db : (int)db - 1;   // db == 0: -1 is below every float >= -1
+          if (lim >= 0) {
+#pragma unroll
+            for (int w2 = 0; w2 < kWarps; ++w2) atomicMax(row + 2 * w2, lim);
+          }
+        }
+      }
+      __syncwarp();
+    };
+
     for (unsigned long long item = item_lo; item < item_hi; ++item) {
       const uint32_t chunk = (uint32_t)(item / p.ntiles);
       const uint32_t slot = p.slot0 + (uint32_t)(item % p.ntiles);
       const uint32_t tile = p.tile_list ? p.tile_list[slot] : slot;
+      const bool first_of_chunk = (int)chunk != cur_chunk;
       if ((int)chunk != cur_chunk) {
+        xpending = false;
         if (cur_chunk >= 0) flush();
         cur_chunk = (int)chunk;
         cur_k0 = chunk * p.KC;
@@ -290,18 +334,9 @@ __global__ void __maxnreg__(96) screen_stream_kernel(const StreamParams p) {
       if (!ok) continue;
       const unsigned long long tile_base = (unsigned long long)tile * kTile;
 
-      // ---- exchange running maxima with the other CTAs (all merges are maxima, so this
-      // needs no ordering): push this CTA's, pull everyone's; applied after the tile load ----
-      const int xkk = warp + kWarps * lane;          // each candidate of the chunk has one owner lane
-      unsigned long long xmine_k = 0ull, xold_k = 0ull;
-      unsigned int xmine_r = 0u, xold_r = 0u;
-      if (xkk < cur_kc) {
-        xmine_k = *reinterpret_cast<volatile unsigned long long*>(&s.key[xkk]);
-        xmine_r = *reinterpret_cast<volatile unsigned int*>(&s.rel[xkk]);
-        Acc* a = &p.acc[cur_k0 + xkk];
-        xold_k = atomicMax(&a->key, xmine_k);
-        xold_r = atomicMax(&a->rel, xmine_r);
-      }
+      if (xpending) exchange_apply(tile_base);
+      exchange_issue();
+      xpending = !first_of_chunk;
 
       // ---- reference tile: 16 elements per thread stay in registers ----
       float r[kEPT];
@@ -330,27 +365,7 @@ __global__ void __maxnreg__(96) screen_stream_kernel(const StreamParams p) {
           extreme |= (ar > 0.0f && ar < 7.888609052e-31f);
         }
       }
-      if (xkk < cur_kc) {
-        int* row = reinterpret_cast<int*>(&s.thr2[xkk * kWarps]);
-        if (xold_r > xmine_r) {
-          atomicMax(&s.rel[xkk], xold_r);
-#pragma unroll
-          for (int w2 = 0; w2 < kWarps; ++w2) atomicMax(row + 2 * w2 + 1, (int)xold_r);
-        }
-        const unsigned long long gk = xold_k > xmine_k ? xold_k : xmine_k;
-        if (gk != 0ull) {
-          // An error equal to one recorded at a lower index, or strictly below one
-          // recorded anywhere, can never become the maximum.
-          const unsigned int db = (unsigned int)((gk - 1ull) >> 32);
-          const unsigned long long gidx = 0xFFFFFFFFull - ((gk - 1ull) & 0xFFFFFFFFull);
-          const int lim = gidx < tile_base ? (int)db : (int)db - 1;   // db == 0: -1 is below every float >= -1
-          if (lim >= 0) {
-#pragma unroll
-            for (int w2 = 0; w2 < kWarps; ++w2) atomicMax(row + 2 * w2, lim);
-          }
-        }
-      }
-      __syncwarp();
+      if (first_of_chunk) exchange_apply(tile_base);
 
       // ---- the candidates of this chunk against the tile in registers ----
       for (int kk = 0; kk < cur_kc; ++kk) {
