@@ -555,6 +555,7 @@ kb_status screen_impl(kb_ctx* ctx, const void* d_ref, const void* const* h_cands
       sp.KC = (K + nchunks - 1) / nchunks;
       sp.nchunks = (K + sp.KC - 1) / sp.KC;
       sp.done = ctx->d_status + 1;
+      sp.sched = reinterpret_cast<unsigned long long*>(ctx->d_status + 2);
       sp.out = d_out;
       return launch_stream<DT>(ctx, sp, st);
     }

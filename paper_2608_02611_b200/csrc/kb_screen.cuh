@@ -39,6 +39,7 @@ struct StreamParams {
   float rtol_lean;              // rtol*(1-2^-20) rounded down, or -1: see the lean filter below
   unsigned int* status;
   unsigned int* done;           // zeroed ticket counter: the last CTA to finish unpacks the records
+  unsigned long long* sched;    // zeroed work counter: CTAs draw items from it
   kb_screen_result* out;        // [K]
 };
 
@@ -55,9 +56,6 @@ __device__ __forceinline__ bool mask_selected(const MaskDev& m, unsigned long lo
   return (m.bits[t >> 6] >> (t & 63ull)) & 1ull;
 }
 
-__device__ __forceinline__ void consumers_sync() {
-  asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory");
-}
 
 // accumulator -> public record
 __device__ __forceinline__ void unpack_record(const Acc& a, kb_screen_result* dst) {
@@ -101,6 +99,8 @@ struct StreamSmem {
   unsigned char* buf;
   uint64_t* full;
   uint64_t* empty;
+  uint64_t* sync_bar;        // consumer-wide barrier with a bounded wait (flush)
+  unsigned long long* item_id;   // [stages] work item whose reference tile a stage holds
   unsigned long long* cnt;   // [3][kMaxKC] mism, nan, inf
   unsigned long long* key;   // [kMaxKC]
   const void** ptrs;         // [kMaxKC] candidate pointers of the current chunk (producer only)
@@ -112,7 +112,7 @@ struct StreamSmem {
 
 __host__ __device__ inline size_t stream_smem_bytes(uint32_t stages, uint32_t tile_bytes) {
   size_t b = (size_t)stages * tile_bytes;
-  b += 2 * (size_t)stages * 8;
+  b += 3 * (size_t)stages * 8 + 8;
   b += 3 * (size_t)kMaxKC * 8 + (size_t)kMaxKC * 8 + (size_t)kMaxKC * 8 + (size_t)kMaxKC * 4;
   b += (size_t)kMaxKC * kWarps * 8;
   b += 16;
@@ -151,6 +151,10 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
     q += (size_t)p.stages * 8;
     s.empty = reinterpret_cast<uint64_t*>(q);
     q += (size_t)p.stages * 8;
+    s.sync_bar = reinterpret_cast<uint64_t*>(q);
+    q += 8;
+    s.item_id = reinterpret_cast<unsigned long long*>(q);
+    q += (size_t)p.stages * 8;
     s.cnt = reinterpret_cast<unsigned long long*>(q);
     q += 3 * (size_t)kMaxKC * 8;
     s.key = reinterpret_cast<unsigned long long*>(q);
@@ -174,6 +178,7 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
       mbar_init(&s.full[i], 1);
       mbar_init(&s.empty[i], kWarps);
     }
+    mbar_init(s.sync_bar, kWarps);
     *s.abort_flag = 0u;
     mbar_fence_init();
   }
@@ -187,12 +192,11 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
   for (int i = tid; i < kMaxKC * kWarps; i += kStreamThreads) s.thr2[i] = make_float2(-1.0f, 0.0f);
   __syncthreads();
 
-  // Work items (chunk, tile), chunk-major; each CTA takes one contiguous run of them, so
-  // that it stays with one chunk (warm thresholds) and walks tiles in ascending order.
+  // Work items (chunk, tile), chunk-major, are drawn from a global counter: a CTA gets
+  // ascending items (so ascending tiles inside a chunk, which the index tie-break needs),
+  // the CTAs that run together work on neighbouring tiles, and the tail is one item long.
   const unsigned long long nitems = (unsigned long long)p.nchunks * p.ntiles;
-  const unsigned long long per_cta = (nitems + gridDim.x - 1) / gridDim.x;
-  const unsigned long long item_lo = per_cta * blockIdx.x < nitems ? per_cta * blockIdx.x : nitems;
-  const unsigned long long item_hi = item_lo + per_cta < nitems ? item_lo + per_cta : nitems;
+  constexpr unsigned long long kNoItem = ~0ull;
 
   if (warp == kWarps) {
     // ------------------------------ producer ------------------------------
@@ -202,7 +206,12 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
     unsigned long long issued = 0;
     bool ok = true;
     int cur_chunk = -1;
-    for (unsigned long long item = item_lo; item < item_hi; ++item) {
+    unsigned long long next_item = 0ull;
+    if (lane == 0) next_item = atomicAdd(p.sched, 1ull);
+    for (;;) {
+      const unsigned long long item = __shfl_sync(0xFFFFFFFFu, next_item, 0);
+      if (item >= nitems) break;
+      if (lane == 0) next_item = atomicAdd(p.sched, 1ull);   // drawn one item ahead: latency hidden
       const uint32_t chunk = (uint32_t)(item / p.ntiles);
       const uint32_t slot = p.slot0 + (uint32_t)(item % p.ntiles);
       const uint32_t k0 = chunk * p.KC;
@@ -214,24 +223,37 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
         for (int i = lane; i < kc; i += 32) s.ptrs[i] = p.cands[k0 + i];
         __syncwarp();
       }
-      if (lane != 0 || !ok) continue;
-      const uint32_t tile = p.tile_list ? p.tile_list[slot] : slot;
-      const size_t off = (size_t)tile * TILE_BYTES;
-      for (int kk = -1; kk < kc; ++kk) {
-        if (!mbar_wait_bounded(&s.empty[stage], phase ^ 1u, s.abort_flag, p.status)) {
-          ok = false;
-          break;
+      if (lane == 0) {
+        const uint32_t tile = p.tile_list ? p.tile_list[slot] : slot;
+        const size_t off = (size_t)tile * TILE_BYTES;
+        for (int kk = -1; kk < kc; ++kk) {
+          if (!mbar_wait_bounded(&s.empty[stage], phase ^ 1u, s.abort_flag, p.status)) {
+            ok = false;
+            break;
+          }
+          if (kk < 0) s.item_id[stage] = item;   // visible to the consumers with the phase
+          const unsigned char* src =
+              reinterpret_cast<const unsigned char*>(kk < 0 ? p.ref : s.ptrs[kk]) + off;
+          mbar_arrive_expect_tx(&s.full[stage], TILE_BYTES);
+          bulk_g2s(s.buf + (size_t)stage * TILE_BYTES, src, TILE_BYTES, &s.full[stage],
+                   (kk < 0 && p.nchunks > 1) ? pol_last : pol_first);
+          ++issued;
+          if (++stage == stages) {
+            stage = 0;
+            phase ^= 1u;
+          }
         }
-        const unsigned char* src =
-            reinterpret_cast<const unsigned char*>(kk < 0 ? p.ref : s.ptrs[kk]) + off;
-        mbar_arrive_expect_tx(&s.full[stage], TILE_BYTES);
-        bulk_g2s(s.buf + (size_t)stage * TILE_BYTES, src, TILE_BYTES, &s.full[stage],
-                 (kk < 0 && p.nchunks > 1) ? pol_last : pol_first);
-        ++issued;
-        if (++stage == stages) {
-          stage = 0;
-          phase ^= 1u;
-        }
+      }
+      ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
+      if (!ok) break;
+    }
+    if (lane == 0 && ok) {
+      // no more work: an empty stage that carries the end marker
+      if (mbar_wait_bounded(&s.empty[stage], phase ^ 1u, s.abort_flag, p.status)) {
+        s.item_id[stage] = kNoItem;
+        mbar_arrive(&s.full[stage]);
+      } else {
+        ok = false;
       }
     }
     if (lane == 0 && !ok) {
@@ -254,11 +276,20 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
     uint32_t cur_k0 = 0;
     bool ok = true;
 
-    // Every consumer warp calls flush the same number of times, also after a
-    // wait gave up (ok == false), so the named barrier can never be left waiting.
-    auto flush = [&]() {
-      consumers_sync();
-      for (int i = tid; ok && i < cur_kc; i += kConsumers) {
+    // Consumer-wide barrier whose wait is bounded (a timed-out warp raises the abort flag,
+    // which releases everyone else's waits as well).
+    uint32_t sync_phase = 0;
+    auto consumers_barrier = [&]() -> bool {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(s.sync_bar);
+      const bool done = mbar_wait_bounded(s.sync_bar, sync_phase, s.abort_flag, p.status);
+      sync_phase ^= 1u;
+      return done;
+    };
+    // Move the chunk's shared-memory accumulators to global memory and reset them.
+    auto flush = [&]() -> bool {
+      if (!consumers_barrier()) return false;
+      for (int i = tid; i < cur_kc; i += kConsumers) {
         Acc* a = &p.acc[cur_k0 + i];
         unsigned long long v;
         if ((v = s.cnt[i]) != 0ull) atomicAdd(&a->mism, v);
@@ -274,7 +305,7 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
         s.rel[i] = 0u;
       }
       for (int i = tid; i < kMaxKC * kWarps; i += kConsumers) s.thr2[i] = make_float2(-1.0f, 0.0f);
-      consumers_sync();
+      return consumers_barrier();
     };
 
     // Exchange of running maxima with the other CTAs.  Every merge is a maximum, so the
@@ -319,19 +350,28 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
       __syncwarp();
     };
 
-    for (unsigned long long item = item_lo; item < item_hi; ++item) {
+    for (;;) {
+      // the next stage holds a reference tile and names its work item (or the end)
+      if (!mbar_wait_bounded(&s.full[stage], phase, s.abort_flag, p.status)) {
+        ok = false;
+        break;
+      }
+      const unsigned long long item = *reinterpret_cast<volatile unsigned long long*>(&s.item_id[stage]);
+      if (item == kNoItem) break;
       const uint32_t chunk = (uint32_t)(item / p.ntiles);
       const uint32_t slot = p.slot0 + (uint32_t)(item % p.ntiles);
       const uint32_t tile = p.tile_list ? p.tile_list[slot] : slot;
       const bool first_of_chunk = (int)chunk != cur_chunk;
-      if ((int)chunk != cur_chunk) {
+      if (first_of_chunk) {
         xpending = false;
-        if (cur_chunk >= 0) flush();
+        if (cur_chunk >= 0 && !flush()) {
+          ok = false;
+          break;
+        }
         cur_chunk = (int)chunk;
         cur_k0 = chunk * p.KC;
         cur_kc = (int)min(p.KC, p.K - cur_k0);
       }
-      if (!ok) continue;
       const unsigned long long tile_base = (unsigned long long)tile * kTile;
 
       if (xpending) exchange_apply(tile_base);
@@ -343,10 +383,6 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
       bool extreme = false;   // 0 < |r| < 2^-100: the fused multiply-add of the filter could
                               // underflow to zero and lose its sign; such threads go exact
       {
-        if (!mbar_wait_bounded(&s.full[stage], phase, s.abort_flag, p.status)) {
-          ok = false;
-          continue;
-        }
         const uint4* src = reinterpret_cast<const uint4*>(s.buf + (size_t)stage * TILE_BYTES);
         uint4 w[NV];
 #pragma unroll
@@ -489,8 +525,9 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
         }
         __syncwarp();
       }
+      if (!ok) break;
     }
-    if (cur_chunk >= 0) flush();
+    if (ok && cur_chunk >= 0) flush();
   }
   // ---- the last CTA to get here unpacks all K records (saves a launch) ----
   __shared__ unsigned int s_ticket;
@@ -620,7 +657,11 @@ __global__ void screen_prep_kernel(const PtrChunk chunk, const void** table, Acc
     z.rel = z.pad = 0u;
     acc[offset + i] = z;
   }
-  if (i == 0) *done = 0u;
+  if (i == 0) {
+    done[0] = 0u;   // ticket counter
+    done[1] = 0u;   // work counter (64 bits)
+    done[2] = 0u;
+  }
 }
 
 }  // namespace kb
