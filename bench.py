@@ -149,7 +149,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -163,7 +163,7 @@ def main():
 
     import torch
     import torch.distributed as dist
-    from paper_2608_02611_b200 import binding, synth
+    from paper_2608_02611_b200 import binding, sharding, synth
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -227,9 +227,7 @@ def main():
     wins_ms = ctx.read_timer(binding.KB_TIMER_WINS)
     ctx.enable_timing(False)
     if world > 1:
-        t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
+        elapsed_ms = sharding.max_over_ranks(elapsed_ms, dev)
     ms_per_step = elapsed_ms / steps
     value = world * K_CANDS * N / (ms_per_step * 1e-3)
 
@@ -258,9 +256,7 @@ def main():
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
     if world > 1:
-        t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
+        e2e_s = sharding.max_over_ranks(e2e_s, dev)
     esz = synth.ELEM_SIZE[case.dtype]
     h2d = (K_CANDS + 1) * N * esz + K_CANDS * S_TIMINGS * 4 + K_CANDS * binding.RESULT_BYTES
     d2h = K_CANDS * binding.RESULT_BYTES + BUDGET * 4 + 4 + 2 * K_CANDS * 4 + K_CANDS * K_CANDS * 4
