@@ -125,6 +125,11 @@ kb_status kb_ctx_enable_timing(kb_ctx* ctx, int on);
  * durations in milliseconds (oldest first, at most `cap`) to h_ms (HOST) and
  * their number to *n (HOST); the record is then cleared. */
 kb_status kb_ctx_read_timer(kb_ctx* ctx, kb_timer which, float* h_ms, uint32_t cap, uint32_t* n);
+/* Choose how kb_adjudicate counts wins: 0 = automatic (binary search on the
+ * sorted rows when 8 rows fit shared memory, i.e. S <= 4096, else direct
+ * comparison), 1 = always direct comparison of all sample pairs, 2 = always
+ * binary search (S <= 4096 only).  The integers produced are identical. */
+kb_status kb_ctx_set_wins_algo(kb_ctx* ctx, int algo);
 /* Number of kernels this context has launched since it was created (HOST out). */
 kb_status kb_ctx_launch_count(const kb_ctx* ctx, uint64_t* n);
 

@@ -35,7 +35,7 @@ RESULT_BYTES = 48
 
 EXPORTS = [
     "kb_ctx_create", "kb_ctx_destroy", "kb_last_error", "kb_ctx_poll", "kb_ctx_set_grid",
-    "kb_ctx_enable_timing", "kb_ctx_read_timer", "kb_ctx_launch_count",
+    "kb_ctx_enable_timing", "kb_ctx_read_timer", "kb_ctx_launch_count", "kb_ctx_set_wins_algo",
     "kb_mask_create_strided", "kb_mask_create_bitmap", "kb_mask_count", "kb_mask_destroy",
     "kb_screen", "kb_screen_host", "kb_screen_static", "kb_adjudicate", "kb_select",
 ]
@@ -72,6 +72,7 @@ def load() -> ctypes.CDLL:
     L.kb_ctx_enable_timing.argtypes = [vp, i32]
     L.kb_ctx_read_timer.argtypes = [vp, i32, vp, u32, ctypes.POINTER(u32)]
     L.kb_ctx_launch_count.argtypes = [vp, ctypes.POINTER(u64)]
+    L.kb_ctx_set_wins_algo.argtypes = [vp, i32]
     L.kb_mask_create_strided.argtypes = [vp, u64, u32, u32, u32, pvp]
     L.kb_mask_create_bitmap.argtypes = [vp, u64, u32, vp, pvp]
     L.kb_mask_count.argtypes = [vp, ctypes.POINTER(u64)]
@@ -155,6 +156,10 @@ class Context:
 
     def set_grid(self, blocks: int):
         self._check(load().kb_ctx_set_grid(self._h, int(blocks)), "kb_ctx_set_grid")
+
+    def set_wins_algo(self, algo: int):
+        """0 automatic, 1 direct comparison of all sample pairs, 2 binary search on sorted rows."""
+        self._check(load().kb_ctx_set_wins_algo(self._h, int(algo)), "kb_ctx_set_wins_algo")
 
     def enable_timing(self, on: bool = True):
         self._check(load().kb_ctx_enable_timing(self._h, 1 if on else 0), "kb_ctx_enable_timing")

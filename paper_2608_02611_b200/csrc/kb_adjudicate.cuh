@@ -4,7 +4,12 @@
 // rows_kernel         one CTA per candidate: sort its S timings in shared
 //                     memory (bitonic), take the type-7 quartiles with the
 //                     operation order fixed, write median and IQR.
-// wins_kernel         pairwise doubled Mann-Whitney counts.  A CTA takes a
+// wins_rank_kernel    the same integers from the SORTED rows: for a sample x of
+//                     row a, lb = #{b_j < x} and ub = #{b_j <= x} by binary search
+//                     in row b; W[b][a] = sum_x (lb + ub), W[a][b] = 2*S*S - that.
+//                     O(K^2 S log S) instead of O(K^2 S^2); the default when a
+//                     block of 8 sorted rows fits shared memory (S <= 4096).
+// wins_kernel         pairwise doubled Mann-Whitney counts by direct comparison.  A CTA takes a
 //                     block of 8 "a" rows x 8 "b" rows and a chunk of samples
 //                     of each; the a-chunk is staged in shared memory, each
 //                     warp owns one b row and each lane keeps up to 8 of its
@@ -27,6 +32,7 @@ __global__ void __launch_bounds__(kRowsThreads) rows_kernel(const float* __restr
                                                             unsigned int S, unsigned int P /*pow2 >= S*/,
                                                             float* __restrict__ median,
                                                             float* __restrict__ iqr,
+                                                            float* __restrict__ sorted_out /*[K][S] or NULL*/,
                                                             unsigned int* status) {
   extern __shared__ float xs[];
   const unsigned int k = blockIdx.x;
@@ -57,6 +63,9 @@ __global__ void __launch_bounds__(kRowsThreads) rows_kernel(const float* __restr
       }
       __syncthreads();
     }
+  }
+  if (sorted_out) {
+    for (unsigned int i = threadIdx.x; i < S; i += kRowsThreads) sorted_out[(size_t)k * S + i] = xs[i];
   }
   if (threadIdx.x == 0) {
     float q[4];
@@ -181,6 +190,58 @@ __global__ void __launch_bounds__(kWinsThreads) wins_kernel(const WinsParams p) 
         if (total) atomicAdd(wab, total);
         if (Ab != Bb && mirror) atomicAdd(wba, mirror);
       }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
+struct WinsRankParams {
+  const float* sorted;   // [K][S], each row ascending
+  unsigned int* wins;
+  unsigned int K, S, P;  // P: smallest power of two > S
+  unsigned int KB, TA;   // blocks of 8 rows; a rows per CTA
+};
+
+__global__ void __launch_bounds__(kWinsThreads) wins_rank_kernel(const WinsRankParams p) {
+  extern __shared__ float bs[];   // [8][S] sorted b rows
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const unsigned int nsub = kWinsRowsPerBlock / p.TA;
+  const unsigned int sub = blockIdx.x % nsub;
+  const unsigned int pair = blockIdx.x / nsub;
+  unsigned int Ab = 0, rem = pair;
+  while (rem >= p.KB - Ab) {
+    rem -= p.KB - Ab;
+    ++Ab;
+  }
+  const unsigned int Bb = Ab + rem;
+  const unsigned int b0 = Bb * kWinsRowsPerBlock;
+  const unsigned int nb = min((unsigned int)kWinsRowsPerBlock, p.K - b0);
+  for (unsigned int t = threadIdx.x; t < nb * p.S; t += kWinsThreads) bs[t] = p.sorted[(size_t)b0 * p.S + t];
+  __syncthreads();
+  const unsigned int b = b0 + warp;
+  if (b >= p.K) return;
+  const float* brow = bs + (size_t)warp * p.S;
+  const unsigned int a0 = Ab * kWinsRowsPerBlock + sub * p.TA;
+  for (unsigned int rr = 0; rr < p.TA; ++rr) {
+    const unsigned int a = a0 + rr;
+    if (a >= p.K) break;
+    const float* arow = p.sorted + (size_t)a * p.S;
+    unsigned int sum = 0u;
+    for (unsigned int i = lane; i < p.S; i += 32) {
+      const float x = arow[i];
+      unsigned int lb = 0u;                       // number of b samples < x
+      for (unsigned int step = p.P >> 1; step > 0; step >>= 1) {
+        const unsigned int nxt = lb + step;
+        if (nxt <= p.S && brow[nxt - 1] < x) lb = nxt;
+      }
+      unsigned int ub = lb;                       // number of b samples <= x
+      while (ub < p.S && brow[ub] == x) ++ub;
+      sum += lb + ub;
+    }
+    sum = warp_add_u32(sum);
+    if (lane == 0) {
+      p.wins[(size_t)a * p.K + b] = 2u * p.S * p.S - sum;
+      if (Ab != Bb) p.wins[(size_t)b * p.K + a] = sum;
     }
   }
 }

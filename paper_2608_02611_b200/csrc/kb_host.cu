@@ -23,6 +23,9 @@ struct kb_ctx {
   size_t ws_bytes = 0;
   unsigned int* d_status = nullptr;
   uint32_t forced_grid = 0;
+  int wins_algo = 0;                // 0 auto, 1 direct comparison, 2 binary search on sorted rows
+  float* srt = nullptr;             // [K][S] sorted timings (binary-search win count)
+  size_t srt_bytes = 0;
   char err[512] = {0};
   // staging owned for kb_screen_host
   unsigned char* st_ref = nullptr;
@@ -236,6 +239,11 @@ extern "C" kb_status kb_ctx_create(int device, kb_ctx** out) {
     fail(ctx, KB_ERR_CUDA, "cannot raise the shared-memory limit of the row kernel");
     return bail(KB_ERR_CUDA);
   }
+  if (cudaFuncSetAttribute(wins_rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           kWinsRowsPerBlock * 4096 * (int)sizeof(float)) != cudaSuccess) {
+    fail(ctx, KB_ERR_CUDA, "cannot raise the shared-memory limit of the win-count kernel");
+    return bail(KB_ERR_CUDA);
+  }
   *out = ctx;
   return KB_OK;
 }
@@ -247,6 +255,7 @@ extern "C" kb_status kb_ctx_destroy(kb_ctx* ctx) {
   if (ctx->ws) cudaFree(ctx->ws);
   if (ctx->d_status) cudaFree(ctx->d_status);
   if (ctx->st_ref) cudaFree(ctx->st_ref);
+  if (ctx->srt) cudaFree(ctx->srt);
   for (int i = 0; i < 2; ++i) {
     if (ctx->st_batch[i]) cudaFree(ctx->st_batch[i]);
     if (ctx->ev_copied[i]) cudaEventDestroy(ctx->ev_copied[i]);
@@ -281,6 +290,12 @@ extern "C" kb_status kb_ctx_poll(kb_ctx* ctx, void* stream, kb_status* device_st
 extern "C" kb_status kb_ctx_set_grid(kb_ctx* ctx, uint32_t blocks) {
   if (!ctx) return KB_ERR_INVALID_ARG;
   ctx->forced_grid = blocks;
+  return KB_OK;
+}
+
+extern "C" kb_status kb_ctx_set_wins_algo(kb_ctx* ctx, int algo) {
+  if (!ctx || algo < 0 || algo > 2) return KB_ERR_INVALID_ARG;
+  ctx->wins_algo = algo;
   return KB_OK;
 }
 
@@ -733,14 +748,54 @@ extern "C" kb_status kb_adjudicate(kb_ctx* ctx, const float* d_timings, uint32_t
   DeviceGuard g(ctx->device);
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
 
+  // which win-count algorithm
+  bool rank = d_wins && S <= 4096 && ctx->wins_algo != 1;
+  if (ctx->wins_algo == 2 && d_wins && S > 4096)
+    return fail(ctx, KB_ERR_UNSUPPORTED, "kb_adjudicate: the binary-search win count needs S <= 4096");
+  if (rank) {
+    size_t have = ctx->srt_bytes;
+    if (ensure_buf(ctx, &ctx->srt, &have, (size_t)K * S * sizeof(float)) == KB_OK) {
+      ctx->srt_bytes = have;
+    } else if (ctx->wins_algo == 2) {
+      return KB_ERR_WORKSPACE;
+    } else {
+      ctx->srt_bytes = 0;
+      rank = false;     // no room for the sorted copy: count by direct comparison
+    }
+  }
   // rows: sort + quartiles (also the place where non-finite timings are caught)
   unsigned int P = 1;
   while (P < S) P <<= 1;
   rows_kernel<<<K, kRowsThreads, (size_t)P * sizeof(float), st>>>(d_timings, S, P, d_median, d_iqr,
+                                                                   rank ? ctx->srt : nullptr,
                                                                    ctx->d_status);
   ++ctx->launches;
   KB_CUDA(ctx, cudaGetLastError());
   if (!d_wins) return KB_OK;
+
+  if (rank) {
+    WinsRankParams rp;
+    rp.sorted = ctx->srt;
+    rp.wins = d_wins;
+    rp.K = K;
+    rp.S = S;
+    rp.P = 1;
+    while (rp.P <= S) rp.P <<= 1;
+    rp.KB = (K + kWinsRowsPerBlock - 1) / kWinsRowsPerBlock;
+    const unsigned long long npairs_r = (unsigned long long)rp.KB * (rp.KB + 1) / 2;
+    rp.TA = kWinsRowsPerBlock;
+    while (npairs_r * (kWinsRowsPerBlock / rp.TA) < 2ull * ctx->sm_count && rp.TA > 1) rp.TA /= 2;
+    const unsigned long long grid_r = npairs_r * (kWinsRowsPerBlock / rp.TA);
+    if (grid_r > 0x7FFFFFFFull) return fail(ctx, KB_ERR_UNSUPPORTED, "kb_adjudicate: K too large for one launch");
+    {
+      ScopedTimer tm(ctx, KB_TIMER_WINS, st);
+      wins_rank_kernel<<<(unsigned int)grid_r, kWinsThreads,
+                         (size_t)kWinsRowsPerBlock * S * sizeof(float), st>>>(rp);
+    }
+    ++ctx->launches;
+    KB_CUDA(ctx, cudaGetLastError());
+    return KB_OK;
+  }
 
   WinsParams wp;
   wp.timings = d_timings;

@@ -357,6 +357,8 @@ def test_argument_errors(ctx, kb):
                                  (8, 31), (9, 32), (17, 33), (33, 64), (16, 100), (24, 200), (7, 256),
                                  (6, 257), (5, 300), (12, 1000), (4, 2000), (3, 2049)])
 def test_adjudicate_matches_oracle(ctx, kb, K, S):
+    """Both win-count algorithms (direct comparison of all sample pairs; binary search on
+    the sorted rows) give the oracle's integers."""
     rng = np.random.default_rng(K * 10007 + S)
     dev = torch.device("cuda", 0)
     for ties in (False, True):
@@ -364,22 +366,47 @@ def test_adjudicate_matches_oracle(ctx, kb, K, S):
         if ties:
             t = np.round(t, 2)
         t = t.astype(np.float32)
-        med, iqr, wins = ctx.adjudicate(torch.from_numpy(t).to(dev))
-        assert ctx.poll() == 0
         omed, oiqr, owins = oracle.adjudicate(t)
-        assert (fbits(med.cpu().numpy()) == fbits(omed)).all()
-        assert (fbits(iqr.cpu().numpy()) == fbits(oiqr)).all()
-        w = wins.cpu().numpy().view(np.uint32)
-        assert (w == owins).all(), np.argwhere(w != owins)[:5]
+        for algo in (1, 2, 0):
+            try:
+                ctx.set_wins_algo(algo)
+                med, iqr, wins = ctx.adjudicate(torch.from_numpy(t).to(dev))
+            finally:
+                ctx.set_wins_algo(0)
+            assert ctx.poll() == 0
+            assert (fbits(med.cpu().numpy()) == fbits(omed)).all()
+            assert (fbits(iqr.cpu().numpy()) == fbits(oiqr)).all()
+            w = wins.cpu().numpy().view(np.uint32)
+            assert (w == owins).all(), (algo, np.argwhere(w != owins)[:5])
+
+
+def test_adjudicate_long_rows_use_direct_comparison(ctx, kb):
+    """S > 4096: a block of sorted rows no longer fits shared memory."""
+    rng = np.random.default_rng(4097)
+    dev = torch.device("cuda", 0)
+    t = np.round(rng.lognormal(0, 0.1, (3, 4100)), 3).astype(np.float32)
+    med, iqr, wins = ctx.adjudicate(torch.from_numpy(t).to(dev))
+    omed, oiqr, owins = oracle.adjudicate(t)
+    assert (fbits(med.cpu().numpy()) == fbits(omed)).all()
+    assert (wins.cpu().numpy().view(np.uint32) == owins).all()
+    ctx.set_wins_algo(2)
+    try:
+        with pytest.raises(kb.KbError):
+            ctx.adjudicate(torch.from_numpy(t).to(dev))
+    finally:
+        ctx.set_wins_algo(0)
 
 
 def test_adjudicate_negative_and_zero_timings(ctx, kb):
     dev = torch.device("cuda", 0)
     t = np.float32([[0.0, -1.0, 2.0, 0.0, 1.0], [1.0, 0.0, -2.0, 5.0, 1.0], [3.0, 3.0, 3.0, 3.0, 3.0]])
-    med, iqr, wins = ctx.adjudicate(torch.from_numpy(t).to(dev))
     omed, oiqr, owins = oracle.adjudicate(t)
-    assert (med.cpu().numpy() == omed).all() and (iqr.cpu().numpy() == oiqr).all()
-    assert (wins.cpu().numpy().view(np.uint32) == owins).all()
+    for algo in (1, 2):
+        ctx.set_wins_algo(algo)
+        med, iqr, wins = ctx.adjudicate(torch.from_numpy(t).to(dev))
+        ctx.set_wins_algo(0)
+        assert (med.cpu().numpy() == omed).all() and (iqr.cpu().numpy() == oiqr).all()
+        assert (wins.cpu().numpy().view(np.uint32) == owins).all()
 
 
 def test_adjudicate_flags_nonfinite(ctx, kb):
