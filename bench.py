@@ -37,7 +37,7 @@ K_CANDS, SIDE, S_TIMINGS, BUDGET = 64, 4096, 100, 32
 # DRAM bytes moved per algorithmic byte by the streaming screen kernel, from the ncu capture
 # summarised in profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over (K+1)*N*2 bytes);
 # captured at side 2048 (545 MB) and scaled by the bytes a full launch processes.
-DRAM_BYTES_PER_ALGORITHMIC_BYTE = 1.0076
+DRAM_BYTES_PER_ALGORITHMIC_BYTE = 1.0068
 
 WORKLOAD = ("config2: screen K=64 bf16 4096x4096 (atol=1e-2, rtol=1.6e-2) + adjudicate "
             "timings[64][100] + select top 32")
@@ -146,6 +146,52 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def run_adjudicate(args):
+    """kb_adjudicate alone: logical comparisons/s = K^2 S^2 / t; for the direct-comparison kernel
+    also the executed sample-pair evaluations against the ALU-pipe roofline."""
+    import torch
+    from paper_2608_02611_b200 import binding, synth
+    dev = torch.device("cuda", 0)
+    ctx = binding.Context(0)
+    ctx.set_wins_algo(args.wins_algo)
+    K, S = args.K, args.S
+    t_k = synth.base_latencies(synth.MASTER_SEED + 5, K, 0.3)
+    timings = synth.lognormal_timings(synth.MASTER_SEED + 5, t_k, S, 0.15)
+    d_t = torch.from_numpy(timings).to(dev)
+    steps, warmup = max(1, min(args.steps, 200)), max(3, args.warmup)
+    for _ in range(warmup):
+        ctx.adjudicate(d_t)
+    torch.cuda.synchronize()
+    ctx.enable_timing(True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        ctx.adjudicate(d_t)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    wins_ms = float(np.mean(ctx.read_timer(binding.KB_TIMER_WINS)))
+    assert ctx.poll() == 0
+    logical = K * K * S * S
+    line = {"workload": f"adjudicate timings[{K}][{S}]", "wins_algo": args.wins_algo,
+            "ms_per_call": ms, "wins_kernel_ms": wins_ms,
+            "pairwise_comparisons_per_s": logical / (wins_ms * 1e-3), "steps": steps}
+    direct = args.wins_algo == 1 or S > 4096
+    if direct:
+        # every unordered block pair once; R*32 sample slots per lane row; 3 ALU-pipe
+        # instructions (set.lt, set.le, 3-input add) per 32 sample pairs
+        KB = (K + 7) // 8
+        nj = (S + 255) // 256
+        R = ((S + nj - 1) // nj + 31) // 32
+        evals = KB * (KB + 1) // 2 * 64 * S * (nj * R * 32)
+        peak = 148 * 64 * 1.965e9 / 3          # sample-pair evaluations/s at 64 ALU lanes/clk/SM
+        line["roofline"] = {"bound": "alu", "achieved": evals / (wins_ms * 1e-3), "peak": peak,
+                            "unit": "sample-pair evaluations/s", "frac": evals / (wins_ms * 1e-3) / peak,
+                            "traffic": None}
+    print(json.dumps(line), flush=True)
+    ctx.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -154,12 +200,21 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--workload", default="step", choices=["step", "adjudicate"],
+                    help="'adjudicate' times kb_adjudicate alone on timings[K][S] (config 5 tier 1 by "
+                         "default) and reports pairwise comparisons/s against the ALU roofline; it is a "
+                         "secondary measurement, not the benchmark line")
+    ap.add_argument("--K", type=int, default=512)
+    ap.add_argument("--S", type=int, default=200)
+    ap.add_argument("--wins-algo", type=int, default=0, choices=[0, 1, 2])
     ap.add_argument("--side", type=int, default=SIDE,
                     help="tensor side; anything but 4096 is for profiler captures only and is "
                          "not a benchmark configuration")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.workload == "adjudicate":
+        return run_adjudicate(args)
 
     import torch
     import torch.distributed as dist
@@ -193,9 +248,20 @@ def main():
     out = torch.empty((K_CANDS, binding.RESULT_BYTES), dtype=torch.uint8, device=dev)
     torch.cuda.synchronize()
 
+    # The gate and the adjudication do not depend on each other: they go to two streams (each
+    # with its own context, since a context serves one stream at a time) and join for select.
+    ctx_adj = binding.Context(local_rank)
+    main = torch.cuda.current_stream(dev)
+    side = torch.cuda.Stream(dev)
+
     def step():
+        side.wait_stream(main)
+        with torch.cuda.stream(side):
+            med, iqr, wins = ctx_adj.adjudicate(d_timings)
         ctx.screen(case.ref, cands, case.atol, case.rtol, out=out)
-        med, iqr, wins = ctx.adjudicate(d_timings)
+        main.wait_stream(side)
+        for t in (med, iqr, wins):
+            t.record_stream(main)
         return ctx.select(out, med, binding.KB_SELECT_ERR_THEN_TIME, BUDGET)
 
     def barrier():
@@ -206,13 +272,14 @@ def main():
     for _ in range(warmup):
         step()
     barrier()
-    assert ctx.poll() == 0
+    assert ctx.poll() == 0 and ctx_adj.poll() == 0
 
     # ---- timed region: exactly `steps` steps, CUDA events, clocks sampled meanwhile ----
     sampler = ClockSampler(local_rank)
     sampler.start()
     ctx.enable_timing(True)
-    launches0 = ctx.launch_count
+    ctx_adj.enable_timing(True)
+    launches0 = ctx.launch_count + ctx_adj.launch_count
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     e0.record()
@@ -222,10 +289,11 @@ def main():
     barrier()
     clocks = sampler.stop()
     elapsed_ms = e0.elapsed_time(e1)
-    launches = ctx.launch_count - launches0
+    launches = ctx.launch_count + ctx_adj.launch_count - launches0
     stream_ms = ctx.read_timer(binding.KB_TIMER_SCREEN_STREAM)
-    wins_ms = ctx.read_timer(binding.KB_TIMER_WINS)
+    wins_ms = ctx_adj.read_timer(binding.KB_TIMER_WINS)
     ctx.enable_timing(False)
+    ctx_adj.enable_timing(False)
     if world > 1:
         elapsed_ms = sharding.max_over_ranks(elapsed_ms, dev)
     ms_per_step = elapsed_ms / steps
@@ -242,7 +310,7 @@ def main():
     def e2e_step():
         rec = ctx.screen_host(h_ref, h_cands, case.atol, case.rtol)          # H2D + D2H inside
         dt = h_timings.to(dev, non_blocking=True)
-        med, iqr, wins = ctx.adjudicate(dt)
+        med, iqr, wins = ctx_adj.adjudicate(dt)
         d_rec = torch.from_numpy(rec.view(np.uint8).reshape(K_CANDS, binding.RESULT_BYTES)).to(dev)
         surv, n = ctx.select(d_rec, med, binding.KB_SELECT_ERR_THEN_TIME, BUDGET)
         return surv.cpu(), n.cpu(), med.cpu(), iqr.cpu(), wins.cpu()

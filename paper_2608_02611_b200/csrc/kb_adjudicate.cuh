@@ -5,9 +5,11 @@
 //                     memory (bitonic), take the type-7 quartiles with the
 //                     operation order fixed, write median and IQR.
 // wins_rank_kernel    the same integers from the SORTED rows: for a sample x of
-//                     row a, lb = #{b_j < x} and ub = #{b_j <= x} by binary search
-//                     in row b; W[b][a] = sum_x (lb + ub), W[a][b] = 2*S*S - that.
-//                     O(K^2 S log S) instead of O(K^2 S^2); the default when a
+//                     row a, lb = #{b_j < x} and ub = #{b_j <= x}; W[b][a] =
+//                     sum_x (lb + ub), W[a][b] = 2*S*S - that.  A warp takes a
+//                     pair of rows, each lane a contiguous run of a's samples:
+//                     one binary search, then a merge walk.  O(K^2 (S + 32 log S))
+//                     instead of O(K^2 S^2); the default when a
 //                     block of 8 sorted rows fits shared memory (S <= 4096).
 // wins_kernel         pairwise doubled Mann-Whitney counts by direct comparison.  A CTA takes a
 //                     block of 8 "a" rows x 8 "b" rows and a chunk of samples
@@ -226,17 +228,27 @@ __global__ void __launch_bounds__(kWinsThreads) wins_rank_kernel(const WinsRankP
     const unsigned int a = a0 + rr;
     if (a >= p.K) break;
     const float* arow = p.sorted + (size_t)a * p.S;
+    // Each lane takes a contiguous run of a's sorted samples: one binary search for the
+    // first, then both rows are walked in step (a merge), since lb and ub only grow.
+    const unsigned int L = (p.S + 31) / 32;
+    const unsigned int i0 = lane * L;
+    const unsigned int i1 = min(i0 + L, p.S);
     unsigned int sum = 0u;
-    for (unsigned int i = lane; i < p.S; i += 32) {
-      const float x = arow[i];
+    if (i0 < i1) {
+      const float x0 = arow[i0];
       unsigned int lb = 0u;                       // number of b samples < x
       for (unsigned int step = p.P >> 1; step > 0; step >>= 1) {
         const unsigned int nxt = lb + step;
-        if (nxt <= p.S && brow[nxt - 1] < x) lb = nxt;
+        if (nxt <= p.S && brow[nxt - 1] < x0) lb = nxt;
       }
       unsigned int ub = lb;                       // number of b samples <= x
-      while (ub < p.S && brow[ub] == x) ++ub;
-      sum += lb + ub;
+      for (unsigned int i = i0; i < i1; ++i) {
+        const float x = arow[i];
+        while (lb < p.S && brow[lb] < x) ++lb;
+        if (ub < lb) ub = lb;
+        while (ub < p.S && brow[ub] <= x) ++ub;
+        sum += lb + ub;
+      }
     }
     sum = warp_add_u32(sum);
     if (lane == 0) {

@@ -544,7 +544,7 @@ kb_status screen_impl(kb_ctx* ctx, const void* d_ref, const void* const* h_cands
       nscout = sp.ntiles / 128;
       if (nscout < 1) nscout = 1;
       if (nscout > 8) nscout = 8;
-      dim3 sg(nscout * (kTile / 256), K);
+      dim3 sg(nscout * (kTile / kScoutPerBlock), K);
       screen_scout_kernel<DT><<<sg, 256, 0, st>>>(d_ref, table, acc, sp.tile_list, atol, rtol);
       ++ctx->launches;
       KB_CUDA(ctx, cudaGetLastError());
@@ -784,7 +784,7 @@ extern "C" kb_status kb_adjudicate(kb_ctx* ctx, const float* d_timings, uint32_t
     rp.KB = (K + kWinsRowsPerBlock - 1) / kWinsRowsPerBlock;
     const unsigned long long npairs_r = (unsigned long long)rp.KB * (rp.KB + 1) / 2;
     rp.TA = kWinsRowsPerBlock;
-    while (npairs_r * (kWinsRowsPerBlock / rp.TA) < 2ull * ctx->sm_count && rp.TA > 1) rp.TA /= 2;
+    while (npairs_r * (kWinsRowsPerBlock / rp.TA) < 8ull * ctx->sm_count && rp.TA > 1) rp.TA /= 2;
     const unsigned long long grid_r = npairs_r * (kWinsRowsPerBlock / rp.TA);
     if (grid_r > 0x7FFFFFFFull) return fail(ctx, KB_ERR_UNSUPPORTED, "kb_adjudicate: K too large for one launch");
     {

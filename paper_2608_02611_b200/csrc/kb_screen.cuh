@@ -615,7 +615,9 @@ __global__ void __launch_bounds__(256) screen_generic_kernel(const void* __restr
 // Scout: the first `nscout` full tiles (of the list, or tiles 0..nscout-1) of every
 // candidate, classified exactly before the streaming kernel starts.  Their maxima
 // seed the streaming kernel's thresholds, so that its first tile does not have to
-// discover them.  grid = (nscout * kTile / 256, K).
+// discover them.  A block takes 1024 elements of one tile of one candidate and issues
+// one set of atomics.  grid = (nscout * 4, K).
+constexpr unsigned int kScoutPerBlock = 1024;
 template <int DT>
 __global__ void __launch_bounds__(256) screen_scout_kernel(const void* __restrict__ ref,
                                                            const void* const* __restrict__ cands,
@@ -623,14 +625,49 @@ __global__ void __launch_bounds__(256) screen_scout_kernel(const void* __restric
                                                            const uint32_t* __restrict__ tile_list,
                                                            float atol, float rtol) {
   using E = Elem<DT>;
-  constexpr unsigned int kBlocksPerTile = kTile / 256;
+  constexpr unsigned int kBlocksPerTile = kTile / kScoutPerBlock;
+  __shared__ unsigned int s_cnt[3];
+  __shared__ unsigned int s_rel;
+  __shared__ unsigned long long s_key;
+  if (threadIdx.x == 0) {
+    s_cnt[0] = s_cnt[1] = s_cnt[2] = 0u;
+    s_rel = 0u;
+    s_key = 0ull;
+  }
+  __syncthreads();
   const unsigned int k = blockIdx.y;
   const unsigned int slot = blockIdx.x / kBlocksPerTile;
   const unsigned long long tile = tile_list ? tile_list[slot] : slot;
-  const unsigned long long i = tile * kTile + (blockIdx.x % kBlocksPerTile) * 256 + threadIdx.x;
+  const unsigned long long base = tile * kTile + (blockIdx.x % kBlocksPerTile) * kScoutPerBlock;
+  const void* cand = cands[k];
   ExactAcc x;
-  x.add(E::load(ref, i), E::load(cands[k], i), i, atol, rtol);
-  x.commit(&acc[k]);
+#pragma unroll
+  for (unsigned int j = 0; j < kScoutPerBlock / 256; ++j) {
+    const unsigned long long i = base + j * 256 + threadIdx.x;
+    x.add(E::load(ref, i), E::load(cand, i), i, atol, rtol);
+  }
+  // block-level merge in shared memory, then one set of global atomics
+  x.n_mis = warp_add_u32(x.n_mis);
+  x.n_nan = warp_add_u32(x.n_nan);
+  x.n_inf = warp_add_u32(x.n_inf);
+  x.best = warp_max_u64(x.best);
+  x.qb = warp_max_u32(x.qb);
+  if ((threadIdx.x & 31) == 0) {
+    if (x.n_mis) atomicAdd(&s_cnt[0], x.n_mis);
+    if (x.n_nan) atomicAdd(&s_cnt[1], x.n_nan);
+    if (x.n_inf) atomicAdd(&s_cnt[2], x.n_inf);
+    if (x.best) atomicMax(&s_key, x.best);
+    if (x.qb) atomicMax(&s_rel, x.qb);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    Acc* a = &acc[k];
+    if (s_cnt[0]) atomicAdd(&a->mism, (unsigned long long)s_cnt[0]);
+    if (s_cnt[1]) atomicAdd(&a->nan, (unsigned long long)s_cnt[1]);
+    if (s_cnt[2]) atomicAdd(&a->inf, (unsigned long long)s_cnt[2]);
+    if (s_key) atomicMax(&a->key, s_key);
+    if (s_rel) atomicMax(&a->rel, s_rel);
+  }
 }
 
 __global__ void screen_finalize_kernel(const Acc* __restrict__ acc, kb_screen_result* __restrict__ out,

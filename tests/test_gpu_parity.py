@@ -434,3 +434,17 @@ def test_select_matches_oracle(ctx, kb, policy, K, budget):
     osurv, on = oracle.select(rec, med, policy, budget)
     assert int(n.item()) == on
     assert surv.cpu().numpy().tolist() == osurv.tolist()
+
+
+def test_screen_host_matches_screen(ctx, kb):
+    """kb_screen_host (host buffers, batched copies) gives the records of kb_screen."""
+    case, _ = synth.config2("cpu", side=256, K=9, n_bad=2, block=64)
+    N = case.N - 77
+    ref = case.ref[:N].clone()
+    cands = [case.make_cand(k)[:N].clone() for k in range(case.K)]
+    got = ctx.screen_host(ref, cands, case.atol, case.rtol)
+    dev = torch.device("cuda", 0)
+    want = kb.records(ctx.screen(ref.to(dev), [c.to(dev) for c in cands], case.atol, case.rtol))
+    assert got.tobytes() == want.tobytes()
+    oracle_rec = oracle_screen(case.dtype, ref, cands, case.atol, case.rtol)
+    assert_records_equal(got, oracle_rec, "screen_host")
