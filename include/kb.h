@@ -110,6 +110,11 @@ kb_status kb_ctx_poll(kb_ctx* ctx, void* stream, kb_status* device_status);
  * kernel (0 = automatic).  Results do not depend on it. */
 kb_status kb_ctx_set_grid(kb_ctx* ctx, uint32_t blocks);
 
+/* Test/tuning hook: small problems (K <= 480 and K*N <= 2^22 elements) are
+ * screened by a single-launch kernel; on = 0 sends them down the general
+ * (streaming) path instead.  Results do not depend on it. */
+kb_status kb_ctx_set_small_path(kb_ctx* ctx, int on);
+
 /* ---- instrumentation (used by the benchmark; no paper counterpart) ------- */
 
 typedef enum {

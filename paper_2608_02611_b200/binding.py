@@ -35,7 +35,7 @@ RESULT_BYTES = 48
 
 EXPORTS = [
     "kb_ctx_create", "kb_ctx_destroy", "kb_last_error", "kb_ctx_poll", "kb_ctx_set_grid",
-    "kb_ctx_enable_timing", "kb_ctx_read_timer", "kb_ctx_launch_count", "kb_ctx_set_wins_algo",
+    "kb_ctx_enable_timing", "kb_ctx_read_timer", "kb_ctx_launch_count", "kb_ctx_set_wins_algo", "kb_ctx_set_small_path",
     "kb_mask_create_strided", "kb_mask_create_bitmap", "kb_mask_count", "kb_mask_destroy",
     "kb_screen", "kb_screen_host", "kb_screen_static", "kb_adjudicate", "kb_select",
 ]
@@ -73,6 +73,7 @@ def load() -> ctypes.CDLL:
     L.kb_ctx_read_timer.argtypes = [vp, i32, vp, u32, ctypes.POINTER(u32)]
     L.kb_ctx_launch_count.argtypes = [vp, ctypes.POINTER(u64)]
     L.kb_ctx_set_wins_algo.argtypes = [vp, i32]
+    L.kb_ctx_set_small_path.argtypes = [vp, i32]
     L.kb_mask_create_strided.argtypes = [vp, u64, u32, u32, u32, pvp]
     L.kb_mask_create_bitmap.argtypes = [vp, u64, u32, vp, pvp]
     L.kb_mask_count.argtypes = [vp, ctypes.POINTER(u64)]
@@ -156,6 +157,10 @@ class Context:
 
     def set_grid(self, blocks: int):
         self._check(load().kb_ctx_set_grid(self._h, int(blocks)), "kb_ctx_set_grid")
+
+    def set_small_path(self, on: bool):
+        """Enable/disable the single-launch kernel for small problems (a test hook)."""
+        self._check(load().kb_ctx_set_small_path(self._h, 1 if on else 0), "kb_ctx_set_small_path")
 
     def set_wins_algo(self, algo: int):
         """0 automatic, 1 direct comparison of all sample pairs, 2 binary search on sorted rows."""

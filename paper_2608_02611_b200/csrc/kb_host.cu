@@ -23,6 +23,8 @@ struct kb_ctx {
   size_t ws_bytes = 0;
   unsigned int* d_status = nullptr;
   uint32_t forced_grid = 0;
+  unsigned char* small_ws = nullptr; // single-launch path: [tickets 2 KB | partial records 80 KB]
+  bool small_on = true;
   int wins_algo = 0;                // 0 auto, 1 direct comparison, 2 binary search on sorted rows
   float* srt = nullptr;             // [K][S] sorted timings (binary-search win count)
   size_t srt_bytes = 0;
@@ -94,6 +96,9 @@ struct DeviceGuard {
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline int elem_bytes(kb_dtype dt) { return dt == KB_F32 ? 4 : 2; }
+constexpr size_t kSmallTicketBytes = 2048;
+constexpr size_t kSmallMaxPartials = 2048;
+constexpr size_t kSmallWsBytes = kSmallTicketBytes + kSmallMaxPartials * sizeof(Acc);
 
 // Event pair around one launch of an instrumented kernel (no-op unless timing is on).
 struct ScopedTimer {
@@ -231,6 +236,11 @@ extern "C" kb_status kb_ctx_create(int device, kb_ctx** out) {
     fail(ctx, KB_ERR_WORKSPACE, "cannot allocate the device status word");
     return bail(KB_ERR_WORKSPACE);
   }
+  if (cudaMalloc(&ctx->small_ws, kSmallWsBytes) != cudaSuccess ||
+      cudaMemset(ctx->small_ws, 0, kSmallWsBytes) != cudaSuccess) {
+    fail(ctx, KB_ERR_WORKSPACE, "cannot allocate the small-problem workspace");
+    return bail(KB_ERR_WORKSPACE);
+  }
   if ((st = set_stream_attr<KB_F32>(ctx)) != KB_OK) return bail(st);
   if ((st = set_stream_attr<KB_F16>(ctx)) != KB_OK) return bail(st);
   if ((st = set_stream_attr<KB_BF16>(ctx)) != KB_OK) return bail(st);
@@ -256,6 +266,7 @@ extern "C" kb_status kb_ctx_destroy(kb_ctx* ctx) {
   if (ctx->d_status) cudaFree(ctx->d_status);
   if (ctx->st_ref) cudaFree(ctx->st_ref);
   if (ctx->srt) cudaFree(ctx->srt);
+  if (ctx->small_ws) cudaFree(ctx->small_ws);
   for (int i = 0; i < 2; ++i) {
     if (ctx->st_batch[i]) cudaFree(ctx->st_batch[i]);
     if (ctx->ev_copied[i]) cudaEventDestroy(ctx->ev_copied[i]);
@@ -290,6 +301,12 @@ extern "C" kb_status kb_ctx_poll(kb_ctx* ctx, void* stream, kb_status* device_st
 extern "C" kb_status kb_ctx_set_grid(kb_ctx* ctx, uint32_t blocks) {
   if (!ctx) return KB_ERR_INVALID_ARG;
   ctx->forced_grid = blocks;
+  return KB_OK;
+}
+
+extern "C" kb_status kb_ctx_set_small_path(kb_ctx* ctx, int on) {
+  if (!ctx) return KB_ERR_INVALID_ARG;
+  ctx->small_on = on != 0;
   return KB_OK;
 }
 
@@ -493,6 +510,32 @@ template <int DT>
 kb_status screen_impl(kb_ctx* ctx, const void* d_ref, const void* const* h_cands, uint32_t K,
                       uint64_t N, float atol, float rtol, const kb_mask* mask,
                       kb_screen_result* d_out, cudaStream_t st) {
+  // Latency-bound sizes: everything in one launch (pointers as kernel arguments).
+  const uint64_t nb_small = (N + kSmallPerBlock - 1) / kSmallPerBlock;
+  if (ctx->small_ws && ctx->small_on && K <= (uint32_t)kPtrsPerLaunch && (uint64_t)K * N <= (1ull << 22) &&
+      (uint64_t)K * nb_small <= kSmallMaxPartials) {
+    SmallParams sm;
+    sm.ref = d_ref;
+    sm.tickets = reinterpret_cast<unsigned int*>(ctx->small_ws);
+    sm.partials = reinterpret_cast<Acc*>(ctx->small_ws + kSmallTicketBytes);
+    sm.out = d_out;
+    sm.N = N;
+    sm.nb = (unsigned int)nb_small;
+    sm.atol = atol;
+    sm.rtol = rtol;
+    sm.mask.kind = mask ? mask->kind : 0;
+    sm.mask.log2_tile = mask ? mask->log2_tile : 0;
+    sm.mask.stride = mask ? mask->stride : 1;
+    sm.mask.phase = mask ? mask->phase : 0;
+    sm.mask.bits = mask ? mask->d_bits : nullptr;
+    PtrChunk ch;
+    memcpy(ch.p, h_cands, K * sizeof(void*));
+    dim3 grid((unsigned int)nb_small, K);
+    screen_small_kernel<DT><<<grid, 256, 0, st>>>(sm, ch);
+    ++ctx->launches;
+    KB_CUDA(ctx, cudaGetLastError());
+    return KB_OK;
+  }
   kb_status rc = ensure_ws(ctx, K);
   if (rc != KB_OK) return rc;
   Acc* acc = reinterpret_cast<Acc*>(ctx->ws);

@@ -57,6 +57,12 @@ __device__ __forceinline__ bool mask_selected(const MaskDev& m, unsigned long lo
 }
 
 
+// K pointers travel to the device table through kernel arguments (no staging
+// buffer whose reuse would have to be fenced).
+constexpr int kPtrsPerLaunch = 480;
+struct PtrChunk {
+  const void* p[kPtrsPerLaunch];
+};
 // accumulator -> public record
 __device__ __forceinline__ void unpack_record(const Acc& a, kb_screen_result* dst) {
   kb_screen_result r;
@@ -670,6 +676,113 @@ __global__ void __launch_bounds__(256) screen_scout_kernel(const void* __restric
   }
 }
 
+// ---------------------------------------------------------------------------
+// Small problems (the latency-bound regime: a few candidates of at most a few hundred
+// thousand elements, e.g. 21 candidates of a 2048-element mat-vec output): ONE launch.
+// Candidate pointers travel as kernel arguments; block (bx, k) classifies 4096 elements
+// exactly and writes a partial record; the last block of candidate k to finish (a
+// self-resetting ticket per candidate) merges the partials and writes the result.
+// Nothing has to be zeroed beforehand and no atomics touch the accumulators.
+// ---------------------------------------------------------------------------
+constexpr unsigned int kSmallPerBlock = 4096;
+struct SmallParams {
+  const void* ref;
+  Acc* partials;            // [K][nb]
+  unsigned int* tickets;    // [K], zero between launches
+  kb_screen_result* out;    // [K]
+  unsigned long long N;
+  unsigned int nb;
+  float atol, rtol;
+  MaskDev mask;
+};
+
+template <int DT>
+__global__ void __launch_bounds__(256) screen_small_kernel(const SmallParams p, const PtrChunk cands) {
+  using E = Elem<DT>;
+  __shared__ unsigned int s_cnt[3];
+  __shared__ unsigned int s_rel;
+  __shared__ unsigned long long s_key;
+  __shared__ unsigned int s_ticket;
+  if (threadIdx.x == 0) {
+    s_cnt[0] = s_cnt[1] = s_cnt[2] = 0u;
+    s_rel = 0u;
+    s_key = 0ull;
+  }
+  __syncthreads();
+  const unsigned int k = blockIdx.y;
+  const void* cand = cands.p[k];
+  const unsigned long long base = (unsigned long long)blockIdx.x * kSmallPerBlock;
+  ExactAcc x;
+#pragma unroll 4
+  for (unsigned int j = 0; j < kSmallPerBlock / 256; ++j) {
+    const unsigned long long i = base + j * 256 + threadIdx.x;
+    if (i < p.N && mask_selected(p.mask, i)) x.add(E::load(p.ref, i), E::load(cand, i), i, p.atol, p.rtol);
+  }
+  x.n_mis = warp_add_u32(x.n_mis);
+  x.n_nan = warp_add_u32(x.n_nan);
+  x.n_inf = warp_add_u32(x.n_inf);
+  x.best = warp_max_u64(x.best);
+  x.qb = warp_max_u32(x.qb);
+  if ((threadIdx.x & 31) == 0) {
+    if (x.n_mis) atomicAdd(&s_cnt[0], x.n_mis);
+    if (x.n_nan) atomicAdd(&s_cnt[1], x.n_nan);
+    if (x.n_inf) atomicAdd(&s_cnt[2], x.n_inf);
+    if (x.best) atomicMax(&s_key, x.best);
+    if (x.qb) atomicMax(&s_rel, x.qb);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    Acc a;
+    a.mism = s_cnt[0];
+    a.nan = s_cnt[1];
+    a.inf = s_cnt[2];
+    a.key = s_key;
+    a.rel = s_rel;
+    a.pad = 0u;
+    p.partials[(size_t)k * p.nb + blockIdx.x] = a;
+    __threadfence();
+    s_ticket = atomicAdd(&p.tickets[k], 1u);
+  }
+  __syncthreads();
+  if (s_ticket != p.nb - 1) return;
+  // last block of this candidate: merge the partial records (warp 0 is enough)
+  __threadfence();
+  if (threadIdx.x < 32) {
+    unsigned long long mism = 0ull, nan = 0ull, inf = 0ull, key = 0ull;
+    unsigned int rel = 0u;
+    for (unsigned int b = threadIdx.x; b < p.nb; b += 32) {
+      const Acc* q = &p.partials[(size_t)k * p.nb + b];
+      mism += __ldcg(&q->mism);
+      nan += __ldcg(&q->nan);
+      inf += __ldcg(&q->inf);
+      const unsigned long long kv = __ldcg(&q->key);
+      key = kv > key ? kv : key;
+      const unsigned int rv = __ldcg(&q->rel);
+      rel = rv > rel ? rv : rel;
+    }
+    // each partial count is < 2^32 and nb <= 1024, so 32-bit halves add without loss below
+    const unsigned long long tm = (unsigned long long)warp_add_u32((unsigned int)mism) +
+                                  ((unsigned long long)warp_add_u32((unsigned int)(mism >> 32)) << 32);
+    const unsigned long long tn = (unsigned long long)warp_add_u32((unsigned int)nan) +
+                                  ((unsigned long long)warp_add_u32((unsigned int)(nan >> 32)) << 32);
+    const unsigned long long ti = (unsigned long long)warp_add_u32((unsigned int)inf) +
+                                  ((unsigned long long)warp_add_u32((unsigned int)(inf >> 32)) << 32);
+    key = warp_max_u64(key);
+    rel = warp_max_u32(rel);
+    if (threadIdx.x == 0) {
+      Acc a;
+      a.mism = tm;
+      a.nan = tn;
+      a.inf = ti;
+      a.key = key;
+      a.rel = rel;
+      a.pad = 0u;
+      unpack_record(a, &p.out[k]);
+      p.tickets[k] = 0u;   // ready for the next launch
+    }
+  }
+}
+
 __global__ void screen_finalize_kernel(const Acc* __restrict__ acc, kb_screen_result* __restrict__ out,
                                        unsigned int K) {
   const unsigned int k = blockIdx.x * blockDim.x + threadIdx.x;
@@ -677,12 +790,6 @@ __global__ void screen_finalize_kernel(const Acc* __restrict__ acc, kb_screen_re
   unpack_record(acc[k], &out[k]);
 }
 
-// K pointers travel to the device table through kernel arguments (no staging
-// buffer whose reuse would have to be fenced).
-constexpr int kPtrsPerLaunch = 480;
-struct PtrChunk {
-  const void* p[kPtrsPerLaunch];
-};
 // Also zeroes the accumulators of the same candidates and the ticket counter.
 __global__ void screen_prep_kernel(const PtrChunk chunk, const void** table, Acc* acc,
                                    unsigned int* done, unsigned int offset, unsigned int count) {

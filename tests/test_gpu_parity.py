@@ -94,9 +94,16 @@ def run_screen(ctx, kb, ref, cands, atol, rtol, mask_spec=None, N=None):
             mask = ctx.mask_strided(N, mask_spec[1], mask_spec[2], mask_spec[3])
         else:
             mask = ctx.mask_bitmap(N, mask_spec[1], mask_spec[2])
-    out = ctx.screen(ref, cands, atol, rtol, mask)
-    rec = kb.records(out)
+    # both dispatch paths: the general (streaming) one and, where the size allows it, the
+    # single-launch kernel for small problems; they must agree byte for byte
+    try:
+        ctx.set_small_path(False)
+        rec = kb.records(ctx.screen(ref, cands, atol, rtol, mask))
+    finally:
+        ctx.set_small_path(True)
+    rec_small = kb.records(ctx.screen(ref, cands, atol, rtol, mask))
     assert ctx.poll() == 0
+    assert rec.tobytes() == rec_small.tobytes()
     if mask is not None:
         mask.close()
     return rec
