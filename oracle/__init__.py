@@ -75,6 +75,14 @@ def lib() -> ctypes.CDLL:
         L.kbo_wins_rows.restype = i32
         L.kbo_select.argtypes = [vp, vp, u32, i32, u32, vp, vp]
         L.kbo_select.restype = i32
+        L.kbo_score.argtypes = [f32, u32, u32, f32, f32]
+        L.kbo_score.restype = f32
+        L.kbo_select_by_score.argtypes = [vp, vp, u32, u32, u32, f32, f32, u32, vp, vp, vp]
+        L.kbo_select_by_score.restype = i32
+        L.kbo_tail_ratios.argtypes = [vp, u32, vp]
+        L.kbo_tail_ratios.restype = i32
+        L.kbo_copeland.argtypes = [vp, u32, u32, vp, vp]
+        L.kbo_copeland.restype = i32
         L.kbo_decode_f16.argtypes = [ctypes.c_uint16]
         L.kbo_decode_f16.restype = f32
         L.kbo_decode_bf16.argtypes = [ctypes.c_uint16]
@@ -225,3 +233,54 @@ def decode_f16(h: int) -> float:
 
 def decode_bf16(b: int) -> float:
     return float(lib().kbo_decode_bf16(int(b)))
+
+
+def score(median_ms: float, rung: int, rung_budget: int, alpha: float, beta: float) -> np.float32:
+    """Runtime score S(p, r) of Eq. 2 for one adjudicated latency in milliseconds."""
+    return np.float32(lib().kbo_score(float(np.float32(median_ms)), int(rung), int(rung_budget),
+                                      float(np.float32(alpha)), float(np.float32(beta))))
+
+
+def select_by_score(screen_records: np.ndarray, median: np.ndarray, rung: int, rung_budget: int,
+                    alpha: float, beta: float, budget: int):
+    """(scores[K], survivors[budget], n): promotion by runtime score, ties to the lower index."""
+    rec = np.ascontiguousarray(screen_records, dtype=RESULT_DTYPE)
+    med = np.ascontiguousarray(median, dtype=np.float32)
+    K = rec.size
+    sc = np.zeros(K, dtype=np.float32)
+    surv = np.zeros(budget, dtype=np.int32)
+    n = np.zeros(1, dtype=np.uint32)
+    rc = lib().kbo_select_by_score(rec.ctypes.data, med.ctypes.data, K, int(rung), int(rung_budget),
+                                   float(np.float32(alpha)), float(np.float32(beta)), int(budget),
+                                   sc.ctypes.data, surv.ctypes.data, n.ctypes.data)
+    if rc != 0:
+        raise ValueError(f"kbo_select_by_score rejected its arguments (rc={rc})")
+    return sc, surv, int(n[0])
+
+
+def tail_ratios(timings: np.ndarray) -> np.ndarray:
+    """[K][3] = p90/p50, p95/p50, p99/p50 of each row."""
+    t = np.ascontiguousarray(timings, dtype=np.float32)
+    if t.ndim == 1:
+        t = t[None, :]
+    K, S = t.shape
+    out = np.zeros((K, 3), dtype=np.float32)
+    for k in range(K):
+        rc = lib().kbo_tail_ratios(t[k].ctypes.data, S, out[k].ctypes.data)
+        if rc == -2:
+            raise NonFiniteTiming("non-finite timing")
+        if rc != 0:
+            raise ValueError(f"kbo_tail_ratios rejected its arguments (rc={rc})")
+    return out
+
+
+def copeland(wins: np.ndarray, S: int):
+    """(beats[K], ties[K]) from a win matrix."""
+    w = np.ascontiguousarray(wins, dtype=np.uint32)
+    K = w.shape[0]
+    beats = np.zeros(K, dtype=np.uint32)
+    ties = np.zeros(K, dtype=np.uint32)
+    rc = lib().kbo_copeland(w.ctypes.data, K, int(S), beats.ctypes.data, ties.ctypes.data)
+    if rc != 0:
+        raise ValueError(f"kbo_copeland rejected its arguments (rc={rc})")
+    return beats, ties

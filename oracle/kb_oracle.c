@@ -339,3 +339,130 @@ int kbo_select(const kbo_screen_result* screen, const float* median, uint32_t K,
   free(taken);
   return 0;
 }
+
+/* ------------------------------------------------------------------------
+ * Scheduler-side statistics on top of the three calls above.
+ * ------------------------------------------------------------------------ */
+
+/*
+ * Runtime score of one candidate (Sec. 3.1, Eq. 2):
+ *   S(p, r) = 1e6 / max(1, latency_us) + gamma(r),  gamma(r) = alpha*r + beta*b_r
+ * with the latency taken as the adjudicated (median) latency, given in
+ * milliseconds.  Every operation is a binary32 operation in the order written:
+ *   l_us = median_ms * 1000;  m = max(1, l_us);  base = 1e6 / m;
+ *   gamma = (alpha * r) + (beta * b_r);  score = base + gamma.
+ */
+float kbo_score(float median_ms, uint32_t rung, uint32_t rung_budget, float alpha, float beta) {
+  float l_us = median_ms * 1000.0f;
+  float m = (l_us > 1.0f) ? l_us : 1.0f;
+  float base = 1.0e6f / m;
+  float ga = alpha * (float)rung;
+  float gb = beta * (float)rung_budget;
+  float gamma = ga + gb;
+  return base + gamma;
+}
+
+/*
+ * Promotion by runtime score (Sec. 3.4: "ranks candidates by s(c,r) with
+ * deterministic tie-breaking ... promotes the top fraction"): eligible =
+ * pass == 1, order by (score descending, index ascending).  scores[K] (may be
+ * NULL) receives every candidate's score, eligible or not.
+ */
+int kbo_select_by_score(const kbo_screen_result* screen, const float* median, uint32_t K,
+                        uint32_t rung, uint32_t rung_budget, float alpha, float beta,
+                        uint32_t budget, float* scores, int32_t* survivors, uint32_t* n_out) {
+  uint8_t* taken;
+  float* sc;
+  uint32_t n = 0, k, slot;
+  if (!screen || !median || !survivors || !n_out || K == 0 || budget == 0) return -1;
+  taken = (uint8_t*)calloc(K, 1);
+  sc = (float*)malloc((size_t)K * sizeof(float));
+  if (!taken || !sc) return -1;
+  for (k = 0; k < K; ++k) {
+    sc[k] = kbo_score(median[k], rung, rung_budget, alpha, beta);
+    if (scores) scores[k] = sc[k];
+  }
+  for (slot = 0; slot < budget; ++slot) {
+    int64_t best = -1;
+    for (k = 0; k < K; ++k) {
+      if (taken[k] || screen[k].pass != 1u) continue;
+      if (best < 0 || sc[k] > sc[best]) best = k;   /* equal scores: the lower index stays */
+    }
+    if (best < 0) break;
+    taken[best] = 1;
+    survivors[n++] = (int32_t)best;
+  }
+  for (slot = n; slot < budget; ++slot) survivors[slot] = -1;
+  *n_out = n;
+  free(taken);
+  free(sc);
+  return 0;
+}
+
+/*
+ * Tail ratios of one row (Appendix, Relative Variability Metrics: p90/p50,
+ * p95/p50, p99/p50).  Percentile q in {50, 90, 95, 99} of the sorted row by
+ * the linear (type-7) rule with integer position arithmetic:
+ *   pos = q*(S-1); lo = pos/100; rem = pos%100; hi = min(lo+1, S-1)
+ *   P_q = x_lo                                          if rem == 0
+ *       = x_lo + (((float)rem / 100.0f) * (x_hi - x_lo))   otherwise,
+ * each operation rounded; out3 = {P90/P50, P95/P50, P99/P50} (rounded
+ * divisions).  Returns 0; -1 bad argument; -2 non-finite timing.
+ */
+int kbo_tail_ratios(const float* row, uint32_t S, float* out3) {
+  static const uint32_t qs[4] = {50u, 90u, 95u, 99u};
+  float p[4];
+  float* x;
+  uint32_t i, t;
+  if (!row || !out3 || S == 0) return -1;
+  for (i = 0; i < S; ++i)
+    if (!is_finite32(row[i])) return -2;
+  x = (float*)malloc((size_t)S * sizeof(float));
+  if (!x) return -1;
+  memcpy(x, row, (size_t)S * sizeof(float));
+  qsort(x, S, sizeof(float), cmp_float_asc);
+  for (t = 0; t < 4; ++t) {
+    uint64_t pos = (uint64_t)qs[t] * (uint64_t)(S - 1);
+    uint64_t lo = pos / 100u;
+    uint32_t rem = (uint32_t)(pos % 100u);
+    uint64_t hi = (lo + 1 < (uint64_t)S) ? lo + 1 : (uint64_t)S - 1;
+    if (rem == 0) {
+      p[t] = x[lo];
+    } else {
+      float w = (float)rem / 100.0f;
+      float diff = x[hi] - x[lo];
+      float step = w * diff;
+      p[t] = x[lo] + step;
+    }
+  }
+  out3[0] = p[1] / p[0];
+  out3[1] = p[2] / p[0];
+  out3[2] = p[3] / p[0];
+  free(x);
+  return 0;
+}
+
+/*
+ * Copeland counts from the win matrix: candidate a "beats" b when it wins more
+ * than half of the doubled sample pairs, W[a][b] > S*S, and ties with b when
+ * W[a][b] == S*S.  beats[a], ties[a] (may be NULL) count opponents b != a.
+ * A ranking by beats is stable under timing noise in the sense of the
+ * appendix: it only uses the order of samples.
+ */
+int kbo_copeland(const uint32_t* wins, uint32_t K, uint32_t S, uint32_t* beats, uint32_t* ties) {
+  uint32_t a, b;
+  uint64_t half = (uint64_t)S * S;
+  if (!wins || !beats || K == 0 || S == 0) return -1;
+  for (a = 0; a < K; ++a) {
+    uint32_t nb = 0, nt = 0;
+    for (b = 0; b < K; ++b) {
+      uint64_t w = wins[(size_t)a * K + b];
+      if (b == a) continue;
+      if (w > half) ++nb;
+      if (w == half) ++nt;
+    }
+    beats[a] = nb;
+    if (ties) ties[a] = nt;
+  }
+  return 0;
+}
