@@ -256,6 +256,40 @@ kb_status kb_select(kb_ctx* ctx, const kb_screen_result* d_screen, const float* 
                     uint32_t K, kb_select_policy policy, uint32_t budget, int32_t* d_survivors,
                     uint32_t* d_n_survivors, void* stream);
 
+/* ---- scheduler-side statistics ------------------------------------------- */
+
+/* Runtime score and promotion by it (Sec. 3.1, Eq. 2; Sec. 3.4 scheduler):
+ *     S(p, r) = 1e6 / max(1, latency_us) + gamma(r),   gamma(r) = alpha*r + beta*b_r
+ * with latency = the adjudicated (median) latency, given in milliseconds; every
+ * operation in binary32 in this order: l = median*1000; m = max(1, l);
+ * base = 1e6/m; gamma = (alpha*rung) + (beta*rung_budget); score = base + gamma.
+ * Eligible = pass == 1; order by (score descending, index ascending); the first
+ * n = min(budget, #eligible) indices go to d_survivors in rank order, the rest
+ * is -1, n to *d_n_survivors.
+ *   d_score  DEVICE [K] float, every candidate's score (eligible or not); may be NULL.
+ * Other arguments as for kb_select. */
+kb_status kb_select_by_score(kb_ctx* ctx, const kb_screen_result* d_screen, const float* d_median,
+                             uint32_t K, uint32_t rung, uint32_t rung_budget, float alpha,
+                             float beta, uint32_t budget, float* d_score, int32_t* d_survivors,
+                             uint32_t* d_n_survivors, void* stream);
+
+/* Tail ratios per candidate (Appendix "Relative Variability Metrics"):
+ * d_ratios DEVICE [K][3] = {P90/P50, P95/P50, P99/P50} of each row of
+ * d_timings [K][S], with P_q the linear (type-7) percentile of the sorted row:
+ *   pos = q*(S-1); lo = pos/100; rem = pos%100; hi = min(lo+1, S-1);
+ *   P_q = x_lo if rem == 0 else x_lo + (((float)rem / 100.0f) * (x_hi - x_lo)),
+ * each operation (and the final divisions) rounded.  Non-finite timings set
+ * KB_ERR_NONFINITE in the device status.  1 <= S <= KB_MAX_S. */
+kb_status kb_tail_ratios(kb_ctx* ctx, const float* d_timings, uint32_t K, uint32_t S,
+                         float* d_ratios, void* stream);
+
+/* Copeland counts from a win matrix of kb_adjudicate (a ranking that uses only
+ * the order of samples, Appendix "Relative Variability Metrics"):
+ *   d_beats[a] = #{b != a : W[a][b] >  S*S},  d_ties[a] = #{b != a : W[a][b] == S*S}
+ * DEVICE [K] uint32 each; d_ties may be NULL. */
+kb_status kb_copeland(kb_ctx* ctx, const uint32_t* d_wins, uint32_t K, uint32_t S,
+                      uint32_t* d_beats, uint32_t* d_ties, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

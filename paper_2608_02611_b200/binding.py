@@ -38,6 +38,7 @@ EXPORTS = [
     "kb_ctx_enable_timing", "kb_ctx_read_timer", "kb_ctx_launch_count", "kb_ctx_set_wins_algo", "kb_ctx_set_small_path",
     "kb_mask_create_strided", "kb_mask_create_bitmap", "kb_mask_count", "kb_mask_destroy",
     "kb_screen", "kb_screen_host", "kb_screen_static", "kb_adjudicate", "kb_select",
+    "kb_select_by_score", "kb_tail_ratios", "kb_copeland",
 ]
 
 
@@ -83,6 +84,9 @@ def load() -> ctypes.CDLL:
     L.kb_screen_static.argtypes = [vp, vp, u32, u64, i32, f32, f32, vp, vp]
     L.kb_adjudicate.argtypes = [vp, vp, u32, u32, vp, vp, vp, vp]
     L.kb_select.argtypes = [vp, vp, vp, u32, i32, u32, vp, vp, vp]
+    L.kb_select_by_score.argtypes = [vp, vp, vp, u32, u32, u32, f32, f32, u32, vp, vp, vp, vp]
+    L.kb_tail_ratios.argtypes = [vp, vp, u32, u32, vp, vp]
+    L.kb_copeland.argtypes = [vp, vp, u32, u32, vp, vp, vp]
     for name in EXPORTS:
         if name != "kb_last_error":
             getattr(L, name).restype = i32
@@ -289,6 +293,50 @@ def screen_static(ref: torch.Tensor, cands: Sequence[torch.Tensor], atol: float,
     if rc != KB_OK:
         raise KbError(rc, "kb_screen_static", (load().kb_last_error(None) or b"").decode())
     return out
+
+
+def _ctx_method(fn):
+    setattr(Context, fn.__name__, fn)
+    return fn
+
+
+@_ctx_method
+def select_by_score(self, screen_out: torch.Tensor, median: torch.Tensor, rung: int, rung_budget: int,
+                    alpha: float, beta: float, budget: int):
+    """kb_select_by_score -> (score float32 [K], survivors int32 [budget], n int32 [1])."""
+    K = median.numel()
+    score = torch.empty(K, dtype=torch.float32, device=median.device)
+    surv = torch.empty(budget, dtype=torch.int32, device=median.device)
+    n = torch.empty(1, dtype=torch.int32, device=median.device)
+    rc = load().kb_select_by_score(self._h, screen_out.data_ptr(), median.data_ptr(), K, int(rung),
+                                   int(rung_budget), float(alpha), float(beta), int(budget),
+                                   score.data_ptr(), surv.data_ptr(), n.data_ptr(),
+                                   _stream_ptr(median.device))
+    self._check(rc, "kb_select_by_score")
+    return score, surv, n
+
+
+@_ctx_method
+def tail_ratios(self, timings: torch.Tensor) -> torch.Tensor:
+    """kb_tail_ratios -> float32 [K, 3] = p90/p50, p95/p50, p99/p50."""
+    K, S = timings.shape
+    out = torch.empty((K, 3), dtype=torch.float32, device=timings.device)
+    rc = load().kb_tail_ratios(self._h, timings.data_ptr(), K, S, out.data_ptr(),
+                               _stream_ptr(timings.device))
+    self._check(rc, "kb_tail_ratios")
+    return out
+
+
+@_ctx_method
+def copeland(self, wins: torch.Tensor, S: int):
+    """kb_copeland -> (beats int32 [K], ties int32 [K])."""
+    K = wins.shape[0]
+    beats = torch.empty(K, dtype=torch.int32, device=wins.device)
+    ties = torch.empty(K, dtype=torch.int32, device=wins.device)
+    rc = load().kb_copeland(self._h, wins.data_ptr(), K, int(S), beats.data_ptr(), ties.data_ptr(),
+                            _stream_ptr(wins.device))
+    self._check(rc, "kb_copeland")
+    return beats, ties
 
 
 def records(screen_out: torch.Tensor) -> np.ndarray:

@@ -30,15 +30,10 @@ namespace kb {
 
 constexpr int kRowsThreads = 256;
 
-__global__ void __launch_bounds__(kRowsThreads) rows_kernel(const float* __restrict__ timings,
-                                                            unsigned int S, unsigned int P /*pow2 >= S*/,
-                                                            float* __restrict__ median,
-                                                            float* __restrict__ iqr,
-                                                            float* __restrict__ sorted_out /*[K][S] or NULL*/,
-                                                            unsigned int* status) {
-  extern __shared__ float xs[];
-  const unsigned int k = blockIdx.x;
-  const float* row = timings + (size_t)k * S;
+// Load one row into shared memory (padded with +Inf to P, a power of two), flag
+// non-finite timings, sort ascending (bitonic network).
+__device__ __forceinline__ void load_and_sort_row(const float* __restrict__ row, unsigned int S,
+                                                  unsigned int P, float* xs, unsigned int* status) {
   const float inf = __uint_as_float(0x7F800000u);
   bool nonfinite = false;
   for (unsigned int i = threadIdx.x; i < P; i += kRowsThreads) {
@@ -66,6 +61,17 @@ __global__ void __launch_bounds__(kRowsThreads) rows_kernel(const float* __restr
       __syncthreads();
     }
   }
+}
+
+__global__ void __launch_bounds__(kRowsThreads) rows_kernel(const float* __restrict__ timings,
+                                                            unsigned int S, unsigned int P /*pow2 >= S*/,
+                                                            float* __restrict__ median,
+                                                            float* __restrict__ iqr,
+                                                            float* __restrict__ sorted_out /*[K][S] or NULL*/,
+                                                            unsigned int* status) {
+  extern __shared__ float xs[];
+  const unsigned int k = blockIdx.x;
+  load_and_sort_row(timings + (size_t)k * S, S, P, xs, status);
   if (sorted_out) {
     for (unsigned int i = threadIdx.x; i < S; i += kRowsThreads) sorted_out[(size_t)k * S + i] = xs[i];
   }
@@ -86,6 +92,37 @@ __global__ void __launch_bounds__(kRowsThreads) rows_kernel(const float* __restr
     }
     if (median) median[k] = q[2];
     if (iqr) iqr[k] = __fsub_rn(q[3], q[1]);
+  }
+}
+
+// Tail ratios P90/P50, P95/P50, P99/P50 of every row (Appendix "Relative Variability
+// Metrics"): the same sort, percentiles by the linear rule with q*(S-1)/100 positions.
+__global__ void __launch_bounds__(kRowsThreads) tails_kernel(const float* __restrict__ timings,
+                                                             unsigned int S, unsigned int P,
+                                                             float* __restrict__ ratios /*[K][3]*/,
+                                                             unsigned int* status) {
+  extern __shared__ float xs[];
+  const unsigned int k = blockIdx.x;
+  load_and_sort_row(timings + (size_t)k * S, S, P, xs, status);
+  if (threadIdx.x == 0) {
+    const unsigned int qs[4] = {50u, 90u, 95u, 99u};
+    float pq[4];
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      const unsigned long long pos = (unsigned long long)qs[t] * (S - 1);
+      const unsigned int lo = (unsigned int)(pos / 100ull);
+      const unsigned int rem = (unsigned int)(pos % 100ull);
+      const unsigned int hi = (lo + 1 < S) ? lo + 1 : S - 1;
+      if (rem == 0) {
+        pq[t] = xs[lo];
+      } else {
+        const float w = __fdiv_rn((float)rem, 100.0f);
+        pq[t] = __fadd_rn(xs[lo], __fmul_rn(w, __fsub_rn(xs[hi], xs[lo])));
+      }
+    }
+    ratios[(size_t)k * 3 + 0] = __fdiv_rn(pq[1], pq[0]);
+    ratios[(size_t)k * 3 + 1] = __fdiv_rn(pq[2], pq[0]);
+    ratios[(size_t)k * 3 + 2] = __fdiv_rn(pq[3], pq[0]);
   }
 }
 

@@ -249,6 +249,11 @@ extern "C" kb_status kb_ctx_create(int device, kb_ctx** out) {
     fail(ctx, KB_ERR_CUDA, "cannot raise the shared-memory limit of the row kernel");
     return bail(KB_ERR_CUDA);
   }
+  if (cudaFuncSetAttribute(tails_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)(KB_MAX_S * sizeof(float))) != cudaSuccess) {
+    fail(ctx, KB_ERR_CUDA, "cannot raise the shared-memory limit of the tail-ratio kernel");
+    return bail(KB_ERR_CUDA);
+  }
   if (cudaFuncSetAttribute(wins_rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            kWinsRowsPerBlock * 4096 * (int)sizeof(float)) != cudaSuccess) {
     fail(ctx, KB_ERR_CUDA, "cannot raise the shared-memory limit of the win-count kernel");
@@ -903,6 +908,65 @@ extern "C" kb_status kb_select(kb_ctx* ctx, const kb_screen_result* d_screen, co
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   select_kernel<<<(K + kSelectThreads - 1) / kSelectThreads, kSelectThreads, 0, st>>>(
       d_screen, d_median, K, (int)policy, budget, d_survivors, d_n_survivors);
+  ++ctx->launches;
+  KB_CUDA(ctx, cudaGetLastError());
+  return KB_OK;
+}
+
+// ---------------------------------------------------------------------------
+// scheduler-side statistics
+// ---------------------------------------------------------------------------
+
+extern "C" kb_status kb_select_by_score(kb_ctx* ctx, const kb_screen_result* d_screen,
+                                        const float* d_median, uint32_t K, uint32_t rung,
+                                        uint32_t rung_budget, float alpha, float beta,
+                                        uint32_t budget, float* d_score, int32_t* d_survivors,
+                                        uint32_t* d_n_survivors, void* stream) {
+  if (!ctx) return KB_ERR_INVALID_ARG;
+  if (!d_screen || !d_median || !d_survivors || !d_n_survivors)
+    return fail(ctx, KB_ERR_INVALID_ARG, "kb_select_by_score: null pointer");
+  if (K == 0 || K > KB_MAX_K) return fail(ctx, KB_ERR_INVALID_ARG, "kb_select_by_score: K=%u outside [1, %u]", K, KB_MAX_K);
+  if (budget == 0) return fail(ctx, KB_ERR_INVALID_ARG, "kb_select_by_score: budget must be >= 1");
+  if (!std::isfinite(alpha) || !std::isfinite(beta))
+    return fail(ctx, KB_ERR_INVALID_ARG, "kb_select_by_score: alpha and beta must be finite");
+  DeviceGuard g(ctx->device);
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  // gamma(r) = (alpha*r) + (beta*b_r), each operation in binary32 (host floats are IEEE binary32)
+  volatile float ga = alpha * (float)rung;
+  volatile float gb = beta * (float)rung_budget;
+  const float gamma = ga + gb;
+  select_by_score_kernel<<<(K + kSelectThreads - 1) / kSelectThreads, kSelectThreads, 0, st>>>(
+      d_screen, d_median, K, gamma, budget, d_score, d_survivors, d_n_survivors);
+  ++ctx->launches;
+  KB_CUDA(ctx, cudaGetLastError());
+  return KB_OK;
+}
+
+extern "C" kb_status kb_tail_ratios(kb_ctx* ctx, const float* d_timings, uint32_t K, uint32_t S,
+                                    float* d_ratios, void* stream) {
+  if (!ctx) return KB_ERR_INVALID_ARG;
+  if (!d_timings || !d_ratios) return fail(ctx, KB_ERR_INVALID_ARG, "kb_tail_ratios: null pointer");
+  if (K == 0 || K > KB_MAX_K) return fail(ctx, KB_ERR_INVALID_ARG, "kb_tail_ratios: K=%u outside [1, %u]", K, KB_MAX_K);
+  if (S == 0 || S > KB_MAX_S) return fail(ctx, KB_ERR_INVALID_ARG, "kb_tail_ratios: S=%u outside [1, %u]", S, KB_MAX_S);
+  DeviceGuard g(ctx->device);
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  unsigned int P = 1;
+  while (P < S) P <<= 1;
+  tails_kernel<<<K, kRowsThreads, (size_t)P * sizeof(float), st>>>(d_timings, S, P, d_ratios, ctx->d_status);
+  ++ctx->launches;
+  KB_CUDA(ctx, cudaGetLastError());
+  return KB_OK;
+}
+
+extern "C" kb_status kb_copeland(kb_ctx* ctx, const uint32_t* d_wins, uint32_t K, uint32_t S,
+                                 uint32_t* d_beats, uint32_t* d_ties, void* stream) {
+  if (!ctx) return KB_ERR_INVALID_ARG;
+  if (!d_wins || !d_beats) return fail(ctx, KB_ERR_INVALID_ARG, "kb_copeland: null pointer");
+  if (K == 0 || K > KB_MAX_K) return fail(ctx, KB_ERR_INVALID_ARG, "kb_copeland: K=%u outside [1, %u]", K, KB_MAX_K);
+  if (S == 0 || S > KB_MAX_S) return fail(ctx, KB_ERR_INVALID_ARG, "kb_copeland: S=%u outside [1, %u]", S, KB_MAX_S);
+  DeviceGuard g(ctx->device);
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  copeland_kernel<<<(K + 7) / 8, 256, 0, st>>>(d_wins, K, S, d_beats, d_ties);
   ++ctx->launches;
   KB_CUDA(ctx, cudaGetLastError());
   return KB_OK;

@@ -65,4 +65,82 @@ __global__ void __launch_bounds__(kSelectThreads) select_kernel(
   if (gtid == 0) *n_out = n;
 }
 
+// ---------------------------------------------------------------------------
+// Runtime score (Sec. 3.1, Eq. 2) and promotion by it: (score descending, index ascending).
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ float runtime_score(float median_ms, float gamma) {
+  const float l_us = __fmul_rn(median_ms, 1000.0f);
+  const float m = l_us > 1.0f ? l_us : 1.0f;
+  return __fadd_rn(__fdiv_rn(1.0e6f, m), gamma);
+}
+
+__global__ void __launch_bounds__(kSelectThreads) select_by_score_kernel(
+    const kb_screen_result* __restrict__ screen, const float* __restrict__ median, unsigned int K,
+    float gamma, unsigned int budget, float* __restrict__ score_out, int* __restrict__ survivors,
+    unsigned int* __restrict__ n_out) {
+  __shared__ unsigned int skey[kSelectThreads];
+  __shared__ unsigned char selig[kSelectThreads];
+  const unsigned int k = blockIdx.x * kSelectThreads + threadIdx.x;
+  bool mine_ok = false;
+  unsigned int mine = 0u;   // descending score = ascending complement of the ordered bits
+  if (k < K) {
+    const float sc = runtime_score(median[k], gamma);
+    if (score_out) score_out[k] = sc;
+    mine = ~ordered_bits(sc);
+    mine_ok = screen[k].pass == 1u;
+  }
+  unsigned int rank = 0, n_elig = 0;
+  for (unsigned int base = 0; base < K; base += kSelectThreads) {
+    const unsigned int m = base + threadIdx.x;
+    bool ok = false;
+    unsigned int key = 0u;
+    if (m < K) {
+      key = ~ordered_bits(runtime_score(median[m], gamma));
+      ok = screen[m].pass == 1u;
+    }
+    __syncthreads();
+    skey[threadIdx.x] = key;
+    selig[threadIdx.x] = ok ? 1 : 0;
+    __syncthreads();
+    const unsigned int lim = min((unsigned int)kSelectThreads, K - base);
+    for (unsigned int t = 0; t < lim; ++t) {
+      if (!selig[t]) continue;
+      ++n_elig;
+      const unsigned int other = skey[t];
+      const unsigned int mi = base + t;
+      rank += (other < mine || (other == mine && mi < k)) ? 1u : 0u;
+    }
+  }
+  const unsigned int n = n_elig < budget ? n_elig : budget;
+  if (k < K && mine_ok && rank < budget) survivors[rank] = (int)k;
+  const unsigned long long gtid = (unsigned long long)blockIdx.x * kSelectThreads + threadIdx.x;
+  const unsigned long long gsz = (unsigned long long)gridDim.x * kSelectThreads;
+  for (unsigned long long slot = n + gtid; slot < budget; slot += gsz) survivors[slot] = -1;
+  if (gtid == 0) *n_out = n;
+}
+
+// Copeland counts: one warp per row of the win matrix.
+__global__ void __launch_bounds__(256) copeland_kernel(const unsigned int* __restrict__ wins,
+                                                       unsigned int K, unsigned int S,
+                                                       unsigned int* __restrict__ beats,
+                                                       unsigned int* __restrict__ ties) {
+  const unsigned int a = blockIdx.x * 8 + (threadIdx.x >> 5);
+  const unsigned int lane = threadIdx.x & 31;
+  if (a >= K) return;
+  const unsigned int half = S * S;
+  unsigned int nb = 0, nt = 0;
+  for (unsigned int b = lane; b < K; b += 32) {
+    if (b == a) continue;
+    const unsigned int w = wins[(size_t)a * K + b];
+    nb += w > half ? 1u : 0u;
+    nt += w == half ? 1u : 0u;
+  }
+  nb = warp_add_u32(nb);
+  nt = warp_add_u32(nt);
+  if (lane == 0) {
+    beats[a] = nb;
+    if (ties) ties[a] = nt;
+  }
+}
+
 }  // namespace kb

@@ -455,3 +455,50 @@ def test_screen_host_matches_screen(ctx, kb):
     assert got.tobytes() == want.tobytes()
     oracle_rec = oracle_screen(case.dtype, ref, cands, case.atol, case.rtol)
     assert_records_equal(got, oracle_rec, "screen_host")
+
+
+# --------------------------------------------------------------------------
+# scheduler-side statistics: runtime score, tail ratios, Copeland counts
+# --------------------------------------------------------------------------
+
+@pytest.mark.parametrize("K,budget", [(1, 1), (9, 4), (64, 32), (300, 50), (1000, 1000)])
+def test_select_by_score_matches_oracle(ctx, kb, K, budget):
+    rng = np.random.default_rng(K + budget)
+    dev = torch.device("cuda", 0)
+    for rung, b_r in [(0, 4), (1, 16), (2, 60)]:
+        rec = np.zeros(K, dtype=oracle.RESULT_DTYPE)
+        rec["pass"] = rng.random(K) < 0.7
+        med = rng.lognormal(0, 1.0, K).astype(np.float32)
+        med[rng.random(K) < 0.2] = np.float32(0.0005)             # below 1 us: scores tie
+        med[rng.random(K) < 0.2] = np.float32(1.0)
+        d_rec = torch.from_numpy(rec.view(np.uint8).reshape(K, 48).copy()).to(dev)
+        score, surv, n = ctx.select_by_score(d_rec, torch.from_numpy(med).to(dev), rung, b_r, 0.02, 0.01, budget)
+        osc, osurv, on = oracle.select_by_score(rec, med, rung, b_r, 0.02, 0.01, budget)
+        assert (fbits(score.cpu().numpy()) == fbits(osc)).all()
+        assert int(n.item()) == on and surv.cpu().numpy().tolist() == osurv.tolist()
+
+
+@pytest.mark.parametrize("K,S", [(1, 1), (3, 2), (21, 4), (21, 16), (21, 60), (7, 101), (64, 100),
+                                 (5, 2000), (2, 5000)])
+def test_tail_ratios_match_oracle(ctx, kb, K, S):
+    rng = np.random.default_rng(K * 77 + S)
+    dev = torch.device("cuda", 0)
+    t = rng.lognormal(0, 0.1, (K, S)).astype(np.float32)
+    got = ctx.tail_ratios(torch.from_numpy(t).to(dev)).cpu().numpy()
+    assert ctx.poll() == 0
+    want = oracle.tail_ratios(t)
+    assert (fbits(got) == fbits(want)).all()
+
+
+@pytest.mark.parametrize("K,S", [(1, 3), (2, 3), (9, 16), (64, 100), (130, 20)])
+def test_copeland_matches_oracle(ctx, kb, K, S):
+    rng = np.random.default_rng(K + S)
+    dev = torch.device("cuda", 0)
+    t = np.round(rng.lognormal(0, 0.1, (K, S)), 2).astype(np.float32)
+    if K > 1:
+        t[K - 1] = t[0]
+    med, iqr, wins = ctx.adjudicate(torch.from_numpy(t).to(dev))
+    beats, ties = ctx.copeland(wins, S)
+    ob, ot = oracle.copeland(oracle.adjudicate(t)[2], S)
+    assert (beats.cpu().numpy().view(np.uint32) == ob).all()
+    assert (ties.cpu().numpy().view(np.uint32) == ot).all()
