@@ -83,6 +83,8 @@ def lib() -> ctypes.CDLL:
         L.kbo_tail_ratios.restype = i32
         L.kbo_copeland.argtypes = [vp, u32, u32, vp, vp]
         L.kbo_copeland.restype = i32
+        L.kbo_confirm.argtypes = [vp, vp, vp, u32, f32, vp, vp]
+        L.kbo_confirm.restype = i32
         L.kbo_decode_f16.argtypes = [ctypes.c_uint16]
         L.kbo_decode_f16.restype = f32
         L.kbo_decode_bf16.argtypes = [ctypes.c_uint16]
@@ -284,3 +286,18 @@ def copeland(wins: np.ndarray, S: int):
     if rc != 0:
         raise ValueError(f"kbo_copeland rejected its arguments (rc={rc})")
     return beats, ties
+
+
+def confirm(s1, s2, prev, threshold: float):
+    """(status uint32 [K], score float32 [K]) of the re-measure-and-confirm rule."""
+    a = np.ascontiguousarray(s1, dtype=np.float32)
+    b = np.ascontiguousarray(s2, dtype=np.float32)
+    c = np.ascontiguousarray(prev, dtype=np.float32)
+    K = a.size
+    st = np.zeros(K, dtype=np.uint32)
+    sc = np.zeros(K, dtype=np.float32)
+    rc = lib().kbo_confirm(a.ctypes.data, b.ctypes.data, c.ctypes.data, K, float(np.float32(threshold)),
+                           st.ctypes.data, sc.ctypes.data)
+    if rc != 0:
+        raise ValueError(f"kbo_confirm rejected its arguments (rc={rc})")
+    return st, sc

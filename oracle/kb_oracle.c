@@ -466,3 +466,40 @@ int kbo_copeland(const uint32_t* wins, uint32_t K, uint32_t S, uint32_t* beats, 
   }
   return 0;
 }
+
+/*
+ * Re-measure-and-confirm adjudication.  The paper's only description of
+ * "stability adjudication" is a commented-out passage of Sec. 3: when a
+ * candidate's score change exceeds a configurable threshold, it is measured
+ * again at the same fidelity and reverted if the improvement is not confirmed.
+ * Reading (binary32, operations as written), per candidate k with the
+ * incumbent's score prev, the first score s1 and the re-measured score s2:
+ *   flagged   = (s1 - prev) > (threshold * prev)
+ *   confirmed = (s2 - prev) > (threshold * prev)
+ *   status = 0, score = s1            if not flagged            (no re-measurement needed)
+ *   status = 1, score = min(s1, s2)   if flagged and confirmed  (the cautious of the two)
+ *   status = 2, score = prev          if flagged, not confirmed (reverted)
+ */
+int kbo_confirm(const float* s1, const float* s2, const float* prev, uint32_t K, float threshold,
+                uint32_t* status, float* score) {
+  uint32_t k;
+  if (!s1 || !s2 || !prev || !status || !score || K == 0) return -1;
+  for (k = 0; k < K; ++k) {
+    float bar = threshold * prev[k];
+    float d1 = s1[k] - prev[k];
+    float d2 = s2[k] - prev[k];
+    int flagged = d1 > bar;
+    int confirmed = d2 > bar;
+    if (!flagged) {
+      status[k] = 0u;
+      score[k] = s1[k];
+    } else if (confirmed) {
+      status[k] = 1u;
+      score[k] = (s2[k] < s1[k]) ? s2[k] : s1[k];
+    } else {
+      status[k] = 2u;
+      score[k] = prev[k];
+    }
+  }
+  return 0;
+}

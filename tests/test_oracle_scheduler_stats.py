@@ -164,3 +164,34 @@ def test_copeland_separated_candidates_rank_by_speed():
     t = np.float32([[3, 3.1, 3.2], [1, 1.1, 1.2], [2, 2.1, 2.2], [4, 4.1, 4.2]])
     beats, ties = oracle.copeland(oracle.adjudicate(t)[2], 3)
     assert beats.tolist() == [1, 3, 2, 0] and ties.tolist() == [0, 0, 0, 0]
+
+
+# ---- re-measure and confirm --------------------------------------------------------------
+
+def test_confirm_truth_table():
+    prev = np.float32([100, 100, 100, 100, 100])
+    s1 = np.float32([104, 120, 120, 90, 105.0001])
+    s2 = np.float32([50, 118, 103, 300, 200])
+    st, sc = oracle.confirm(s1, s2, prev, 0.05)
+    # +4%: below the threshold, taken as is.  +20% re-measured at +18%: confirmed, the lower
+    # of the two.  +20% re-measured at +3%: reverted to the incumbent.  A regression is never
+    # flagged.  Just above the bar and confirmed.
+    assert st.tolist() == [0, 1, 2, 0, 1]
+    assert sc.tolist() == [104.0, 118.0, 100.0, 90.0, np.float32(105.0001)]
+
+
+def test_confirm_boundary_is_strict_and_in_binary32():
+    from fractions import Fraction
+    rng = np.random.default_rng(5)
+    prev = rng.lognormal(5, 1, 500).astype(np.float32)
+    s1 = (prev * rng.choice(np.float32([1.0, 1.05, 1.0500001, 1.2]), 500)).astype(np.float32)
+    s2 = (prev * rng.choice(np.float32([0.9, 1.05, 1.06, 1.3]), 500)).astype(np.float32)
+    thr = np.float32(0.05)
+    st, sc = oracle.confirm(s1, s2, prev, thr)
+    for k in range(500):
+        bar = E.mul(E.from_float(float(thr)), E.from_float(float(prev[k])))
+        f = E.sub(E.from_float(float(s1[k])), E.from_float(float(prev[k]))) > bar
+        c = E.sub(E.from_float(float(s2[k])), E.from_float(float(prev[k]))) > bar
+        want = 0 if not f else (1 if c else 2)
+        assert st[k] == want
+        assert sc[k] == (s1[k] if want == 0 else min(s1[k], s2[k]) if want == 1 else prev[k])
