@@ -290,6 +290,19 @@ kb_status kb_tail_ratios(kb_ctx* ctx, const float* d_timings, uint32_t K, uint32
 kb_status kb_copeland(kb_ctx* ctx, const uint32_t* d_wins, uint32_t K, uint32_t S,
                       uint32_t* d_beats, uint32_t* d_ties, void* stream);
 
+/* Re-measure and confirm (the paper's only description of stability
+ * adjudication, a commented-out passage of Sec. 3: a candidate whose score
+ * change exceeds a threshold is measured again at the same fidelity and
+ * reverted if the improvement is not confirmed).  Per candidate, in binary32:
+ *   flagged   = (first - prev)  > (threshold * prev)
+ *   confirmed = (second - prev) > (threshold * prev)
+ *   not flagged:            status 0, score = first
+ *   flagged and confirmed:  status 1, score = min(first, second)
+ *   flagged, not confirmed: status 2, score = prev
+ * All arrays DEVICE [K]; d_status uint32, the others float. */
+kb_status kb_confirm(kb_ctx* ctx, const float* d_first, const float* d_second, const float* d_prev,
+                     uint32_t K, float threshold, uint32_t* d_status, float* d_score, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

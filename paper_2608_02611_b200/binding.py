@@ -38,7 +38,7 @@ EXPORTS = [
     "kb_ctx_enable_timing", "kb_ctx_read_timer", "kb_ctx_launch_count", "kb_ctx_set_wins_algo", "kb_ctx_set_small_path",
     "kb_mask_create_strided", "kb_mask_create_bitmap", "kb_mask_count", "kb_mask_destroy",
     "kb_screen", "kb_screen_host", "kb_screen_static", "kb_adjudicate", "kb_select",
-    "kb_select_by_score", "kb_tail_ratios", "kb_copeland",
+    "kb_select_by_score", "kb_tail_ratios", "kb_copeland", "kb_confirm",
 ]
 
 
@@ -87,6 +87,7 @@ def load() -> ctypes.CDLL:
     L.kb_select_by_score.argtypes = [vp, vp, vp, u32, u32, u32, f32, f32, u32, vp, vp, vp, vp]
     L.kb_tail_ratios.argtypes = [vp, vp, u32, u32, vp, vp]
     L.kb_copeland.argtypes = [vp, vp, u32, u32, vp, vp, vp]
+    L.kb_confirm.argtypes = [vp, vp, vp, vp, u32, f32, vp, vp, vp]
     for name in EXPORTS:
         if name != "kb_last_error":
             getattr(L, name).restype = i32
@@ -337,6 +338,19 @@ def copeland(self, wins: torch.Tensor, S: int):
                             _stream_ptr(wins.device))
     self._check(rc, "kb_copeland")
     return beats, ties
+
+
+@_ctx_method
+def confirm(self, first: torch.Tensor, second: torch.Tensor, prev: torch.Tensor, threshold: float):
+    """kb_confirm -> (status int32 [K], score float32 [K])."""
+    K = first.numel()
+    status = torch.empty(K, dtype=torch.int32, device=first.device)
+    score = torch.empty(K, dtype=torch.float32, device=first.device)
+    rc = load().kb_confirm(self._h, first.data_ptr(), second.data_ptr(), prev.data_ptr(), K,
+                           float(threshold), status.data_ptr(), score.data_ptr(),
+                           _stream_ptr(first.device))
+    self._check(rc, "kb_confirm")
+    return status, score
 
 
 def records(screen_out: torch.Tensor) -> np.ndarray:

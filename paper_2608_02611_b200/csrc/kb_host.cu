@@ -971,3 +971,19 @@ extern "C" kb_status kb_copeland(kb_ctx* ctx, const uint32_t* d_wins, uint32_t K
   KB_CUDA(ctx, cudaGetLastError());
   return KB_OK;
 }
+
+extern "C" kb_status kb_confirm(kb_ctx* ctx, const float* d_first, const float* d_second,
+                                const float* d_prev, uint32_t K, float threshold,
+                                uint32_t* d_status, float* d_score, void* stream) {
+  if (!ctx) return KB_ERR_INVALID_ARG;
+  if (!d_first || !d_second || !d_prev || !d_status || !d_score)
+    return fail(ctx, KB_ERR_INVALID_ARG, "kb_confirm: null pointer");
+  if (K == 0 || K > KB_MAX_K) return fail(ctx, KB_ERR_INVALID_ARG, "kb_confirm: K=%u outside [1, %u]", K, KB_MAX_K);
+  if (!std::isfinite(threshold)) return fail(ctx, KB_ERR_INVALID_ARG, "kb_confirm: threshold must be finite");
+  DeviceGuard g(ctx->device);
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  confirm_kernel<<<(K + 255) / 256, 256, 0, st>>>(d_first, d_second, d_prev, K, threshold, d_status, d_score);
+  ++ctx->launches;
+  KB_CUDA(ctx, cudaGetLastError());
+  return KB_OK;
+}

@@ -143,4 +143,30 @@ __global__ void __launch_bounds__(256) copeland_kernel(const unsigned int* __res
   }
 }
 
+// Re-measure-and-confirm rule, one thread per candidate.
+__global__ void confirm_kernel(const float* __restrict__ s1, const float* __restrict__ s2,
+                               const float* __restrict__ prev, unsigned int K, float threshold,
+                               unsigned int* __restrict__ status, float* __restrict__ score) {
+  const unsigned int k = blockIdx.x * blockDim.x + threadIdx.x;
+  if (k >= K) return;
+  const float p = prev[k], a = s1[k], b = s2[k];
+  const float bar = __fmul_rn(threshold, p);
+  const bool flagged = __fsub_rn(a, p) > bar;
+  const bool confirmed = __fsub_rn(b, p) > bar;
+  unsigned int st;
+  float sc;
+  if (!flagged) {
+    st = 0u;
+    sc = a;
+  } else if (confirmed) {
+    st = 1u;
+    sc = b < a ? b : a;
+  } else {
+    st = 2u;
+    sc = p;
+  }
+  status[k] = st;
+  score[k] = sc;
+}
+
 }  // namespace kb

@@ -502,3 +502,18 @@ def test_copeland_matches_oracle(ctx, kb, K, S):
     ob, ot = oracle.copeland(oracle.adjudicate(t)[2], S)
     assert (beats.cpu().numpy().view(np.uint32) == ob).all()
     assert (ties.cpu().numpy().view(np.uint32) == ot).all()
+
+
+def test_confirm_matches_oracle(ctx, kb):
+    rng = np.random.default_rng(21)
+    dev = torch.device("cuda", 0)
+    K = 3000
+    prev = rng.lognormal(5, 1, K).astype(np.float32)
+    s1 = (prev * rng.choice(np.float32([0.9, 1.0, 1.05, 1.0500001, 1.2]), K)).astype(np.float32)
+    s2 = (prev * rng.choice(np.float32([0.9, 1.05, 1.06, 1.3]), K)).astype(np.float32)
+    st, sc = ctx.confirm(torch.from_numpy(s1).to(dev), torch.from_numpy(s2).to(dev),
+                         torch.from_numpy(prev).to(dev), 0.05)
+    ost, osc = oracle.confirm(s1, s2, prev, 0.05)
+    assert (st.cpu().numpy().view(np.uint32) == ost).all()
+    assert (fbits(sc.cpu().numpy()) == fbits(osc)).all()
+    assert set(ost.tolist()) == {0, 1, 2}
