@@ -182,6 +182,24 @@ kb_status kb_screen_host(kb_ctx* ctx, const void* h_ref, const void* const* h_ca
                          uint32_t K, uint64_t N, kb_dtype dtype, float atol, float rtol,
                          const kb_mask* mask, kb_screen_result* h_out, void* stream);
 
+/* The same gate on a selection that lives on the device (tier chaining without
+ * a host round trip, e.g. kb_select's output feeding the next tier's screen;
+ * the whole sequence can be recorded in one CUDA graph).  Slot j of the call
+ * is candidate d_table[d_index[j]] for j < *d_count; slots j >= *d_count hold
+ * no candidate and get the record {counts 0, argmax_idx -1, errors 0, pass 0}.
+ *   d_table  DEVICE array of K_all DEVICE pointers (N elements of dtype each).
+ *   d_index  DEVICE int32 [Kmax] (kb_select's d_survivors fits as it is).
+ *   d_count  DEVICE uint32 (kb_select's d_n_survivors).
+ *   d_out    DEVICE [Kmax] records.   1 <= Kmax <= 1024.
+ * What the host cannot check is checked on the device before any tensor is
+ * touched: an index outside [0, K_all), a null or misaligned pointer, or
+ * *d_count > Kmax turns the call into a no-op (all slots "no candidate") and
+ * sets the device status to KB_ERR_INVALID_ARG / KB_ERR_ALIGNMENT. */
+kb_status kb_screen_indexed(kb_ctx* ctx, const void* d_ref, const void* const* d_table,
+                            uint32_t K_all, const int32_t* d_index, const uint32_t* d_count,
+                            uint32_t Kmax, uint64_t N, kb_dtype dtype, float atol, float rtol,
+                            const kb_mask* mask, kb_screen_result* d_out, void* stream);
+
 /* ---- the same gate for callers that must not allocate ----------------------
  * (The paper has no counterpart; this entry point exists for integration.)
  *

@@ -37,7 +37,7 @@ EXPORTS = [
     "kb_ctx_create", "kb_ctx_destroy", "kb_last_error", "kb_ctx_poll", "kb_ctx_set_grid",
     "kb_ctx_enable_timing", "kb_ctx_read_timer", "kb_ctx_launch_count", "kb_ctx_set_wins_algo", "kb_ctx_set_small_path",
     "kb_mask_create_strided", "kb_mask_create_bitmap", "kb_mask_count", "kb_mask_destroy",
-    "kb_screen", "kb_screen_host", "kb_screen_static", "kb_adjudicate", "kb_select",
+    "kb_screen", "kb_screen_host", "kb_screen_static", "kb_screen_indexed", "kb_adjudicate", "kb_select",
     "kb_select_by_score", "kb_tail_ratios", "kb_copeland", "kb_confirm",
 ]
 
@@ -81,6 +81,7 @@ def load() -> ctypes.CDLL:
     L.kb_mask_destroy.argtypes = [vp]
     L.kb_screen.argtypes = [vp, vp, vp, u32, u64, i32, f32, f32, vp, vp, vp]
     L.kb_screen_host.argtypes = [vp, vp, vp, u32, u64, i32, f32, f32, vp, vp, vp]
+    L.kb_screen_indexed.argtypes = [vp, vp, vp, u32, vp, vp, u32, u64, i32, f32, f32, vp, vp, vp]
     L.kb_screen_static.argtypes = [vp, vp, u32, u64, i32, f32, f32, vp, vp]
     L.kb_adjudicate.argtypes = [vp, vp, u32, u32, vp, vp, vp, vp]
     L.kb_select.argtypes = [vp, vp, vp, u32, i32, u32, vp, vp, vp]
@@ -338,6 +339,30 @@ def copeland(self, wins: torch.Tensor, S: int):
                             _stream_ptr(wins.device))
     self._check(rc, "kb_copeland")
     return beats, ties
+
+
+@_ctx_method
+def pointer_table(self, cands: Sequence[torch.Tensor]) -> torch.Tensor:
+    """A device array holding the candidates' addresses (for screen_indexed)."""
+    return torch.tensor([c.data_ptr() for c in cands], dtype=torch.int64, device=self.device)
+
+
+@_ctx_method
+def screen_indexed(self, ref: torch.Tensor, table: torch.Tensor, index: torch.Tensor,
+                   count: torch.Tensor, atol: float, rtol: float, mask=None,
+                   out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """kb_screen_indexed: slot j is candidate table[index[j]] for j < count; everything stays
+    on the device (no host synchronisation).  Returns a uint8 CUDA tensor [len(index), 48]."""
+    Kmax = index.numel()
+    if out is None:
+        out = torch.empty((Kmax, RESULT_BYTES), dtype=torch.uint8, device=ref.device)
+    rc = load().kb_screen_indexed(self._h, ref.data_ptr(), table.data_ptr(), table.numel(),
+                                  index.data_ptr(), count.data_ptr(), Kmax, ref.numel(),
+                                  DTYPE_CODE.get(ref.dtype, -1), float(atol), float(rtol),
+                                  mask._h if mask is not None else None, out.data_ptr(),
+                                  _stream_ptr(ref.device))
+    self._check(rc, "kb_screen_indexed")
+    return out
 
 
 @_ctx_method

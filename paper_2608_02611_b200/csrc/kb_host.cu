@@ -166,14 +166,14 @@ kb_status launch_stream(kb_ctx* ctx, StreamParams& sp, cudaStream_t st) {
 template <int DT>
 kb_status launch_generic(kb_ctx* ctx, const void* ref, const void* const* tab, Acc* acc, uint32_t K,
                          uint64_t e0, uint64_t e1, float atol, float rtol, const MaskDev& md,
-                         cudaStream_t st) {
+                         const unsigned int* count, cudaStream_t st) {
   if (e1 <= e0) return KB_OK;
   const uint64_t len = e1 - e0;
   uint64_t bx = (len + 255) / 256;
   const uint64_t cap = (uint64_t)ctx->sm_count * 8;
   if (bx > cap) bx = cap;
   dim3 grid((unsigned int)bx, K);
-  screen_generic_kernel<DT><<<grid, 256, 0, st>>>(ref, tab, acc, e0, e1, atol, rtol, md);
+  screen_generic_kernel<DT><<<grid, 256, 0, st>>>(ref, tab, acc, e0, e1, atol, rtol, md, count);
   ++ctx->launches;
   KB_CUDA(ctx, cudaGetLastError());
   return KB_OK;
@@ -511,13 +511,21 @@ kb_status validate_screen(kb_ctx* ctx, const void* ref, const void* const* cands
   return KB_OK;
 }
 
+// A selection of candidates that lives on the device (kb_screen_indexed).
+struct IndexedSel {
+  const void* const* d_table;
+  uint32_t K_all;
+  const int32_t* d_index;
+  const uint32_t* d_count;
+};
+
 template <int DT>
 kb_status screen_impl(kb_ctx* ctx, const void* d_ref, const void* const* h_cands, uint32_t K,
                       uint64_t N, float atol, float rtol, const kb_mask* mask,
-                      kb_screen_result* d_out, cudaStream_t st) {
+                      kb_screen_result* d_out, cudaStream_t st, const IndexedSel* sel = nullptr) {
   // Latency-bound sizes: everything in one launch (pointers as kernel arguments).
   const uint64_t nb_small = (N + kSmallPerBlock - 1) / kSmallPerBlock;
-  if (ctx->small_ws && ctx->small_on && K <= (uint32_t)kPtrsPerLaunch && (uint64_t)K * N <= (1ull << 22) &&
+  if (!sel && ctx->small_ws && ctx->small_on && K <= (uint32_t)kPtrsPerLaunch && (uint64_t)K * N <= (1ull << 22) &&
       (uint64_t)K * nb_small <= kSmallMaxPartials) {
     SmallParams sm;
     sm.ref = d_ref;
@@ -546,7 +554,15 @@ kb_status screen_impl(kb_ctx* ctx, const void* d_ref, const void* const* h_cands
   Acc* acc = reinterpret_cast<Acc*>(ctx->ws);
   const void** table = reinterpret_cast<const void**>(ctx->ws + round_up((size_t)K * sizeof(Acc), 256));
 
-  for (uint32_t off = 0; off < K; off += kPtrsPerLaunch) {
+  // with a device-resident selection the later kernels read the effective candidate count
+  const unsigned int* count = sel ? ctx->d_status + 4 : nullptr;
+  if (sel) {
+    screen_prep_indexed_kernel<<<1, 256, 0, st>>>(sel->d_table, sel->K_all, sel->d_index, sel->d_count, K,
+                                                  table, acc, ctx->d_status, ctx->d_status);
+    ++ctx->launches;
+    KB_CUDA(ctx, cudaGetLastError());
+  }
+  for (uint32_t off = 0; !sel && off < K; off += kPtrsPerLaunch) {
     PtrChunk ch;
     const uint32_t cnt = (K - off < (uint32_t)kPtrsPerLaunch) ? K - off : (uint32_t)kPtrsPerLaunch;
     memcpy(ch.p, h_cands + off, cnt * sizeof(void*));
@@ -564,7 +580,7 @@ kb_status screen_impl(kb_ctx* ctx, const void* d_ref, const void* const* h_cands
 
   if (mask && !mask->coarse) {
     // finer than a kernel tile: every sector is touched anyway
-    rc = launch_generic<DT>(ctx, d_ref, table, acc, K, 0, N, atol, rtol, md, st);
+    rc = launch_generic<DT>(ctx, d_ref, table, acc, K, 0, N, atol, rtol, md, count, st);
     if (rc != KB_OK) return rc;
   } else {
     const uint64_t nfull = N / kTile;
@@ -575,6 +591,7 @@ kb_status screen_impl(kb_ctx* ctx, const void* d_ref, const void* const* h_cands
     sp.tile_list = mask ? mask->d_tiles : nullptr;
     sp.ntiles = mask ? mask->n_tiles : (uint32_t)nfull;
     sp.K = K;
+    sp.K_dev = count;
     sp.atol = atol;
     sp.rtol = rtol;
     sp.rtol_lean = -1.0f;
@@ -593,7 +610,7 @@ kb_status screen_impl(kb_ctx* ctx, const void* d_ref, const void* const* h_cands
       if (nscout < 1) nscout = 1;
       if (nscout > 8) nscout = 8;
       dim3 sg(nscout * (kTile / kScoutPerBlock), K);
-      screen_scout_kernel<DT><<<sg, 256, 0, st>>>(d_ref, table, acc, sp.tile_list, atol, rtol);
+      screen_scout_kernel<DT><<<sg, 256, 0, st>>>(d_ref, table, acc, sp.tile_list, atol, rtol, count);
       ++ctx->launches;
       KB_CUDA(ctx, cudaGetLastError());
     }
@@ -601,7 +618,7 @@ kb_status screen_impl(kb_ctx* ctx, const void* d_ref, const void* const* h_cands
     sp.ntiles -= nscout;
     // ragged tail (elements past the last full kernel tile), before the streaming
     // kernel so that its last CTA can unpack the finished records
-    rc = launch_generic<DT>(ctx, d_ref, table, acc, K, nfull * kTile, N, atol, rtol, md, st);
+    rc = launch_generic<DT>(ctx, d_ref, table, acc, K, nfull * kTile, N, atol, rtol, md, count, st);
     if (rc != KB_OK) return rc;
     if (sp.ntiles) {
       // chunk the candidates: shared-memory accumulators hold kMaxKC of them, and
@@ -623,7 +640,7 @@ kb_status screen_impl(kb_ctx* ctx, const void* d_ref, const void* const* h_cands
       return launch_stream<DT>(ctx, sp, st);
     }
   }
-  screen_finalize_kernel<<<(K + 127) / 128, 128, 0, st>>>(acc, d_out, K);
+  screen_finalize_kernel<<<(K + 127) / 128, 128, 0, st>>>(acc, d_out, K, count);
   ++ctx->launches;
   KB_CUDA(ctx, cudaGetLastError());
   return KB_OK;
@@ -631,11 +648,11 @@ kb_status screen_impl(kb_ctx* ctx, const void* d_ref, const void* const* h_cands
 
 kb_status screen_dispatch(kb_ctx* ctx, const void* d_ref, const void* const* h_cands, uint32_t K,
                           uint64_t N, kb_dtype dtype, float atol, float rtol, const kb_mask* mask,
-                          kb_screen_result* d_out, cudaStream_t st) {
+                          kb_screen_result* d_out, cudaStream_t st, const IndexedSel* sel = nullptr) {
   switch (dtype) {
-    case KB_F32: return screen_impl<KB_F32>(ctx, d_ref, h_cands, K, N, atol, rtol, mask, d_out, st);
-    case KB_F16: return screen_impl<KB_F16>(ctx, d_ref, h_cands, K, N, atol, rtol, mask, d_out, st);
-    default: return screen_impl<KB_BF16>(ctx, d_ref, h_cands, K, N, atol, rtol, mask, d_out, st);
+    case KB_F32: return screen_impl<KB_F32>(ctx, d_ref, h_cands, K, N, atol, rtol, mask, d_out, st, sel);
+    case KB_F16: return screen_impl<KB_F16>(ctx, d_ref, h_cands, K, N, atol, rtol, mask, d_out, st, sel);
+    default: return screen_impl<KB_BF16>(ctx, d_ref, h_cands, K, N, atol, rtol, mask, d_out, st, sel);
   }
 }
 
@@ -649,6 +666,32 @@ extern "C" kb_status kb_screen(kb_ctx* ctx, const void* d_ref, const void* const
   DeviceGuard g(ctx->device);
   return screen_dispatch(ctx, d_ref, h_cands, K, N, dtype, atol, rtol, mask, d_out,
                          reinterpret_cast<cudaStream_t>(stream));
+}
+
+extern "C" kb_status kb_screen_indexed(kb_ctx* ctx, const void* d_ref, const void* const* d_table,
+                                       uint32_t K_all, const int32_t* d_index,
+                                       const uint32_t* d_count, uint32_t Kmax, uint64_t N,
+                                       kb_dtype dtype, float atol, float rtol, const kb_mask* mask,
+                                       kb_screen_result* d_out, void* stream) {
+  if (!ctx) return KB_ERR_INVALID_ARG;
+  if (!d_ref || !d_table || !d_index || !d_count || !d_out)
+    return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen_indexed: null pointer");
+  if (Kmax == 0 || Kmax > 1024) return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen_indexed: Kmax=%u outside [1, 1024]", Kmax);
+  if (K_all == 0) return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen_indexed: K_all is 0");
+  if (N == 0 || N > KB_MAX_N) return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen_indexed: N outside [1, 2^32]");
+  if (dtype != KB_F32 && dtype != KB_F16 && dtype != KB_BF16)
+    return fail(ctx, KB_ERR_UNSUPPORTED, "kb_screen_indexed: unknown dtype %d", (int)dtype);
+  if (!(atol >= 0.0f) || !(rtol >= 0.0f) || std::isinf(atol) || std::isinf(rtol))
+    return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen_indexed: atol and rtol must be finite and >= 0");
+  if (mask && (mask->N != N || mask->ctx != ctx))
+    return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen_indexed: the mask was created for another N or context");
+  if (!aligned16(d_ref)) return fail(ctx, KB_ERR_ALIGNMENT, "kb_screen_indexed: reference not 16-byte aligned");
+  if ((reinterpret_cast<uintptr_t>(d_out) & 7u) != 0)
+    return fail(ctx, KB_ERR_ALIGNMENT, "kb_screen_indexed: output not 8-byte aligned");
+  DeviceGuard g(ctx->device);
+  IndexedSel sel{d_table, K_all, d_index, d_count};
+  return screen_dispatch(ctx, d_ref, nullptr, Kmax, N, dtype, atol, rtol, mask, d_out,
+                         reinterpret_cast<cudaStream_t>(stream), &sel);
 }
 
 // ---------------------------------------------------------------------------

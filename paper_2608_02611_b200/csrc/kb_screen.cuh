@@ -34,6 +34,7 @@ struct StreamParams {
   uint32_t ntiles;              // number of full tiles to visit
   uint32_t slot0;               // first slot of the tile list / first tile (earlier ones were scouted)
   uint32_t K, KC, nchunks;
+  const unsigned int* K_dev;    // optional: the number of candidates actually present (<= K)
   uint32_t stages;
   float atol, rtol;
   float rtol_lean;              // rtol*(1-2^-20) rounded down, or -1: see the lean filter below
@@ -79,6 +80,18 @@ __device__ __forceinline__ void unpack_record(const Acc& a, kb_screen_result* ds
   }
   r.max_rel_err = __uint_as_float(a.rel);
   r.pass = a.mism == 0ull ? 1u : 0u;
+  r.reserved = 0u;
+  *dst = r;
+}
+
+// record of a candidate slot that holds no candidate (indexed screening with fewer
+// survivors than slots): nothing counted, no index, not passed
+__device__ __forceinline__ void write_absent_record(kb_screen_result* dst) {
+  kb_screen_result r;
+  r.mismatch_count = r.nan_count = r.inf_count = 0ull;
+  r.argmax_idx = -1;
+  r.max_abs_err = r.max_rel_err = 0.0f;
+  r.pass = 0u;
   r.reserved = 0u;
   *dst = r;
 }
@@ -201,7 +214,9 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
   // Work items (chunk, tile), chunk-major, are drawn from a global counter: a CTA gets
   // ascending items (so ascending tiles inside a chunk, which the index tie-break needs),
   // the CTAs that run together work on neighbouring tiles, and the tail is one item long.
-  const unsigned long long nitems = (unsigned long long)p.nchunks * p.ntiles;
+  const uint32_t K_eff = p.K_dev ? min(*p.K_dev, p.K) : p.K;
+  const uint32_t nchunks_eff = (K_eff + p.KC - 1) / p.KC;
+  const unsigned long long nitems = (unsigned long long)nchunks_eff * p.ntiles;
   constexpr unsigned long long kNoItem = ~0ull;
 
   if (warp == kWarps) {
@@ -221,7 +236,7 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
       const uint32_t chunk = (uint32_t)(item / p.ntiles);
       const uint32_t slot = p.slot0 + (uint32_t)(item % p.ntiles);
       const uint32_t k0 = chunk * p.KC;
-      const int kc = (int)min(p.KC, p.K - k0);
+      const int kc = (int)min(p.KC, K_eff - k0);
       if ((int)chunk != cur_chunk) {
         // the chunk's candidate pointers go to shared memory once (whole warp)
         cur_chunk = (int)chunk;
@@ -376,7 +391,7 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
         }
         cur_chunk = (int)chunk;
         cur_k0 = chunk * p.KC;
-        cur_kc = (int)min(p.KC, p.K - cur_k0);
+        cur_kc = (int)min(p.KC, K_eff - cur_k0);
       }
       const unsigned long long tile_base = (unsigned long long)tile * kTile;
 
@@ -544,6 +559,10 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
   if (s_ticket == gridDim.x - 1) {
     __threadfence();
     for (unsigned int k = tid; k < p.K; k += kStreamThreads) {
+      if (k >= K_eff) {
+        write_absent_record(&p.out[k]);
+        continue;
+      }
       Acc a;
       a.mism = __ldcg(&p.acc[k].mism);
       a.nan = __ldcg(&p.acc[k].nan);
@@ -604,9 +623,11 @@ __global__ void __launch_bounds__(256) screen_generic_kernel(const void* __restr
                                                              Acc* __restrict__ acc,
                                                              unsigned long long e0,
                                                              unsigned long long e1, float atol,
-                                                             float rtol, MaskDev mask) {
+                                                             float rtol, MaskDev mask,
+                                                             const unsigned int* __restrict__ count) {
   using E = Elem<DT>;
   const unsigned int k = blockIdx.y;
+  if (count && k >= *count) return;
   const void* cand = cands[k];
   ExactAcc x;
   const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
@@ -629,9 +650,11 @@ __global__ void __launch_bounds__(256) screen_scout_kernel(const void* __restric
                                                            const void* const* __restrict__ cands,
                                                            Acc* __restrict__ acc,
                                                            const uint32_t* __restrict__ tile_list,
-                                                           float atol, float rtol) {
+                                                           float atol, float rtol,
+                                                           const unsigned int* __restrict__ count) {
   using E = Elem<DT>;
   constexpr unsigned int kBlocksPerTile = kTile / kScoutPerBlock;
+  if (count && blockIdx.y >= *count) return;
   __shared__ unsigned int s_cnt[3];
   __shared__ unsigned int s_rel;
   __shared__ unsigned long long s_key;
@@ -784,10 +807,13 @@ __global__ void __launch_bounds__(256) screen_small_kernel(const SmallParams p, 
 }
 
 __global__ void screen_finalize_kernel(const Acc* __restrict__ acc, kb_screen_result* __restrict__ out,
-                                       unsigned int K) {
+                                       unsigned int K, const unsigned int* __restrict__ count) {
   const unsigned int k = blockIdx.x * blockDim.x + threadIdx.x;
   if (k >= K) return;
-  unpack_record(acc[k], &out[k]);
+  if (count && k >= *count)
+    write_absent_record(&out[k]);
+  else
+    unpack_record(acc[k], &out[k]);
 }
 
 // Also zeroes the accumulators of the same candidates and the ticket counter.
@@ -805,6 +831,49 @@ __global__ void screen_prep_kernel(const PtrChunk chunk, const void** table, Acc
     done[0] = 0u;   // ticket counter
     done[1] = 0u;   // work counter (64 bits)
     done[2] = 0u;
+  }
+}
+
+// Indexed screening: candidate slot j holds table[index[j]] for j < *count.  Builds the
+// slot pointer table on the device, zeroes accumulators and counters, and validates what
+// the host cannot see: an index outside [0, K_all), a null or misaligned pointer, or a
+// count above the slots makes the whole call a no-op (effective count 0) and sets the
+// device status, so that no later kernel ever touches a bad address.
+__global__ void screen_prep_indexed_kernel(const void* const* __restrict__ all, unsigned int K_all,
+                                           const int* __restrict__ index,
+                                           const unsigned int* __restrict__ count, unsigned int Kmax,
+                                           const void** table, Acc* acc, unsigned int* words,
+                                           unsigned int* status) {
+  // single block: Kmax <= 1024 slots
+  __shared__ unsigned int s_bad;
+  if (threadIdx.x == 0) s_bad = 0u;
+  __syncthreads();
+  const unsigned int n = *count;
+  if (n > Kmax && threadIdx.x == 0) s_bad = 1u;
+  for (unsigned int j = threadIdx.x; j < Kmax; j += blockDim.x) {
+    const void* ptr = nullptr;
+    if (j < n && n <= Kmax) {
+      const int ix = index[j];
+      if (ix < 0 || (unsigned int)ix >= K_all) {
+        atomicOr(&s_bad, 1u);
+      } else {
+        ptr = all[ix];
+        if (!ptr || (reinterpret_cast<uintptr_t>(ptr) & 15u)) atomicOr(&s_bad, 2u);
+      }
+    }
+    table[j] = ptr;
+    Acc z;
+    z.mism = z.nan = z.inf = z.key = 0ull;
+    z.rel = z.pad = 0u;
+    acc[j] = z;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    words[1] = 0u;   // ticket counter
+    words[2] = 0u;   // work counter (64 bits)
+    words[3] = 0u;
+    words[4] = s_bad ? 0u : n;   // effective number of candidates
+    if (s_bad) set_status(status, (unsigned int)((s_bad & 2u) ? KB_ERR_ALIGNMENT : KB_ERR_INVALID_ARG));
   }
 }
 

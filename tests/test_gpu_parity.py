@@ -517,3 +517,104 @@ def test_confirm_matches_oracle(ctx, kb):
     assert (st.cpu().numpy().view(np.uint32) == ost).all()
     assert (fbits(sc.cpu().numpy()) == fbits(osc)).all()
     assert set(ost.tolist()) == {0, 1, 2}
+
+
+# --------------------------------------------------------------------------
+# device-resident tier chaining: select -> screen_indexed, no host round trip
+# --------------------------------------------------------------------------
+
+def _tier_setup(dev):
+    c5 = synth.config5("cpu", N=(1 << 20) + 333, K=32, budget=4, S1=20, S2=40)
+    case = c5["case"]
+    ref = case.ref.to(dev)
+    cands_cpu = case.cands()
+    cands = [c.to(dev) for c in cands_cpu]
+    return c5, case, ref, cands_cpu, cands
+
+
+@pytest.mark.parametrize("budget", [4, 30])
+def test_screen_indexed_chain(ctx, kb, budget):
+    dev = torch.device("cuda", 0)
+    c5, case, ref, cands_cpu, cands = _tier_setup(dev)
+    _, log2_tile, stride, phase = case.mask
+    mask = ctx.mask_strided(case.N, log2_tile, stride, phase)
+    table = ctx.pointer_table(cands)
+    out1 = ctx.screen(ref, cands, case.atol, case.rtol, mask)
+    med1, _, _ = ctx.adjudicate(torch.from_numpy(c5["timings1"]).to(dev))
+    surv, n = ctx.select(out1, med1, kb.KB_SELECT_ERR_THEN_TIME, budget)
+    out2 = ctx.screen_indexed(ref, table, surv, n, case.atol, case.rtol)      # nothing came to the host yet
+    assert ctx.poll() == 0
+    s = surv.cpu().numpy()
+    nn = int(n.item())
+    assert nn == min(budget, 16) and (s[nn:] == -1).all()
+    rec2 = kb.records(out2)
+    want = oracle_screen(case.dtype, case.ref, [cands_cpu[k] for k in s[:nn]], case.atol, case.rtol)
+    assert_records_equal(rec2[:nn], want, "indexed tier 2")
+    for j in range(nn, budget):                                            # empty slots
+        r = rec2[j]
+        assert (r["mismatch_count"], r["nan_count"], r["inf_count"], r["argmax_idx"], r["pass"]) == (0, 0, 0, -1, 0)
+    # the same through the host-driven call
+    rec_host = kb.records(ctx.screen(ref, [cands[k] for k in s[:nn]], case.atol, case.rtol))
+    assert rec_host.tobytes() == rec2[:nn].tobytes()
+    mask.close()
+
+
+def test_screen_indexed_rejects_bad_selections_on_the_device(ctx, kb):
+    dev = torch.device("cuda", 0)
+    N = 3 * 4096 + 5
+    ref = torch.zeros(N, dtype=torch.float32, device=dev)
+    big = torch.zeros(N + 1, dtype=torch.float32, device=dev)
+    good = ref.clone()                                                     # must outlive the table
+    table = ctx.pointer_table([good, big[1:]])                             # entry 1 is misaligned
+    one = torch.tensor([1], dtype=torch.int32, device=dev)
+    cases = [(torch.tensor([0, 7], dtype=torch.int32, device=dev), torch.tensor([2], dtype=torch.int32, device=dev), 1),
+             (torch.tensor([0, 1], dtype=torch.int32, device=dev), torch.tensor([2], dtype=torch.int32, device=dev), 2),
+             (torch.tensor([0, 0], dtype=torch.int32, device=dev), torch.tensor([3], dtype=torch.int32, device=dev), 1)]
+    for index, count, status in cases:
+        out = ctx.screen_indexed(ref, table, index, count, 0.0, 0.0)
+        assert ctx.poll() == status
+        rec = kb.records(out)
+        assert (rec["pass"] == 0).all() and (rec["argmax_idx"] == -1).all()
+    out = ctx.screen_indexed(ref, table, torch.tensor([0, 1], dtype=torch.int32, device=dev), one, 0.0, 0.0)
+    assert ctx.poll() == 0                                                  # the bad entry is beyond the count
+    rec = kb.records(out)
+    assert rec["pass"].tolist() == [1, 0] and rec["argmax_idx"].tolist() == [0, -1]
+
+
+def test_two_tier_chain_in_one_cuda_graph(ctx, kb):
+    dev = torch.device("cuda", 0)
+    c5, case, ref, cands_cpu, cands = _tier_setup(dev)
+    _, log2_tile, stride, phase = case.mask
+    mask = ctx.mask_strided(case.N, log2_tile, stride, phase)
+    table = ctx.pointer_table(cands)
+    t1 = torch.from_numpy(c5["timings1"]).to(dev)
+    budget = 4
+    out1 = torch.empty((case.K, kb.RESULT_BYTES), dtype=torch.uint8, device=dev)
+    out2 = torch.empty((budget, kb.RESULT_BYTES), dtype=torch.uint8, device=dev)
+
+    def chain():
+        ctx.screen(ref, cands, case.atol, case.rtol, mask, out=out1)
+        med, iqr, wins = ctx.adjudicate(t1)
+        surv, n = ctx.select(out1, med, kb.KB_SELECT_ERR_THEN_TIME, budget)
+        ctx.screen_indexed(ref, table, surv, n, case.atol, case.rtol, out=out2)
+        return surv, n
+
+    surv, n = chain()                      # warm-up: grows every workspace before the capture
+    torch.cuda.synchronize()
+    want1, want2 = kb.records(out1).tobytes(), kb.records(out2).tobytes()
+    want_s = surv.cpu().numpy().tolist()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            g_surv, g_n = chain()
+    for _ in range(2):
+        out1.fill_(0xEE)
+        out2.fill_(0xEE)
+        graph.replay()
+        torch.cuda.synchronize()
+        assert kb.records(out1).tobytes() == want1 and kb.records(out2).tobytes() == want2
+        assert g_surv.cpu().numpy().tolist() == want_s
+    assert ctx.poll() == 0
+    mask.close()
