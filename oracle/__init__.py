@@ -85,6 +85,8 @@ def lib() -> ctypes.CDLL:
         L.kbo_copeland.restype = i32
         L.kbo_confirm.argtypes = [vp, vp, vp, u32, f32, vp, vp]
         L.kbo_confirm.restype = i32
+        L.kbo_adjudicate_ragged.argtypes = [vp, vp, u32, vp, vp, vp]
+        L.kbo_adjudicate_ragged.restype = i32
         L.kbo_decode_f16.argtypes = [ctypes.c_uint16]
         L.kbo_decode_f16.restype = f32
         L.kbo_decode_bf16.argtypes = [ctypes.c_uint16]
@@ -301,3 +303,22 @@ def confirm(s1, s2, prev, threshold: float):
     if rc != 0:
         raise ValueError(f"kbo_confirm rejected its arguments (rc={rc})")
     return st, sc
+
+
+def adjudicate_ragged(rows):
+    """median[K], iqr[K], wins[K][K] for rows of different lengths (a list of 1-D arrays)."""
+    rows = [np.ascontiguousarray(r, dtype=np.float32).reshape(-1) for r in rows]
+    K = len(rows)
+    off = np.zeros(K + 1, dtype=np.uint32)
+    off[1:] = np.cumsum([r.size for r in rows])
+    flat = np.concatenate(rows) if K else np.zeros(0, np.float32)
+    med = np.zeros(K, dtype=np.float32)
+    iqr = np.zeros(K, dtype=np.float32)
+    wins = np.zeros((K, K), dtype=np.uint32)
+    rc = lib().kbo_adjudicate_ragged(flat.ctypes.data, off.ctypes.data, K, med.ctypes.data,
+                                     iqr.ctypes.data, wins.ctypes.data)
+    if rc == -2:
+        raise NonFiniteTiming("non-finite timing")
+    if rc != 0:
+        raise ValueError(f"kbo_adjudicate_ragged rejected its arguments (rc={rc})")
+    return med, iqr, wins

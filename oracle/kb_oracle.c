@@ -503,3 +503,41 @@ int kbo_confirm(const float* s1, const float* s2, const float* prev, uint32_t K,
   }
   return 0;
 }
+
+/*
+ * Adjudication with a different number of timings per candidate (a candidate
+ * may have been measured at another fidelity, Sec. 3.2 "Fidelity level").
+ * Row k is timings[offsets[k] .. offsets[k+1]), S_k = its length >= 1.
+ * median/iqr as in kbo_quantiles on each row; the win count is the same double
+ * loop, so that W[a][b] + W[b][a] = 2*S_a*S_b and W[a][a] = S_a*S_a.
+ * Returns 0; -1 bad argument; -2 non-finite timing.
+ */
+int kbo_adjudicate_ragged(const float* timings, const uint32_t* offsets, uint32_t K, float* median,
+                          float* iqr, uint32_t* wins) {
+  uint32_t a, b, i, j;
+  if (!timings || !offsets || K == 0) return -1;
+  for (a = 0; a < K; ++a)
+    if (offsets[a + 1] <= offsets[a]) return -1;
+  for (i = offsets[0]; i < offsets[K]; ++i)
+    if (!is_finite32(timings[i])) return -2;
+  for (a = 0; a < K; ++a) {
+    float q[4];
+    int rc = kbo_quantiles(timings + offsets[a], offsets[a + 1] - offsets[a], q, NULL);
+    if (rc != 0) return rc;
+    if (median) median[a] = q[1];
+    if (iqr) iqr[a] = q[3];
+  }
+  if (wins) {
+    for (a = 0; a < K; ++a)
+      for (b = 0; b < K; ++b) {
+        uint64_t w = 0;
+        for (i = offsets[a]; i < offsets[a + 1]; ++i)
+          for (j = offsets[b]; j < offsets[b + 1]; ++j) {
+            if (timings[i] < timings[j]) w += 2;
+            if (timings[i] == timings[j]) w += 1;
+          }
+        wins[(size_t)a * K + b] = (uint32_t)w;
+      }
+  }
+  return 0;
+}

@@ -139,3 +139,33 @@ def test_nonfinite_timing_is_an_error():
             oracle.adjudicate(t2)
         with pytest.raises(oracle.NonFiniteTiming):
             oracle.quantiles(t2[1])
+
+
+# ---- rows of different lengths --------------------------------------------------------------
+
+def test_ragged_wins_equal_scipy_and_sum_to_twice_the_product():
+    """U_ab + U_ba = S_a * S_b (doubled here), for unequal sample counts."""
+    rng = np.random.default_rng(31)
+    rows = [np.round(rng.lognormal(0, 0.2, n), 1).astype(np.float32) for n in (1, 4, 7, 16, 60, 3)]
+    med, iqr, W = oracle.adjudicate_ragged(rows)
+    K = len(rows)
+    for a in range(K):
+        q, _ = oracle.quantiles(rows[a])
+        assert med[a] == q[1] and iqr[a] == q[3]
+        assert W[a, a] == rows[a].size ** 2
+        for b in range(K):
+            assert int(W[a, b]) + int(W[b, a]) == 2 * rows[a].size * rows[b].size
+            if a != b:
+                U = stats.mannwhitneyu(rows[a].astype(np.float64), rows[b].astype(np.float64),
+                                       alternative="two-sided", method="asymptotic").statistic
+                assert int(W[a, b]) == round(2 * rows[a].size * rows[b].size - 2 * U)
+
+
+def test_ragged_with_equal_lengths_is_the_rectangular_case():
+    rng = np.random.default_rng(32)
+    t = np.round(rng.lognormal(0, 0.1, (6, 9)), 2).astype(np.float32)
+    m1, i1, w1 = oracle.adjudicate(t)
+    m2, i2, w2 = oracle.adjudicate_ragged(list(t))
+    assert (m1 == m2).all() and (i1 == i2).all() and (w1 == w2).all()
+    with pytest.raises(oracle.NonFiniteTiming):
+        oracle.adjudicate_ragged([np.float32([1, 2]), np.float32([np.inf])])
