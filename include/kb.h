@@ -254,6 +254,19 @@ kb_status kb_screen_static(const void* d_ref, const void* const* h_cands, uint32
 kb_status kb_adjudicate(kb_ctx* ctx, const float* d_timings, uint32_t K, uint32_t S,
                         float* d_median, float* d_iqr, uint32_t* d_wins, void* stream);
 
+/* The same with a different number of timings per candidate (candidates
+ * measured at different fidelities): row k is d_timings[d_offsets[k] ..
+ * d_offsets[k+1]), S_k = its length.  Median and IQR per row as above;
+ * W[a][b] by the same double sum, so W[a][b] + W[b][a] = 2*S_a*S_b and
+ * W[a][a] = S_a*S_a.
+ *   d_offsets  DEVICE uint32 [K+1], ascending.
+ *   S_max      an upper bound of every S_k, 1 <= S_max <= 4096.  A row that is
+ *              empty or longer than S_max sets the device status to
+ *              KB_ERR_INVALID_ARG; its outputs are then unspecified. */
+kb_status kb_adjudicate_ragged(kb_ctx* ctx, const float* d_timings, const uint32_t* d_offsets,
+                               uint32_t K, uint32_t S_max, uint64_t total, float* d_median,
+                               float* d_iqr, uint32_t* d_wins, void* stream);
+
 /* ---- promotion decision (Sec. 3.2; Sec. 3.4 scheduler; Algorithm 1, D) --- */
 
 typedef enum {

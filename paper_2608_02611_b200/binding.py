@@ -37,7 +37,7 @@ EXPORTS = [
     "kb_ctx_create", "kb_ctx_destroy", "kb_last_error", "kb_ctx_poll", "kb_ctx_set_grid",
     "kb_ctx_enable_timing", "kb_ctx_read_timer", "kb_ctx_launch_count", "kb_ctx_set_wins_algo", "kb_ctx_set_small_path",
     "kb_mask_create_strided", "kb_mask_create_bitmap", "kb_mask_count", "kb_mask_destroy",
-    "kb_screen", "kb_screen_host", "kb_screen_static", "kb_screen_indexed", "kb_adjudicate", "kb_select",
+    "kb_screen", "kb_screen_host", "kb_screen_static", "kb_screen_indexed", "kb_adjudicate", "kb_adjudicate_ragged", "kb_select",
     "kb_select_by_score", "kb_tail_ratios", "kb_copeland", "kb_confirm",
 ]
 
@@ -84,6 +84,7 @@ def load() -> ctypes.CDLL:
     L.kb_screen_indexed.argtypes = [vp, vp, vp, u32, vp, vp, u32, u64, i32, f32, f32, vp, vp, vp]
     L.kb_screen_static.argtypes = [vp, vp, u32, u64, i32, f32, f32, vp, vp]
     L.kb_adjudicate.argtypes = [vp, vp, u32, u32, vp, vp, vp, vp]
+    L.kb_adjudicate_ragged.argtypes = [vp, vp, vp, u32, u32, u64, vp, vp, vp, vp]
     L.kb_select.argtypes = [vp, vp, vp, u32, i32, u32, vp, vp, vp]
     L.kb_select_by_score.argtypes = [vp, vp, vp, u32, u32, u32, f32, f32, u32, vp, vp, vp, vp]
     L.kb_tail_ratios.argtypes = [vp, vp, u32, u32, vp, vp]
@@ -363,6 +364,21 @@ def screen_indexed(self, ref: torch.Tensor, table: torch.Tensor, index: torch.Te
                                   _stream_ptr(ref.device))
     self._check(rc, "kb_screen_indexed")
     return out
+
+
+@_ctx_method
+def adjudicate_ragged(self, flat: torch.Tensor, offsets: torch.Tensor, S_max: int):
+    """kb_adjudicate_ragged: flat float32 timings, int32 offsets [K+1] (both CUDA) ->
+    (median[K], iqr[K], wins[K,K])."""
+    K = offsets.numel() - 1
+    med = torch.empty(K, dtype=torch.float32, device=flat.device)
+    iqr = torch.empty(K, dtype=torch.float32, device=flat.device)
+    wins = torch.empty((K, K), dtype=torch.int32, device=flat.device)
+    rc = load().kb_adjudicate_ragged(self._h, flat.data_ptr(), offsets.data_ptr(), K, int(S_max),
+                                     flat.numel(), med.data_ptr(), iqr.data_ptr(), wins.data_ptr(),
+                                     _stream_ptr(flat.device))
+    self._check(rc, "kb_adjudicate_ragged")
+    return med, iqr, wins
 
 
 @_ctx_method

@@ -295,4 +295,119 @@ __global__ void __launch_bounds__(kWinsThreads) wins_rank_kernel(const WinsRankP
   }
 }
 
+// ---------------------------------------------------------------------------
+// Rows of different lengths: row k = timings[offsets[k] .. offsets[k+1]).
+// ---------------------------------------------------------------------------
+
+// Sort + quartiles per row; a row longer than S_max or empty marks the call invalid.
+__global__ void __launch_bounds__(kRowsThreads) rows_ragged_kernel(
+    const float* __restrict__ timings, const unsigned int* __restrict__ offsets, unsigned int S_max,
+    float* __restrict__ median, float* __restrict__ iqr, float* __restrict__ sorted_out,
+    unsigned int* status) {
+  extern __shared__ float xs[];
+  const unsigned int k = blockIdx.x;
+  const unsigned int o0 = offsets[k], o1 = offsets[k + 1];
+  if (o1 <= o0 || o1 - o0 > S_max) {
+    if (threadIdx.x == 0) set_status(status, (unsigned int)KB_ERR_INVALID_ARG);
+    return;
+  }
+  const unsigned int S = o1 - o0;
+  unsigned int P = 1;
+  while (P < S) P <<= 1;
+  load_and_sort_row(timings + o0, S, P, xs, status);
+  if (sorted_out) {
+    for (unsigned int i = threadIdx.x; i < S; i += kRowsThreads) sorted_out[o0 + i] = xs[i];
+  }
+  if (threadIdx.x == 0) {
+    float q[4];
+#pragma unroll
+    for (unsigned int j = 1; j <= 3; ++j) {
+      const unsigned long long pos = (unsigned long long)j * (S - 1);
+      const unsigned int lo = (unsigned int)(pos >> 2);
+      const unsigned int rem = (unsigned int)(pos & 3ull);
+      const unsigned int hi = (lo + 1 < S) ? lo + 1 : S - 1;
+      if (rem == 0) {
+        q[j] = xs[lo];
+      } else {
+        const float w = (float)rem * 0.25f;
+        q[j] = __fadd_rn(xs[lo], __fmul_rn(w, __fsub_rn(xs[hi], xs[lo])));
+      }
+    }
+    if (median) median[k] = q[2];
+    if (iqr) iqr[k] = __fsub_rn(q[3], q[1]);
+  }
+}
+
+struct WinsRaggedParams {
+  const float* sorted;            // rows ascending, at the offsets of the input
+  const unsigned int* offsets;    // [K+1]
+  unsigned int* wins;
+  unsigned int K, S_max, KB, TA;
+};
+
+// As wins_rank_kernel, with per-row lengths: W[b][a] = sum over a's samples of (lb + ub) in
+// row b, W[a][b] = 2*S_a*S_b - that.
+__global__ void __launch_bounds__(kWinsThreads) wins_ragged_kernel(const WinsRaggedParams p) {
+  extern __shared__ float bs[];   // [8][S_max]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const unsigned int nsub = kWinsRowsPerBlock / p.TA;
+  const unsigned int sub = blockIdx.x % nsub;
+  const unsigned int pair = blockIdx.x / nsub;
+  unsigned int Ab = 0, rem = pair;
+  while (rem >= p.KB - Ab) {
+    rem -= p.KB - Ab;
+    ++Ab;
+  }
+  const unsigned int Bb = Ab + rem;
+  const unsigned int b = Bb * kWinsRowsPerBlock + warp;
+  unsigned int Sb = 0, ob = 0;
+  bool bad = false;
+  if (b < p.K) {
+    ob = p.offsets[b];
+    const unsigned int oe = p.offsets[b + 1];
+    bad = oe <= ob || oe - ob > p.S_max;
+    Sb = bad ? 0u : oe - ob;
+    for (unsigned int i = lane; i < Sb; i += 32) bs[(size_t)warp * p.S_max + i] = p.sorted[ob + i];
+  }
+  __syncthreads();
+  if (b >= p.K || bad) return;
+  const float* brow = bs + (size_t)warp * p.S_max;
+  unsigned int P = 1;
+  while (P <= Sb) P <<= 1;
+  const unsigned int a0 = Ab * kWinsRowsPerBlock + sub * p.TA;
+  for (unsigned int rr = 0; rr < p.TA; ++rr) {
+    const unsigned int a = a0 + rr;
+    if (a >= p.K) break;
+    const unsigned int oa = p.offsets[a], oae = p.offsets[a + 1];
+    if (oae <= oa || oae - oa > p.S_max) continue;
+    const unsigned int Sa = oae - oa;
+    const float* arow = p.sorted + oa;
+    const unsigned int L = (Sa + 31) / 32;
+    const unsigned int i0 = lane * L;
+    const unsigned int i1 = min(i0 + L, Sa);
+    unsigned int sum = 0u;
+    if (i0 < i1) {
+      const float x0 = arow[i0];
+      unsigned int lb = 0u;
+      for (unsigned int step = P >> 1; step > 0; step >>= 1) {
+        const unsigned int nxt = lb + step;
+        if (nxt <= Sb && brow[nxt - 1] < x0) lb = nxt;
+      }
+      unsigned int ub = lb;
+      for (unsigned int i = i0; i < i1; ++i) {
+        const float x = arow[i];
+        while (lb < Sb && brow[lb] < x) ++lb;
+        if (ub < lb) ub = lb;
+        while (ub < Sb && brow[ub] <= x) ++ub;
+        sum += lb + ub;
+      }
+    }
+    sum = warp_add_u32(sum);
+    if (lane == 0) {
+      p.wins[(size_t)a * p.K + b] = 2u * Sa * Sb - sum;
+      if (Ab != Bb) p.wins[(size_t)b * p.K + a] = sum;
+    }
+  }
+}
+
 }  // namespace kb

@@ -254,6 +254,11 @@ extern "C" kb_status kb_ctx_create(int device, kb_ctx** out) {
     fail(ctx, KB_ERR_CUDA, "cannot raise the shared-memory limit of the tail-ratio kernel");
     return bail(KB_ERR_CUDA);
   }
+  if (cudaFuncSetAttribute(wins_ragged_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           kWinsRowsPerBlock * 4096 * (int)sizeof(float)) != cudaSuccess) {
+    fail(ctx, KB_ERR_CUDA, "cannot raise the shared-memory limit of the ragged win-count kernel");
+    return bail(KB_ERR_CUDA);
+  }
   if (cudaFuncSetAttribute(wins_rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            kWinsRowsPerBlock * 4096 * (int)sizeof(float)) != cudaSuccess) {
     fail(ctx, KB_ERR_CUDA, "cannot raise the shared-memory limit of the win-count kernel");
@@ -1026,6 +1031,57 @@ extern "C" kb_status kb_confirm(kb_ctx* ctx, const float* d_first, const float* 
   DeviceGuard g(ctx->device);
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   confirm_kernel<<<(K + 255) / 256, 256, 0, st>>>(d_first, d_second, d_prev, K, threshold, d_status, d_score);
+  ++ctx->launches;
+  KB_CUDA(ctx, cudaGetLastError());
+  return KB_OK;
+}
+
+extern "C" kb_status kb_adjudicate_ragged(kb_ctx* ctx, const float* d_timings,
+                                          const uint32_t* d_offsets, uint32_t K, uint32_t S_max,
+                                          uint64_t total, float* d_median, float* d_iqr,
+                                          uint32_t* d_wins, void* stream) {
+  if (!ctx) return KB_ERR_INVALID_ARG;
+  if (!d_timings || !d_offsets) return fail(ctx, KB_ERR_INVALID_ARG, "kb_adjudicate_ragged: null pointer");
+  if (K == 0 || K > KB_MAX_K) return fail(ctx, KB_ERR_INVALID_ARG, "kb_adjudicate_ragged: K=%u outside [1, %u]", K, KB_MAX_K);
+  if (S_max == 0 || S_max > 4096) return fail(ctx, KB_ERR_INVALID_ARG, "kb_adjudicate_ragged: S_max=%u outside [1, 4096]", S_max);
+  if (total == 0 || total > (uint64_t)K * S_max)
+    return fail(ctx, KB_ERR_INVALID_ARG, "kb_adjudicate_ragged: total sample count outside [1, K*S_max]");
+  DeviceGuard g(ctx->device);
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  float* srt = nullptr;
+  if (d_wins) {
+    size_t have = ctx->srt_bytes;
+    kb_status rc = ensure_buf(ctx, &ctx->srt, &have, (size_t)total * sizeof(float));
+    if (rc != KB_OK) {
+      ctx->srt_bytes = 0;
+      return rc;
+    }
+    ctx->srt_bytes = have;
+    srt = ctx->srt;
+  }
+  unsigned int P = 1;
+  while (P < S_max) P <<= 1;
+  rows_ragged_kernel<<<K, kRowsThreads, (size_t)P * sizeof(float), st>>>(d_timings, d_offsets, S_max, d_median,
+                                                                          d_iqr, srt, ctx->d_status);
+  ++ctx->launches;
+  KB_CUDA(ctx, cudaGetLastError());
+  if (!d_wins) return KB_OK;
+  WinsRaggedParams rp;
+  rp.sorted = srt;
+  rp.offsets = d_offsets;
+  rp.wins = d_wins;
+  rp.K = K;
+  rp.S_max = S_max;
+  rp.KB = (K + kWinsRowsPerBlock - 1) / kWinsRowsPerBlock;
+  const unsigned long long npairs = (unsigned long long)rp.KB * (rp.KB + 1) / 2;
+  rp.TA = kWinsRowsPerBlock;
+  while (npairs * (kWinsRowsPerBlock / rp.TA) < 8ull * ctx->sm_count && rp.TA > 1) rp.TA /= 2;
+  const unsigned long long grid = npairs * (kWinsRowsPerBlock / rp.TA);
+  if (grid > 0x7FFFFFFFull) return fail(ctx, KB_ERR_UNSUPPORTED, "kb_adjudicate_ragged: K too large for one launch");
+  {
+    ScopedTimer tm(ctx, KB_TIMER_WINS, st);
+    wins_ragged_kernel<<<(unsigned int)grid, kWinsThreads, (size_t)kWinsRowsPerBlock * S_max * sizeof(float), st>>>(rp);
+  }
   ++ctx->launches;
   KB_CUDA(ctx, cudaGetLastError());
   return KB_OK;

@@ -618,3 +618,29 @@ def test_two_tier_chain_in_one_cuda_graph(ctx, kb):
         assert g_surv.cpu().numpy().tolist() == want_s
     assert ctx.poll() == 0
     mask.close()
+
+
+@pytest.mark.parametrize("K,smax", [(1, 5), (6, 60), (21, 60), (40, 300), (9, 4096)])
+def test_adjudicate_ragged_matches_oracle(ctx, kb, K, smax):
+    rng = np.random.default_rng(K * 13 + smax)
+    dev = torch.device("cuda", 0)
+    lens = rng.integers(1, smax + 1, K)
+    lens[0] = smax
+    rows = [np.round(rng.lognormal(0, 0.1, int(n)), 2).astype(np.float32) for n in lens]
+    off = np.zeros(K + 1, dtype=np.int32)
+    off[1:] = np.cumsum(lens)
+    flat = torch.from_numpy(np.concatenate(rows)).to(dev)
+    med, iqr, wins = ctx.adjudicate_ragged(flat, torch.from_numpy(off).to(dev), smax)
+    assert ctx.poll() == 0
+    omed, oiqr, owins = oracle.adjudicate_ragged(rows)
+    assert (fbits(med.cpu().numpy()) == fbits(omed)).all()
+    assert (fbits(iqr.cpu().numpy()) == fbits(oiqr)).all()
+    assert (wins.cpu().numpy().view(np.uint32) == owins).all()
+
+
+def test_adjudicate_ragged_flags_a_row_longer_than_the_bound(ctx, kb):
+    dev = torch.device("cuda", 0)
+    flat = torch.ones(30, dtype=torch.float32, device=dev)
+    off = torch.tensor([0, 10, 30], dtype=torch.int32, device=dev)       # second row has 20 > 16
+    ctx.adjudicate_ragged(flat, off, 16)
+    assert ctx.poll() == 1
