@@ -200,6 +200,22 @@ kb_status kb_screen_indexed(kb_ctx* ctx, const void* d_ref, const void* const* d
                             uint32_t Kmax, uint64_t N, kb_dtype dtype, float atol, float rtol,
                             const kb_mask* mask, kb_screen_result* d_out, void* stream);
 
+/* Several shapes in one launch (the fidelity level includes the set of input
+ * shapes, Sec. 3.2): G groups, group g with one reference of h_N[g] elements
+ * and h_K[g] candidates of that size; all of one dtype.  Meant for the
+ * latency-bound regime of many small tensors (e.g. 21 candidates of a 512-,
+ * 1024- and 2048-element output): one kernel launch for everything.
+ *   h_refs   HOST array of G DEVICE pointers.
+ *   h_cands  HOST array of sum(h_K) DEVICE pointers, group after group.
+ *   d_out    DEVICE records in the order of h_cands.
+ * 1 <= G <= 64, sum(h_K) <= 1024, and the tensors together at most 2048
+ * blocks of 4096 elements (sum over candidates of ceil(N_g / 4096)); no mask.
+ * Larger jobs: call kb_screen per group. */
+kb_status kb_screen_multi(kb_ctx* ctx, uint32_t G, const void* const* h_refs,
+                          const void* const* h_cands, const uint32_t* h_K, const uint64_t* h_N,
+                          kb_dtype dtype, float atol, float rtol, kb_screen_result* d_out,
+                          void* stream);
+
 /* ---- the same gate for callers that must not allocate ----------------------
  * (The paper has no counterpart; this entry point exists for integration.)
  *

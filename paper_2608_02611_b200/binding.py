@@ -37,7 +37,7 @@ EXPORTS = [
     "kb_ctx_create", "kb_ctx_destroy", "kb_last_error", "kb_ctx_poll", "kb_ctx_set_grid",
     "kb_ctx_enable_timing", "kb_ctx_read_timer", "kb_ctx_launch_count", "kb_ctx_set_wins_algo", "kb_ctx_set_small_path",
     "kb_mask_create_strided", "kb_mask_create_bitmap", "kb_mask_count", "kb_mask_destroy",
-    "kb_screen", "kb_screen_host", "kb_screen_static", "kb_screen_indexed", "kb_adjudicate", "kb_adjudicate_ragged", "kb_select",
+    "kb_screen", "kb_screen_host", "kb_screen_static", "kb_screen_indexed", "kb_screen_multi", "kb_adjudicate", "kb_adjudicate_ragged", "kb_select",
     "kb_select_by_score", "kb_tail_ratios", "kb_copeland", "kb_confirm",
 ]
 
@@ -82,6 +82,7 @@ def load() -> ctypes.CDLL:
     L.kb_screen.argtypes = [vp, vp, vp, u32, u64, i32, f32, f32, vp, vp, vp]
     L.kb_screen_host.argtypes = [vp, vp, vp, u32, u64, i32, f32, f32, vp, vp, vp]
     L.kb_screen_indexed.argtypes = [vp, vp, vp, u32, vp, vp, u32, u64, i32, f32, f32, vp, vp, vp]
+    L.kb_screen_multi.argtypes = [vp, u32, vp, vp, vp, vp, i32, f32, f32, vp, vp]
     L.kb_screen_static.argtypes = [vp, vp, u32, u64, i32, f32, f32, vp, vp]
     L.kb_adjudicate.argtypes = [vp, vp, u32, u32, vp, vp, vp, vp]
     L.kb_adjudicate_ragged.argtypes = [vp, vp, vp, u32, u32, u64, vp, vp, vp, vp]
@@ -379,6 +380,29 @@ def adjudicate_ragged(self, flat: torch.Tensor, offsets: torch.Tensor, S_max: in
                                      _stream_ptr(flat.device))
     self._check(rc, "kb_adjudicate_ragged")
     return med, iqr, wins
+
+
+@_ctx_method
+def screen_multi(self, groups, atol: float, rtol: float) -> torch.Tensor:
+    """kb_screen_multi: groups = [(ref, [cands...]), ...] of different sizes, one launch.
+    Returns a uint8 CUDA tensor [sum K, 48] in group order."""
+    G = len(groups)
+    refs = (ctypes.c_void_p * G)(*[r.data_ptr() for r, _ in groups])
+    Ks = (ctypes.c_uint32 * G)(*[len(c) for _, c in groups])
+    Ns = (ctypes.c_uint64 * G)(*[r.numel() for r, _ in groups])
+    flat = [c for _, cs in groups for c in cs]
+    for r, cs in groups:
+        for c in cs:
+            if c.dtype != groups[0][0].dtype or c.numel() != r.numel() or not c.is_contiguous():
+                raise KbError(1, "kb_screen_multi", "every tensor of a group must have the group's size "
+                                                    "and the call's dtype")
+    ptrs = (ctypes.c_void_p * max(len(flat), 1))(*[c.data_ptr() for c in flat])
+    dev = groups[0][0].device
+    out = torch.empty((len(flat), RESULT_BYTES), dtype=torch.uint8, device=dev)
+    rc = load().kb_screen_multi(self._h, G, refs, ptrs, Ks, Ns, DTYPE_CODE.get(groups[0][0].dtype, -1),
+                                float(atol), float(rtol), out.data_ptr(), _stream_ptr(dev))
+    self._check(rc, "kb_screen_multi")
+    return out
 
 
 @_ctx_method

@@ -96,7 +96,7 @@ struct DeviceGuard {
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline int elem_bytes(kb_dtype dt) { return dt == KB_F32 ? 4 : 2; }
-constexpr size_t kSmallTicketBytes = 2048;
+constexpr size_t kSmallTicketBytes = 4096;
 constexpr size_t kSmallMaxPartials = 2048;
 constexpr size_t kSmallWsBytes = kSmallTicketBytes + kSmallMaxPartials * sizeof(Acc);
 
@@ -697,6 +697,66 @@ extern "C" kb_status kb_screen_indexed(kb_ctx* ctx, const void* d_ref, const voi
   IndexedSel sel{d_table, K_all, d_index, d_count};
   return screen_dispatch(ctx, d_ref, nullptr, Kmax, N, dtype, atol, rtol, mask, d_out,
                          reinterpret_cast<cudaStream_t>(stream), &sel);
+}
+
+extern "C" kb_status kb_screen_multi(kb_ctx* ctx, uint32_t G, const void* const* h_refs,
+                                     const void* const* h_cands, const uint32_t* h_K,
+                                     const uint64_t* h_N, kb_dtype dtype, float atol, float rtol,
+                                     kb_screen_result* d_out, void* stream) {
+  if (!ctx) return KB_ERR_INVALID_ARG;
+  if (!h_refs || !h_cands || !h_K || !h_N || !d_out)
+    return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen_multi: null pointer");
+  if (G == 0 || G > (uint32_t)kMultiMaxGroups)
+    return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen_multi: G=%u outside [1, %d]", G, kMultiMaxGroups);
+  if (dtype != KB_F32 && dtype != KB_F16 && dtype != KB_BF16)
+    return fail(ctx, KB_ERR_UNSUPPORTED, "kb_screen_multi: unknown dtype %d", (int)dtype);
+  if (!(atol >= 0.0f) || !(rtol >= 0.0f) || std::isinf(atol) || std::isinf(rtol))
+    return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen_multi: atol and rtol must be finite and >= 0");
+  if ((reinterpret_cast<uintptr_t>(d_out) & 7u) != 0)
+    return fail(ctx, KB_ERR_ALIGNMENT, "kb_screen_multi: output not 8-byte aligned");
+  if (!ctx->small_ws) return fail(ctx, KB_ERR_WORKSPACE, "kb_screen_multi: this context has no small-problem workspace");
+  static thread_local MultiParams mp;   // 12 KB: kept off the stack
+  uint32_t rows = 0;
+  uint64_t blocks = 0;
+  for (uint32_t g = 0; g < G; ++g) {
+    if (!h_refs[g] || h_K[g] == 0 || h_N[g] == 0 || h_N[g] > KB_MAX_N)
+      return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen_multi: group %u has a null reference, K = 0 or a bad N", g);
+    if (!aligned16(h_refs[g])) return fail(ctx, KB_ERR_ALIGNMENT, "kb_screen_multi: reference %u not 16-byte aligned", g);
+    mp.ref[g] = h_refs[g];
+    mp.N[g] = h_N[g];
+    const uint64_t nb = (h_N[g] + kSmallPerBlock - 1) / kSmallPerBlock;
+    for (uint32_t k = 0; k < h_K[g]; ++k) {
+      if (rows >= (uint32_t)kMultiMaxRows || blocks + nb > kSmallMaxPartials)
+        return fail(ctx, KB_ERR_UNSUPPORTED,
+                    "kb_screen_multi: more than %d candidates or %zu blocks of 4096 elements; "
+                    "call kb_screen per group", kMultiMaxRows, kSmallMaxPartials);
+      const void* c = h_cands[rows];
+      if (!c) return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen_multi: candidate %u is NULL", rows);
+      if (!aligned16(c)) return fail(ctx, KB_ERR_ALIGNMENT, "kb_screen_multi: candidate %u not 16-byte aligned", rows);
+      mp.cand[rows] = c;
+      mp.group[rows] = (unsigned char)g;
+      mp.first_block[rows] = (unsigned int)blocks;
+      blocks += nb;
+      ++rows;
+    }
+  }
+  mp.first_block[rows] = (unsigned int)blocks;
+  mp.rows = rows;
+  mp.tickets = reinterpret_cast<unsigned int*>(ctx->small_ws);
+  mp.partials = reinterpret_cast<Acc*>(ctx->small_ws + kSmallTicketBytes);
+  mp.out = d_out;
+  mp.atol = atol;
+  mp.rtol = rtol;
+  DeviceGuard gd(ctx->device);
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  switch (dtype) {
+    case KB_F32: screen_multi_kernel<KB_F32><<<(unsigned int)blocks, 256, 0, st>>>(mp); break;
+    case KB_F16: screen_multi_kernel<KB_F16><<<(unsigned int)blocks, 256, 0, st>>>(mp); break;
+    default: screen_multi_kernel<KB_BF16><<<(unsigned int)blocks, 256, 0, st>>>(mp); break;
+  }
+  ++ctx->launches;
+  KB_CUDA(ctx, cudaGetLastError());
+  return KB_OK;
 }
 
 // ---------------------------------------------------------------------------

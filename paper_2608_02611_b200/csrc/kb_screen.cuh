@@ -719,8 +719,15 @@ struct SmallParams {
   MaskDev mask;
 };
 
+// One block's share of a small problem: classify elements [base, base+4096) of one candidate
+// exactly, store the partial record, and -- if this block is the candidate's last to finish --
+// merge the nb partials and write the candidate's result.
 template <int DT>
-__global__ void __launch_bounds__(256) screen_small_kernel(const SmallParams p, const PtrChunk cands) {
+__device__ __forceinline__ void small_block(const void* ref, const void* cand, unsigned long long N,
+                                            unsigned long long base, const MaskDev& mask, float atol,
+                                            float rtol, Acc* partials /*[nb] of this candidate*/,
+                                            unsigned int bx, unsigned int nb, unsigned int* ticket,
+                                            kb_screen_result* out) {
   using E = Elem<DT>;
   __shared__ unsigned int s_cnt[3];
   __shared__ unsigned int s_rel;
@@ -732,14 +739,11 @@ __global__ void __launch_bounds__(256) screen_small_kernel(const SmallParams p, 
     s_key = 0ull;
   }
   __syncthreads();
-  const unsigned int k = blockIdx.y;
-  const void* cand = cands.p[k];
-  const unsigned long long base = (unsigned long long)blockIdx.x * kSmallPerBlock;
   ExactAcc x;
 #pragma unroll 4
   for (unsigned int j = 0; j < kSmallPerBlock / 256; ++j) {
     const unsigned long long i = base + j * 256 + threadIdx.x;
-    if (i < p.N && mask_selected(p.mask, i)) x.add(E::load(p.ref, i), E::load(cand, i), i, p.atol, p.rtol);
+    if (i < N && mask_selected(mask, i)) x.add(E::load(ref, i), E::load(cand, i), i, atol, rtol);
   }
   x.n_mis = warp_add_u32(x.n_mis);
   x.n_nan = warp_add_u32(x.n_nan);
@@ -762,19 +766,19 @@ __global__ void __launch_bounds__(256) screen_small_kernel(const SmallParams p, 
     a.key = s_key;
     a.rel = s_rel;
     a.pad = 0u;
-    p.partials[(size_t)k * p.nb + blockIdx.x] = a;
+    partials[bx] = a;
     __threadfence();
-    s_ticket = atomicAdd(&p.tickets[k], 1u);
+    s_ticket = atomicAdd(ticket, 1u);
   }
   __syncthreads();
-  if (s_ticket != p.nb - 1) return;
+  if (s_ticket != nb - 1) return;
   // last block of this candidate: merge the partial records (warp 0 is enough)
   __threadfence();
   if (threadIdx.x < 32) {
     unsigned long long mism = 0ull, nan = 0ull, inf = 0ull, key = 0ull;
     unsigned int rel = 0u;
-    for (unsigned int b = threadIdx.x; b < p.nb; b += 32) {
-      const Acc* q = &p.partials[(size_t)k * p.nb + b];
+    for (unsigned int b = threadIdx.x; b < nb; b += 32) {
+      const Acc* q = &partials[b];
       mism += __ldcg(&q->mism);
       nan += __ldcg(&q->nan);
       inf += __ldcg(&q->inf);
@@ -783,13 +787,10 @@ __global__ void __launch_bounds__(256) screen_small_kernel(const SmallParams p, 
       const unsigned int rv = __ldcg(&q->rel);
       rel = rv > rel ? rv : rel;
     }
-    // each partial count is < 2^32 and nb <= 1024, so 32-bit halves add without loss below
-    const unsigned long long tm = (unsigned long long)warp_add_u32((unsigned int)mism) +
-                                  ((unsigned long long)warp_add_u32((unsigned int)(mism >> 32)) << 32);
-    const unsigned long long tn = (unsigned long long)warp_add_u32((unsigned int)nan) +
-                                  ((unsigned long long)warp_add_u32((unsigned int)(nan >> 32)) << 32);
-    const unsigned long long ti = (unsigned long long)warp_add_u32((unsigned int)inf) +
-                                  ((unsigned long long)warp_add_u32((unsigned int)(inf >> 32)) << 32);
+    // each partial count is <= 4096 and nb <= 2048: the 32-bit adds below cannot overflow
+    const unsigned long long tm = warp_add_u32((unsigned int)mism);
+    const unsigned long long tn = warp_add_u32((unsigned int)nan);
+    const unsigned long long ti = warp_add_u32((unsigned int)inf);
     key = warp_max_u64(key);
     rel = warp_max_u32(rel);
     if (threadIdx.x == 0) {
@@ -800,10 +801,59 @@ __global__ void __launch_bounds__(256) screen_small_kernel(const SmallParams p, 
       a.key = key;
       a.rel = rel;
       a.pad = 0u;
-      unpack_record(a, &p.out[k]);
-      p.tickets[k] = 0u;   // ready for the next launch
+      unpack_record(a, out);
+      *ticket = 0u;   // ready for the next launch
     }
   }
+}
+
+template <int DT>
+__global__ void __launch_bounds__(256) screen_small_kernel(const SmallParams p, const PtrChunk cands) {
+  const unsigned int k = blockIdx.y;
+  small_block<DT>(p.ref, cands.p[k], p.N, (unsigned long long)blockIdx.x * kSmallPerBlock, p.mask,
+                  p.atol, p.rtol, p.partials + (size_t)k * p.nb, blockIdx.x, p.nb, &p.tickets[k],
+                  &p.out[k]);
+}
+
+// Several (reference, candidates) groups of different sizes in ONE launch (the paper's
+// fidelity includes the set of input shapes, Sec. 3.2): every candidate of every group is a
+// "row"; blocks are numbered row-major over the rows' 4096-element blocks.  Everything the
+// kernel needs travels as kernel arguments.
+constexpr int kMultiMaxGroups = 64;
+constexpr int kMultiMaxRows = 1024;
+struct MultiParams {
+  const void* ref[kMultiMaxGroups];
+  unsigned long long N[kMultiMaxGroups];
+  const void* cand[kMultiMaxRows];
+  unsigned int first_block[kMultiMaxRows + 1];   // prefix sums of the rows' block counts
+  unsigned char group[kMultiMaxRows];
+  Acc* partials;
+  unsigned int* tickets;
+  kb_screen_result* out;
+  unsigned int rows;
+  float atol, rtol;
+};
+
+template <int DT>
+__global__ void __launch_bounds__(256) screen_multi_kernel(const __grid_constant__ MultiParams p) {
+  // row of this block: the last row whose first block is <= blockIdx.x
+  unsigned int lo = 0, hi = p.rows;
+  while (hi - lo > 1) {
+    const unsigned int mid = (lo + hi) >> 1;
+    if (p.first_block[mid] <= blockIdx.x) lo = mid; else hi = mid;
+  }
+  const unsigned int row = lo;
+  const unsigned int g = p.group[row];
+  const unsigned int bx = blockIdx.x - p.first_block[row];
+  const unsigned int nb = p.first_block[row + 1] - p.first_block[row];
+  MaskDev none;
+  none.kind = 0;
+  none.log2_tile = 0;
+  none.stride = 1;
+  none.phase = 0;
+  none.bits = nullptr;
+  small_block<DT>(p.ref[g], p.cand[row], p.N[g], (unsigned long long)bx * kSmallPerBlock, none, p.atol,
+                  p.rtol, p.partials + p.first_block[row], bx, nb, &p.tickets[row], &p.out[row]);
 }
 
 __global__ void screen_finalize_kernel(const Acc* __restrict__ acc, kb_screen_result* __restrict__ out,

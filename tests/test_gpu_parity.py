@@ -644,3 +644,29 @@ def test_adjudicate_ragged_flags_a_row_longer_than_the_bound(ctx, kb):
     off = torch.tensor([0, 10, 30], dtype=torch.int32, device=dev)       # second row has 20 > 16
     ctx.adjudicate_ragged(flat, off, 16)
     assert ctx.poll() == 1
+
+
+@pytest.mark.parametrize("dtype_code", [synth.F32, synth.BF16])
+def test_screen_multi_shapes_in_one_launch(ctx, kb, dtype_code):
+    """Three output shapes of one benchmark (512, 1024, 2048 elements, as the mat-vec sweep of
+    the paper's appendix) plus an awkward one, 21 candidates each, one launch."""
+    rng = np.random.default_rng(7 + dtype_code)
+    dev = torch.device("cuda", 0)
+    groups, want = [], []
+    for N in (512, 1024, 2048, 3 * 4096 + 17):
+        ref = awkward(N, dtype_code, rng, dev)
+        cands = [ref.clone()] + [perturbed(ref, dtype_code, rng, dev) for _ in range(20)]
+        groups.append((ref, cands))
+        want.append(oracle_screen(dtype_code, ref, cands, 1e-2, 1.6e-2))
+    launches0 = ctx.launch_count
+    for _ in range(2):                                    # twice: the tickets reset themselves
+        out = ctx.screen_multi(groups, 1e-2, 1.6e-2)
+        got = kb.records(out)
+        assert_records_equal(got, np.concatenate(want), "multi")
+    assert ctx.launch_count - launches0 == 2
+    assert ctx.poll() == 0
+    # a job that is too large is refused with a pointer to kb_screen
+    big = torch.zeros(4096 * 30, dtype=synth.TORCH_DTYPE[dtype_code], device=dev)
+    with pytest.raises(kb.KbError) as e:
+        ctx.screen_multi([(big, [big] * 100)], 0.0, 0.0)
+    assert e.value.status == 3
