@@ -6,7 +6,8 @@ the benchmark may import this package; the product never does, and this
 package never imports the product.
 
 Inputs are numpy arrays: ``float32`` for fp32 tensors and timings, ``uint16``
-holding the raw bit patterns for fp16 / bf16 tensors.
+holding the raw bit patterns for fp16 / bf16 tensors, ``uint8`` for the two
+8-bit float formats.
 """
 from __future__ import annotations
 
@@ -21,7 +22,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "kb_oracle.c")
 _LIB = os.path.join(_HERE, "libkb_oracle.so")
 
-F32, F16, BF16 = 0, 1, 2
+F32, F16, BF16, F8E4M3, F8E5M2 = 0, 1, 2, 3, 4
 MASK_NONE, MASK_STRIDED, MASK_BITMAP = 0, 1, 2
 
 RESULT_DTYPE = np.dtype(
@@ -91,12 +92,16 @@ def lib() -> ctypes.CDLL:
         L.kbo_decode_f16.restype = f32
         L.kbo_decode_bf16.argtypes = [ctypes.c_uint16]
         L.kbo_decode_bf16.restype = f32
+        L.kbo_decode_f8e4m3.argtypes = [ctypes.c_uint8]
+        L.kbo_decode_f8e4m3.restype = f32
+        L.kbo_decode_f8e5m2.argtypes = [ctypes.c_uint8]
+        L.kbo_decode_f8e5m2.restype = f32
         _lib = L
     return _lib
 
 
 def _tensor(a: np.ndarray, dtype: int) -> np.ndarray:
-    want = np.float32 if dtype == F32 else np.uint16
+    want = np.float32 if dtype == F32 else (np.uint8 if dtype in (F8E4M3, F8E5M2) else np.uint16)
     a = np.ascontiguousarray(a)
     if a.dtype != want:
         raise TypeError(f"dtype code {dtype} needs a {want.__name__} array, got {a.dtype}")

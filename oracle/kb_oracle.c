@@ -38,7 +38,7 @@
 #include <string.h>
 
 /* dtype codes of this oracle's own interface */
-enum { KBO_F32 = 0, KBO_F16 = 1, KBO_BF16 = 2 };
+enum { KBO_F32 = 0, KBO_F16 = 1, KBO_BF16 = 2, KBO_F8E4M3 = 3, KBO_F8E5M2 = 4 };
 
 /* mask kinds */
 enum { KBO_MASK_NONE = 0, KBO_MASK_STRIDED = 1, KBO_MASK_BITMAP = 2 };
@@ -103,10 +103,31 @@ float kbo_decode_f16(uint16_t h) {
 /* bfloat16 -> binary32: the 16 bits are the top half of the binary32 word. */
 float kbo_decode_bf16(uint16_t b) { return bits_to_float((uint32_t)b << 16); }
 
+/* 8-bit float, 4 exponent bits (bias 7), 3 fraction bits, the "fn" flavour: no
+ * infinities, the only NaN is S.1111.111, S.1111.110 is the largest finite (448). */
+float kbo_decode_f8e4m3(uint8_t v) {
+  uint32_t sign = (uint32_t)(v >> 7) & 1u;
+  uint32_t expo = (uint32_t)(v >> 3) & 0xFu;
+  uint32_t frac = (uint32_t)v & 0x7u;
+  float mag;
+  if (expo == 0xFu && frac == 0x7u) return bits_to_float((sign << 31) | 0x7FC00000u);
+  if (expo == 0)
+    mag = ldexpf((float)frac, -9);                      /* subnormal: frac * 2^-3 * 2^-6 */
+  else
+    mag = ldexpf((float)(8u + frac), (int)expo - 10);   /* (1 + frac/8) * 2^(expo-7) */
+  return sign ? -mag : mag;
+}
+
+/* 8-bit float, 5 exponent bits (bias 15), 2 fraction bits, IEEE-like: the top half
+ * of a binary16. */
+float kbo_decode_f8e5m2(uint8_t v) { return kbo_decode_f16((uint16_t)((uint16_t)v << 8)); }
+
 static float load_as_f32(const void* base, uint64_t i, int dtype) {
   if (dtype == KBO_F32) return ((const float*)base)[i];
   if (dtype == KBO_F16) return kbo_decode_f16(((const uint16_t*)base)[i]);
-  return kbo_decode_bf16(((const uint16_t*)base)[i]);
+  if (dtype == KBO_BF16) return kbo_decode_bf16(((const uint16_t*)base)[i]);
+  if (dtype == KBO_F8E4M3) return kbo_decode_f8e4m3(((const uint8_t*)base)[i]);
+  return kbo_decode_f8e5m2(((const uint8_t*)base)[i]);
 }
 
 /* Is element i selected by the fidelity mask?  A mask selects whole tiles of
@@ -142,7 +163,7 @@ int kbo_screen(const void* ref, const void* cand, uint64_t N, int dtype, float a
   float max_abs = 0.0f, max_rel = 0.0f;
   int64_t argmax = -1;
   if (!ref || !cand || !out || N == 0) return -1;
-  if (dtype != KBO_F32 && dtype != KBO_F16 && dtype != KBO_BF16) return -1;
+  if (dtype < KBO_F32 || dtype > KBO_F8E5M2) return -1;
   if (mask_kind == KBO_MASK_STRIDED && (stride == 0 || phase >= stride)) return -1;
   if (mask_kind == KBO_MASK_BITMAP && !bits) return -1;
 

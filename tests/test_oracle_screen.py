@@ -393,3 +393,38 @@ def test_rejects_bad_arguments():
         oracle.screen_one(a.astype(np.float64), a, F32, 0, 0)
     with pytest.raises(ValueError):
         oracle.screen_one(a, a, F32, 0, 0, mask=("strided", 0, 2, 2))
+
+
+# --------------------------------------------------------------------------
+# 8-bit float formats
+# --------------------------------------------------------------------------
+
+def test_fp8_decoders_against_torch():
+    """All 256 patterns of both formats against torch's float8 -> float32 conversion."""
+    pat = torch.arange(256, dtype=torch.uint8)
+    L = oracle.lib()
+    for name, fn in (("float8_e4m3fn", L.kbo_decode_f8e4m3), ("float8_e5m2", L.kbo_decode_f8e5m2)):
+        want = pat.view(getattr(torch, name)).to(torch.float32).numpy().view(np.uint32)
+        for p in range(256):
+            g = struct.unpack("<I", struct.pack("<f", fn(p)))[0]
+            if (want[p] & 0x7FFFFFFF) > 0x7F800000:
+                assert (g & 0x7FFFFFFF) > 0x7F800000, (name, hex(p))
+            else:
+                assert g == want[p], (name, hex(p))
+    assert L.kbo_decode_f8e4m3(0x7E) == 448.0 and L.kbo_decode_f8e5m2(0x7B) == 57344.0
+    assert np.isinf(L.kbo_decode_f8e5m2(0x7C)) and np.isnan(L.kbo_decode_f8e4m3(0xFF))
+
+
+@pytest.mark.parametrize("code,name", [(oracle.F8E4M3, "float8_e4m3fn"), (oracle.F8E5M2, "float8_e5m2")])
+def test_fp8_screen_equals_fp32_screen_of_the_decoded_values(code, name):
+    """Decoding is exact, so screening fp8 tensors must equal screening their fp32 images."""
+    rng = np.random.default_rng(code)
+    r8 = rng.integers(0, 256, 5000).astype(np.uint8)
+    c8 = r8.copy()
+    flip = rng.random(5000) < 0.3
+    c8[flip] = (c8[flip].astype(np.int32) + rng.integers(-2, 3, flip.sum())).astype(np.uint8)
+    to32 = lambda a: torch.from_numpy(a).view(getattr(torch, name)).to(torch.float32).numpy()
+    got = oracle.screen_one(r8, c8, code, 1e-2, 6e-2)
+    want = oracle.screen_one(to32(r8), to32(c8), F32, 1e-2, 6e-2)
+    assert got == want
+    assert got["nan_count"] > 0 and got["mismatch_count"] > 0
