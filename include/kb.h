@@ -62,7 +62,13 @@ typedef enum {
   KB_ERR_DEVICE_TIMEOUT = 7 /* device status: a bounded device-side wait ran out  */
 } kb_status;
 
-typedef enum { KB_F32 = 0, KB_F16 = 1, KB_BF16 = 2 } kb_dtype;
+typedef enum {
+  KB_F32 = 0,
+  KB_F16 = 1,
+  KB_BF16 = 2,
+  KB_F8E4M3 = 3, /* 8-bit float, 4 exponent / 3 fraction bits, "fn": no Inf, one NaN (S.1111.111) */
+  KB_F8E5M2 = 4  /* 8-bit float, 5 exponent / 2 fraction bits, IEEE-like                         */
+} kb_dtype;
 
 /* One record per candidate; 48 bytes, 8-byte aligned.
  * With r = ref[i], c = cand[i] decoded exactly to binary32 and, over the

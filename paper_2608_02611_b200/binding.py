@@ -21,10 +21,11 @@ STATUS_NAMES = {
     0: "KB_OK", 1: "KB_ERR_INVALID_ARG", 2: "KB_ERR_ALIGNMENT", 3: "KB_ERR_UNSUPPORTED",
     4: "KB_ERR_WORKSPACE", 5: "KB_ERR_CUDA", 6: "KB_ERR_NONFINITE", 7: "KB_ERR_DEVICE_TIMEOUT",
 }
-KB_F32, KB_F16, KB_BF16 = 0, 1, 2
+KB_F32, KB_F16, KB_BF16, KB_F8E4M3, KB_F8E5M2 = 0, 1, 2, 3, 4
 KB_SELECT_ERR_THEN_TIME, KB_SELECT_TIME = 0, 1
 KB_TIMER_SCREEN_STREAM, KB_TIMER_WINS = 0, 1
-DTYPE_CODE = {torch.float32: KB_F32, torch.float16: KB_F16, torch.bfloat16: KB_BF16}
+DTYPE_CODE = {torch.float32: KB_F32, torch.float16: KB_F16, torch.bfloat16: KB_BF16,
+              torch.float8_e4m3fn: KB_F8E4M3, torch.float8_e5m2: KB_F8E5M2}
 
 # kb_screen_result as a numpy record (48 bytes)
 RESULT_DTYPE = np.dtype([

@@ -100,6 +100,45 @@ template <> struct Elem<KB_F16> {
   }
 };
 
+// The two 8-bit formats: 16 elements per 16-byte vector.  Pairs of bytes are widened to
+// f16x2 by one hardware conversion (exact: every fp8 value is an fp16 value), then the
+// mixed-precision subtract does the rest.
+template <bool E5M2> struct ElemF8 {
+  static constexpr int kBytes = 1;
+  static constexpr int kVec = 16;
+  __device__ __forceinline__ static unsigned int widen2(unsigned short pr) {
+    unsigned int h2;
+    if (E5M2)
+      asm("cvt.rn.f16x2.e5m2x2 %0, %1;" : "=r"(h2) : "h"(pr));
+    else
+      asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"(pr));
+    return h2;
+  }
+  __device__ __forceinline__ static void decode(const uint4& w, float* out) {
+    const unsigned int* u = reinterpret_cast<const unsigned int*>(&w);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const unsigned int h2 = widen2((unsigned short)(u[i >> 1] >> (16 * (i & 1))));
+      const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&h2));
+      out[2 * i] = f.x;
+      out[2 * i + 1] = f.y;
+    }
+  }
+  __device__ __forceinline__ static float load(const void* p, unsigned long long i) {
+    const unsigned int h2 = widen2((unsigned short)reinterpret_cast<const unsigned char*>(p)[i]);
+    return __low2float(*reinterpret_cast<const __half2*>(&h2));
+  }
+  __device__ __forceinline__ static void pair_diff(const unsigned int* words, int e, float r0, float r1,
+                                                   float& d0, float& d1) {
+    const unsigned int h2 = widen2((unsigned short)(words[e >> 2] >> (16 * ((e >> 1) & 1))));
+    asm("{\n.reg .b16 lo, hi;\nmov.b32 {lo, hi}, %2;\nsub.rn.f32.f16 %0, lo, %3;\nsub.rn.f32.f16 %1, hi, %4;\n}"
+        : "=f"(d0), "=f"(d1)
+        : "r"(h2), "f"(r0), "f"(r1));
+  }
+};
+template <> struct Elem<KB_F8E4M3> : ElemF8<false> {};
+template <> struct Elem<KB_F8E5M2> : ElemF8<true> {};
+
 // ---- the gate on one element, written out (used by every slow path) --------
 // tol_c = min(atol + rtol*|r|, FLT_MAX): then  |c-r| <= tol_c  <=>  d finite and d <= tol.
 __device__ __forceinline__ float tol_clamped(float r, float atol, float rtol) {

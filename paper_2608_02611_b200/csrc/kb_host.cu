@@ -95,7 +95,8 @@ struct DeviceGuard {
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
-inline int elem_bytes(kb_dtype dt) { return dt == KB_F32 ? 4 : 2; }
+inline int elem_bytes(kb_dtype dt) { return dt == KB_F32 ? 4 : (dt == KB_F8E4M3 || dt == KB_F8E5M2) ? 1 : 2; }
+inline bool known_dtype(int dt) { return dt >= KB_F32 && dt <= KB_F8E5M2; }
 constexpr size_t kSmallTicketBytes = 4096;
 constexpr size_t kSmallMaxPartials = 2048;
 constexpr size_t kSmallWsBytes = kSmallTicketBytes + kSmallMaxPartials * sizeof(Acc);
@@ -146,10 +147,13 @@ kb_status ensure_buf(kb_ctx* ctx, T** buf, size_t* have, size_t need) {
   return KB_OK;
 }
 
+// ring depth by stage size: 3 CTAs/SM must fit ~75 KB each
+inline uint32_t stream_stages(uint32_t tile_bytes) { return tile_bytes >= 16384 ? 3 : tile_bytes >= 8192 ? 7 : 10; }
+
 template <int DT>
 kb_status launch_stream(kb_ctx* ctx, StreamParams& sp, cudaStream_t st) {
   const uint32_t tile_bytes = kTile * Elem<DT>::kBytes;
-  sp.stages = (tile_bytes == 8192) ? 7 : 3;
+  sp.stages = stream_stages(tile_bytes);
   const size_t smem = stream_smem_bytes(sp.stages, tile_bytes);
   const unsigned long long nitems = (unsigned long long)sp.nchunks * sp.ntiles;
   unsigned long long grid = ctx->forced_grid ? ctx->forced_grid : 3ull * ctx->sm_count;
@@ -182,7 +186,7 @@ kb_status launch_generic(kb_ctx* ctx, const void* ref, const void* const* tab, A
 template <int DT>
 kb_status set_stream_attr(kb_ctx* ctx) {
   const uint32_t tile_bytes = kTile * Elem<DT>::kBytes;
-  const size_t smem = stream_smem_bytes(tile_bytes == 8192 ? 7 : 3, tile_bytes);
+  const size_t smem = stream_smem_bytes(stream_stages(tile_bytes), tile_bytes);
   KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT>,
                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT>,
@@ -244,6 +248,8 @@ extern "C" kb_status kb_ctx_create(int device, kb_ctx** out) {
   if ((st = set_stream_attr<KB_F32>(ctx)) != KB_OK) return bail(st);
   if ((st = set_stream_attr<KB_F16>(ctx)) != KB_OK) return bail(st);
   if ((st = set_stream_attr<KB_BF16>(ctx)) != KB_OK) return bail(st);
+  if ((st = set_stream_attr<KB_F8E4M3>(ctx)) != KB_OK) return bail(st);
+  if ((st = set_stream_attr<KB_F8E5M2>(ctx)) != KB_OK) return bail(st);
   if (cudaFuncSetAttribute(rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)(KB_MAX_S * sizeof(float))) != cudaSuccess) {
     fail(ctx, KB_ERR_CUDA, "cannot raise the shared-memory limit of the row kernel");
@@ -497,7 +503,7 @@ kb_status validate_screen(kb_ctx* ctx, const void* ref, const void* const* cands
   if (!ref || !cands || !out) return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen: null pointer");
   if (K == 0 || K > KB_MAX_K) return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen: K=%u outside [1, %u]", K, KB_MAX_K);
   if (N == 0 || N > KB_MAX_N) return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen: N outside [1, 2^32]");
-  if (dtype != KB_F32 && dtype != KB_F16 && dtype != KB_BF16)
+  if (!known_dtype((int)dtype))
     return fail(ctx, KB_ERR_UNSUPPORTED, "kb_screen: unknown dtype %d", (int)dtype);
   if (!(atol >= 0.0f) || !(rtol >= 0.0f) || std::isinf(atol) || std::isinf(rtol))
     return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen: atol and rtol must be finite and >= 0");
@@ -657,6 +663,8 @@ kb_status screen_dispatch(kb_ctx* ctx, const void* d_ref, const void* const* h_c
   switch (dtype) {
     case KB_F32: return screen_impl<KB_F32>(ctx, d_ref, h_cands, K, N, atol, rtol, mask, d_out, st, sel);
     case KB_F16: return screen_impl<KB_F16>(ctx, d_ref, h_cands, K, N, atol, rtol, mask, d_out, st, sel);
+    case KB_F8E4M3: return screen_impl<KB_F8E4M3>(ctx, d_ref, h_cands, K, N, atol, rtol, mask, d_out, st, sel);
+    case KB_F8E5M2: return screen_impl<KB_F8E5M2>(ctx, d_ref, h_cands, K, N, atol, rtol, mask, d_out, st, sel);
     default: return screen_impl<KB_BF16>(ctx, d_ref, h_cands, K, N, atol, rtol, mask, d_out, st, sel);
   }
 }
@@ -684,7 +692,7 @@ extern "C" kb_status kb_screen_indexed(kb_ctx* ctx, const void* d_ref, const voi
   if (Kmax == 0 || Kmax > 1024) return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen_indexed: Kmax=%u outside [1, 1024]", Kmax);
   if (K_all == 0) return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen_indexed: K_all is 0");
   if (N == 0 || N > KB_MAX_N) return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen_indexed: N outside [1, 2^32]");
-  if (dtype != KB_F32 && dtype != KB_F16 && dtype != KB_BF16)
+  if (!known_dtype((int)dtype))
     return fail(ctx, KB_ERR_UNSUPPORTED, "kb_screen_indexed: unknown dtype %d", (int)dtype);
   if (!(atol >= 0.0f) || !(rtol >= 0.0f) || std::isinf(atol) || std::isinf(rtol))
     return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen_indexed: atol and rtol must be finite and >= 0");
@@ -708,7 +716,7 @@ extern "C" kb_status kb_screen_multi(kb_ctx* ctx, uint32_t G, const void* const*
     return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen_multi: null pointer");
   if (G == 0 || G > (uint32_t)kMultiMaxGroups)
     return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen_multi: G=%u outside [1, %d]", G, kMultiMaxGroups);
-  if (dtype != KB_F32 && dtype != KB_F16 && dtype != KB_BF16)
+  if (!known_dtype((int)dtype))
     return fail(ctx, KB_ERR_UNSUPPORTED, "kb_screen_multi: unknown dtype %d", (int)dtype);
   if (!(atol >= 0.0f) || !(rtol >= 0.0f) || std::isinf(atol) || std::isinf(rtol))
     return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen_multi: atol and rtol must be finite and >= 0");
@@ -752,6 +760,8 @@ extern "C" kb_status kb_screen_multi(kb_ctx* ctx, uint32_t G, const void* const*
   switch (dtype) {
     case KB_F32: screen_multi_kernel<KB_F32><<<(unsigned int)blocks, 256, 0, st>>>(mp); break;
     case KB_F16: screen_multi_kernel<KB_F16><<<(unsigned int)blocks, 256, 0, st>>>(mp); break;
+    case KB_F8E4M3: screen_multi_kernel<KB_F8E4M3><<<(unsigned int)blocks, 256, 0, st>>>(mp); break;
+    case KB_F8E5M2: screen_multi_kernel<KB_F8E5M2><<<(unsigned int)blocks, 256, 0, st>>>(mp); break;
     default: screen_multi_kernel<KB_BF16><<<(unsigned int)blocks, 256, 0, st>>>(mp); break;
   }
   ++ctx->launches;
@@ -798,6 +808,8 @@ kb_status static_setup(int device, kb_ctx** out) {
     if ((st = set_stream_attr<KB_F32>(ctx)) != KB_OK) return st;
     if ((st = set_stream_attr<KB_F16>(ctx)) != KB_OK) return st;
     if ((st = set_stream_attr<KB_BF16>(ctx)) != KB_OK) return st;
+    if ((st = set_stream_attr<KB_F8E4M3>(ctx)) != KB_OK) return st;
+    if ((st = set_stream_attr<KB_F8E5M2>(ctx)) != KB_OK) return st;
     slot.ready = true;
   }
   *out = &slot.ctx;

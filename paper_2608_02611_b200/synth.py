@@ -28,13 +28,16 @@ import torch
 MASTER_SEED = 260802611
 
 # dtype codes at the C boundary
-F32, F16, BF16 = 0, 1, 2
-TORCH_DTYPE = {F32: torch.float32, F16: torch.float16, BF16: torch.bfloat16}
-ELEM_SIZE = {F32: 4, F16: 2, BF16: 2}
-_INT_VIEW = {F32: torch.int32, F16: torch.int16, BF16: torch.int16}
-_MAG_MASK = {F32: 0x7FFFFFFF, F16: 0x7FFF, BF16: 0x7FFF}
-_INF_MAG = {F32: 0x7F800000, F16: 0x7C00, BF16: 0x7F80}
-_SIGN_BIT = {F32: 0x80000000, F16: 0x8000, BF16: 0x8000}
+F32, F16, BF16, F8E4M3, F8E5M2 = 0, 1, 2, 3, 4
+TORCH_DTYPE = {F32: torch.float32, F16: torch.float16, BF16: torch.bfloat16,
+               F8E4M3: torch.float8_e4m3fn, F8E5M2: torch.float8_e5m2}
+ELEM_SIZE = {F32: 4, F16: 2, BF16: 2, F8E4M3: 1, F8E5M2: 1}
+_INT_VIEW = {F32: torch.int32, F16: torch.int16, BF16: torch.int16, F8E4M3: torch.int8, F8E5M2: torch.int8}
+_MAG_MASK = {F32: 0x7FFFFFFF, F16: 0x7FFF, BF16: 0x7FFF, F8E4M3: 0x7F, F8E5M2: 0x7F}
+# first magnitude pattern that is not a finite number (e4m3fn has no Inf: 0x7F is its NaN)
+_INF_MAG = {F32: 0x7F800000, F16: 0x7C00, BF16: 0x7F80, F8E4M3: 0x7F, F8E5M2: 0x7C}
+_SIGN_BIT = {F32: 0x80000000, F16: 0x8000, BF16: 0x8000, F8E4M3: 0x80, F8E5M2: 0x80}
+_BITS = {F32: 32, F16: 16, BF16: 16, F8E4M3: 8, F8E5M2: 8}
 
 
 # --------------------------------------------------------------------------
@@ -91,14 +94,12 @@ def host_rng(seed: int, stream: int = 0) -> np.random.Generator:
 def _bits(t: torch.Tensor, dtype: int) -> torch.Tensor:
     """int64 tensor holding the unsigned bit pattern of each element."""
     b = t.view(_INT_VIEW[dtype]).to(torch.int64)
-    return b & (0xFFFFFFFF if dtype == F32 else 0xFFFF)
+    return b & ((1 << _BITS[dtype]) - 1)
 
 
 def _from_bits(b: torch.Tensor, dtype: int) -> torch.Tensor:
-    if dtype == F32:
-        b = torch.where(b >= (1 << 31), b - (1 << 32), b).to(torch.int32)
-    else:
-        b = torch.where(b >= (1 << 15), b - (1 << 16), b).to(torch.int16)
+    n = _BITS[dtype]
+    b = torch.where(b >= (1 << (n - 1)), b - (1 << n), b).to(_INT_VIEW[dtype])
     return b.view(TORCH_DTYPE[dtype])
 
 
@@ -147,6 +148,8 @@ def to_oracle_array(t: torch.Tensor, dtype: int) -> np.ndarray:
     t = t.detach().contiguous().cpu().reshape(-1)
     if dtype == F32:
         return t.numpy()
+    if _BITS[dtype] == 8:
+        return t.view(torch.int8).numpy().view(np.uint8)
     return t.view(torch.int16).numpy().view(np.uint16)
 
 

@@ -80,9 +80,13 @@ def perturbed(ref, dtype_code, rng, device, p_flip=0.3, p_big=0.01, p_special=0.
     big = torch.from_numpy(rng.random(n) < p_big)
     c = torch.where(big, (c.float() * 1.5 + 0.25).to(c.dtype), c)
     u = torch.from_numpy(rng.random(n))
-    c = torch.where(u < p_special, torch.full_like(c, float("nan")), c)
-    c = torch.where((u >= p_special) & (u < 2 * p_special), torch.full_like(c, float("inf")), c)
-    c = torch.where((u >= 2 * p_special) & (u < 3 * p_special), torch.full_like(c, float("-inf")), c)
+    bits = synth._bits(c.contiguous(), dtype_code)
+    inf_mag, sign = synth._INF_MAG[dtype_code], synth._SIGN_BIT[dtype_code]
+    nan_pat = inf_mag | 1 if dtype_code != synth.F8E4M3 else inf_mag      # e4m3fn: 0x7F is its NaN
+    bits = torch.where(u < p_special, torch.full_like(bits, nan_pat), bits)
+    bits = torch.where((u >= p_special) & (u < 2 * p_special), torch.full_like(bits, inf_mag), bits)
+    bits = torch.where((u >= 2 * p_special) & (u < 3 * p_special), torch.full_like(bits, sign | inf_mag), bits)
+    c = synth._from_bits(bits, dtype_code)
     return c.contiguous().to(device)
 
 
@@ -200,8 +204,8 @@ def test_config5_small_two_tier(ctx, kb):
 # awkward values, ragged sizes, chunk boundaries, grid independence
 # --------------------------------------------------------------------------
 
-@pytest.mark.parametrize("dtype_code", [synth.F32, synth.F16, synth.BF16])
-@pytest.mark.parametrize("N", [1, 7, 8, 9, 4095, 4096, 4097, 3 * 4096 + 5, 20 * 4096 + 123])
+@pytest.mark.parametrize("dtype_code", [synth.F32, synth.F16, synth.BF16, synth.F8E4M3, synth.F8E5M2])
+@pytest.mark.parametrize("N", [1, 7, 8, 9, 15, 16, 17, 4095, 4096, 4097, 3 * 4096 + 5, 20 * 4096 + 123])
 def test_awkward_values_and_ragged_sizes(ctx, kb, dtype_code, N):
     rng = np.random.default_rng(N * 3 + dtype_code)
     dev = torch.device("cuda", 0)
@@ -646,7 +650,7 @@ def test_adjudicate_ragged_flags_a_row_longer_than_the_bound(ctx, kb):
     assert ctx.poll() == 1
 
 
-@pytest.mark.parametrize("dtype_code", [synth.F32, synth.BF16])
+@pytest.mark.parametrize("dtype_code", [synth.F32, synth.BF16, synth.F8E4M3])
 def test_screen_multi_shapes_in_one_launch(ctx, kb, dtype_code):
     """Three output shapes of one benchmark (512, 1024, 2048 elements, as the mat-vec sweep of
     the paper's appendix) plus an awkward one, 21 candidates each, one launch."""
@@ -666,7 +670,26 @@ def test_screen_multi_shapes_in_one_launch(ctx, kb, dtype_code):
     assert ctx.launch_count - launches0 == 2
     assert ctx.poll() == 0
     # a job that is too large is refused with a pointer to kb_screen
-    big = torch.zeros(4096 * 30, dtype=synth.TORCH_DTYPE[dtype_code], device=dev)
+    big = torch.zeros(4096 * 30, dtype=torch.uint8, device=dev).view(torch.int8).to(torch.float32).to(synth.TORCH_DTYPE[dtype_code]) \
+        if dtype_code == synth.F8E4M3 else torch.zeros(4096 * 30, dtype=synth.TORCH_DTYPE[dtype_code], device=dev)
     with pytest.raises(kb.KbError) as e:
         ctx.screen_multi([(big, [big] * 100)], 0.0, 0.0)
     assert e.value.status == 3
+
+
+@pytest.mark.parametrize("dtype_code", [synth.F8E4M3, synth.F8E5M2])
+def test_fp8_large_with_masks_and_grids(ctx, kb, dtype_code):
+    """8-bit formats through the streaming kernel: many tiles, a ragged tail, a coarse mask."""
+    rng = np.random.default_rng(100 + dtype_code)
+    dev = torch.device("cuda", 0)
+    N = 300 * 4096 + 77
+    ref = awkward(N, dtype_code, rng, dev)
+    cands = [perturbed(ref, dtype_code, rng, dev, p_flip=0.01, p_big=0.0, p_special=0.0) for _ in range(6)]
+    cands += [perturbed(ref, dtype_code, rng, dev), ref.clone()]
+    for mask_spec in (None, ("strided", 12, 4, 1)):
+        want = oracle_screen(dtype_code, ref, cands, 1e-2, 7e-2, mask_spec)
+        for grid in (0, 3):
+            ctx.set_grid(grid)
+            got = run_screen(ctx, kb, ref, cands, 1e-2, 7e-2, mask_spec)
+            ctx.set_grid(0)
+            assert_records_equal(got, want, f"fp8 {dtype_code} mask={mask_spec} grid={grid}")
