@@ -52,28 +52,24 @@ def peaks():
 
 
 class ClockSampler(threading.Thread):
-    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+    """Samples SM clock and throttle reasons through NVML while the timed region runs.
+    Everything that talks to NVML (initialisation included) happens on this daemon thread, so a
+    slow or stuck NVML can never block the benchmark itself."""
 
     def __init__(self, index: int, period_s: float = 0.02):
         super().__init__(daemon=True)
         self.index, self.period = index, period_s
         self.samples, self.reasons, self.max_mhz = [], set(), None
         self._halt = threading.Event()
-        self.ok = False
-        try:
-            import pynvml
-            pynvml.nvmlInit()
-            self.nv = pynvml
-            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
-            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
-            self.ok = True
-        except Exception:
-            self.ok = False
 
     def run(self):
-        if not self.ok:
+        try:
+            import pynvml as nv
+            nv.nvmlInit()
+            h = nv.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = int(nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM))
+        except Exception:
             return
-        nv = self.nv
         names = {
             "hw_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
             "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
@@ -82,8 +78,8 @@ class ClockSampler(threading.Thread):
         }
         while not self._halt.is_set():
             try:
-                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
-                mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(h))
                 for name, bit in names.items():
                     if mask & bit:
                         self.reasons.add(name)
@@ -95,9 +91,10 @@ class ClockSampler(threading.Thread):
         self._halt.set()
         if self.is_alive():
             self.join(timeout=2)
-        return {"sm_mhz": int(np.median(self.samples)) if self.samples else None,
+        samples = list(self.samples)
+        return {"sm_mhz": int(np.median(samples)) if samples else None,
                 "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
-                "samples": len(self.samples)}
+                "samples": len(samples)}
 
 
 def host_cores() -> int:
@@ -334,6 +331,9 @@ def main():
         if world > 1:
             dist.barrier()
             dist.destroy_process_group()
+        torch.cuda.synchronize()
+        ctx_adj.close()
+        ctx.close()
         return
 
     # ---- roofline of the dominant kernel (streaming screen): algorithmic bytes / event time ----
@@ -391,6 +391,8 @@ def main():
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
+    torch.cuda.synchronize()
+    ctx_adj.close()
     ctx.close()
 
 

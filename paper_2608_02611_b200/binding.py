@@ -8,6 +8,7 @@ from __future__ import annotations
 
 import ctypes
 import os
+import sys
 from typing import Optional, Sequence
 
 import numpy as np
@@ -124,7 +125,8 @@ class Mask:
 
     def __del__(self):
         try:
-            self.close()
+            if not sys.is_finalizing():
+                self.close()
         except Exception:
             pass
 
@@ -152,8 +154,11 @@ class Context:
             self._h = None
 
     def __del__(self):
+        # never call into CUDA while the interpreter is shutting down (the runtime may be
+        # half torn down by then); the process is about to release everything anyway
         try:
-            self.close()
+            if not sys.is_finalizing():
+                self.close()
         except Exception:
             pass
 

@@ -468,13 +468,40 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
             const float a0 = fabsf(d0), a1 = fabsf(d1);
             const float tol0 = __fadd_rn(p.atol, __fmul_rn(p.rtol, fabsf(r[e])));
             const float tol1 = __fadd_rn(p.atol, __fmul_rn(p.rtol, fabsf(r[e + 1])));
-            bad |= !(a0 <= tol0) || !(a1 <= tol1);   // an infinite error under an infinite tol is caught by (b)
+            bad |= !(a0 <= tol0) || !(a1 <= tol1);   // also true for NaN / Inf differences
             mabs = max3(mabs, a0, a1);
             mrel = max3_nan(mrel, fmaf(-rel, fabsf(r[e]), a0), fmaf(-rel, fabsf(r[e + 1]), a1));
           }
         }
-        const bool trig = bad || (mabs > th) || !(mrel <= 0.0f) || extreme;
-        if (!__any_sync(0xFFFFFFFFu, trig)) continue;
+        bool trig = (mabs > th) || !(mrel <= 0.0f) || extreme;
+        // Every vote below is reached by all 32 lanes: no warp-synchronous call sits under a
+        // condition that could differ between lanes.
+        if (!__any_sync(0xFFFFFFFFu, trig || bad)) continue;
+        // Threads that saw an element out of tolerance count their finite mismatches here, so
+        // that a failing candidate does not send every step down the exact path; a NaN or Inf
+        // difference still does.
+        unsigned int mis_fast = 0u;
+        if (bad) {
+          bool nonfin = false;
+#pragma unroll
+          for (int e = 0; e < kEPT; e += 2) {
+            float d0, d1;
+            E::pair_diff(words, e, r[e], r[e + 1], d0, d1);
+            const float a0 = fabsf(d0), a1 = fabsf(d1);
+            const float tol0 = __fadd_rn(p.atol, __fmul_rn(p.rtol, fabsf(r[e])));
+            const float tol1 = __fadd_rn(p.atol, __fmul_rn(p.rtol, fabsf(r[e + 1])));
+            const bool f0 = a0 <= kFltMax, f1 = a1 <= kFltMax;
+            nonfin |= !f0 || !f1;
+            mis_fast += ((a0 > tol0) && f0) ? 1u : 0u;   // (c == r would give a0 = 0 <= tol0)
+            mis_fast += ((a1 > tol1) && f1) ? 1u : 0u;
+          }
+          trig = trig || nonfin;
+        }
+        if (!__any_sync(0xFFFFFFFFu, trig)) {
+          const unsigned int tot = warp_add_u32(mis_fast);
+          if (lane == 0 && tot) atomicAdd(&s.cnt[kk], (unsigned long long)tot);
+          continue;
+        }
 
         // ---- exact path.  A triggered thread finds its largest finite error (first
         // index on ties) with a running compare, and evaluates by the definition the
@@ -517,6 +544,7 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
             best = pack_key(m, idx);
           }
         }
+        if (!trig) n_mis = mis_fast;   // lanes that did not take the exact path keep their fast count
         n_mis = warp_add_u32(n_mis);
         n_nan = warp_add_u32(n_nan);
         n_inf = warp_add_u32(n_inf);
