@@ -1,18 +1,26 @@
 // Correctness gate kernels (Sec. 3.1 K(p); Sec. 3.4 Verifier): compare K
 // candidate tensors with one reference.
 //
-// screen_stream_kernel  the bandwidth-bound path.  Persistent CTAs walk work
-//   items (candidate chunk, 4096-element tile) in increasing tile order.  One
-//   producer lane feeds a ring of shared-memory stages with 1-D bulk copies
-//   (TMA, no multicast): first the reference tile, then the same tile of each
-//   candidate of the chunk.  256 consumer threads keep their 16 reference
-//   elements (value and clamped tolerance) in registers for the whole
-//   item and run a branch-free filter over each candidate stage; only warps
-//   whose filter fires take the exact slow path.  Merges are integer adds and
-//   integer maxima on packed keys, so the result does not depend on order.
-// screen_generic_kernel  plain loads, every element classified exactly; used
+// screen_stream_kernel  the bandwidth-bound path.  CTAs draw work items
+//   (candidate chunk, 4096-element tile) from a global counter, in ascending
+//   order.  One producer lane feeds a ring of shared-memory stages with 1-D
+//   bulk copies (TMA, no multicast): first the reference tile, then the same
+//   tile of each candidate of the chunk.  256 consumer threads keep their 16
+//   reference elements in registers for the whole item and run a branch-free
+//   filter over each candidate stage; only warps whose filter fires take the
+//   exact path.  Merges are integer adds and integer maxima on packed keys, so
+//   the result does not depend on order.  The last CTA to finish unpacks the
+//   K records.
+// screen_scout_kernel   classifies a few leading tiles exactly before the
+//   streaming kernel starts; their maxima seed its thresholds.
+// screen_generic_kernel plain loads, every element classified exactly; used
 //   for the ragged tail tile and for masks finer than a kernel tile.
-// screen_finalize_kernel  unpack the accumulators into kb_screen_result.
+// screen_small_kernel / screen_multi_kernel  the latency regime: one launch
+//   for a small problem / for several small problems of different shapes.
+// screen_prep_kernel / screen_prep_indexed_kernel  pointer table, zeroed
+//   accumulators and counters (the indexed form also validates a selection
+//   that lives on the device).
+// screen_finalize_kernel  unpacks the accumulators when no streaming launch did.
 #pragma once
 
 #include "kb_common.cuh"
