@@ -173,15 +173,15 @@ def run_adjudicate(args):
     line = {"workload": f"adjudicate timings[{K}][{S}]", "wins_algo": args.wins_algo,
             "ms_per_call": ms, "wins_kernel_ms": wins_ms,
             "pairwise_comparisons_per_s": logical / (wins_ms * 1e-3), "steps": steps}
-    direct = args.wins_algo == 1 or S > 4096
+    direct = (args.wins_algo == 1 or S > 4096) and K % 8 == 0   # the count below assumes full 8-row blocks
     if direct:
-        # every unordered block pair once; R*32 sample slots per lane row; 3 ALU-pipe
-        # instructions (set.lt, set.le, 3-input add) per 32 sample pairs
+        # every unordered block pair once; R*32 sample slots per lane row; at least the two
+        # compares of a sample pair must issue on the ALU pipe (64 lanes/clk/SM)
         KB = (K + 7) // 8
         nj = (S + 255) // 256
         R = ((S + nj - 1) // nj + 31) // 32
         evals = KB * (KB + 1) // 2 * 64 * S * (nj * R * 32)
-        peak = 148 * 64 * 1.965e9 / 3          # sample-pair evaluations/s at 64 ALU lanes/clk/SM
+        peak = 148 * 64 * 1.965e9 / 2          # sample-pair evaluations/s at 64 ALU lanes/clk/SM
         line["roofline"] = {"bound": "alu", "achieved": evals / (wins_ms * 1e-3), "peak": peak,
                             "unit": "sample-pair evaluations/s", "frac": evals / (wins_ms * 1e-3) / peak,
                             "traffic": None}
