@@ -151,7 +151,7 @@ __device__ __forceinline__ void set_status(unsigned int* status, unsigned int co
   atomicCAS(status, 0u, code);
 }
 
-// ---- mbarrier + bulk copy (TMA, 1-D, no multicast) --------------------------
+// ---- mbarrier + bulk copy (TMA, 1-D, each CTA fetches its own tiles) --------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return (uint32_t)__cvta_generic_to_shared(p);
 }

@@ -4,7 +4,7 @@
 // screen_stream_kernel  the bandwidth-bound path.  CTAs draw work items
 //   (candidate chunk, 4096-element tile) from a global counter, in ascending
 //   order.  One producer lane feeds a ring of shared-memory stages with 1-D
-//   bulk copies (TMA, no multicast): first the reference tile, then the same
+//   bulk copies (TMA, each CTA its own): first the reference tile, then the same
 //   tile of each candidate of the chunk.  256 consumer threads keep their 16
 //   reference elements in registers for the whole item and run a branch-free
 //   filter over each candidate stage; only warps whose filter fires take the
