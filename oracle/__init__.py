@@ -39,6 +39,20 @@ RESULT_DTYPE = np.dtype(
 )
 assert RESULT_DTYPE.itemsize == 48
 
+RESULT_F64_DTYPE = np.dtype(
+    [
+        ("mismatch_count", "<u8"),
+        ("nan_count", "<u8"),
+        ("inf_count", "<u8"),
+        ("argmax_idx", "<i8"),
+        ("max_abs_err", "<f8"),
+        ("max_rel_err", "<f8"),
+        ("pass", "<u4"),
+        ("reserved", "<u4"),
+    ]
+)
+assert RESULT_F64_DTYPE.itemsize == 56
+
 
 class NonFiniteTiming(ValueError):
     """A timing was NaN or +-Inf; the adjudication is undefined."""
@@ -66,6 +80,9 @@ def lib() -> ctypes.CDLL:
         vp = ctypes.c_void_p
         L.kbo_screen.argtypes = [vp, vp, u64, i32, f32, f32, i32, u32, u32, u32, vp, vp]
         L.kbo_screen.restype = i32
+        f64 = ctypes.c_double
+        L.kbo_screen_f64.argtypes = [vp, vp, u64, f64, f64, i32, u32, u32, u32, vp, vp]
+        L.kbo_screen_f64.restype = i32
         L.kbo_quantiles.argtypes = [vp, u32, vp, vp]
         L.kbo_quantiles.restype = i32
         L.kbo_wins_pair.argtypes = [vp, vp, u32]
@@ -155,6 +172,36 @@ def screen(ref: np.ndarray, cands, dtype: int, atol: float, rtol: float, mask=No
     else:
         with ThreadPoolExecutor(max_workers=threads) as ex:
             list(ex.map(work, range(K)))
+    return out
+
+
+def screen_f64(ref: np.ndarray, cands, atol: float, rtol: float, mask=None, threads: int = 1) -> np.ndarray:
+    """Gate every float64 candidate in ``cands`` in binary64; returns K RESULT_F64_DTYPE records."""
+    r = np.ascontiguousarray(ref).reshape(-1)
+    if r.dtype != np.float64:
+        raise TypeError("the double-precision gate needs float64 arrays")
+    K = len(cands)
+    out = np.zeros(K, dtype=RESULT_F64_DTYPE)
+    kind, log2_tile, stride, phase, bits_ptr, keep = _mask_args(mask)
+
+    def work(k):
+        c = np.ascontiguousarray(cands[k]).reshape(-1)
+        if c.dtype != np.float64 or c.size != r.size:
+            raise TypeError("candidates must be float64 arrays of the reference's size")
+        one = np.zeros(1, dtype=RESULT_F64_DTYPE)
+        rc = lib().kbo_screen_f64(r.ctypes.data, c.ctypes.data, r.size, float(atol), float(rtol),
+                                  kind, log2_tile, stride, phase, bits_ptr, one.ctypes.data)
+        if rc != 0:
+            raise ValueError(f"kbo_screen_f64 rejected its arguments (rc={rc})")
+        out[k] = one[0]
+
+    if threads <= 1:
+        for k in range(K):
+            work(k)
+    else:
+        with ThreadPoolExecutor(max_workers=threads) as ex:
+            list(ex.map(work, range(K)))
+    del keep
     return out
 
 

@@ -9,7 +9,8 @@
  *
  * Everything is the definition written out: one loop per definition, in the
  * order the definition states, no blocking, no fusion, no reordering.
- * All floating point is IEEE-754 binary32, round-to-nearest-even.  Build with
+ * All floating point is IEEE-754 binary32, round-to-nearest-even (binary64 in
+ * kbo_screen_f64, the gate for double-precision tensors).  Build with
  *     gcc -O2 -std=c99 -ffp-contract=off -fPIC -shared
  * (no -ffast-math, no FTZ/DAZ) so that no multiply-add is fused and
  * subnormals are honoured.
@@ -197,6 +198,82 @@ int kbo_screen(const void* ref, const void* cand, uint64_t N, int dtype, float a
   out->inf_count = infs;
   out->argmax_idx = have_abs ? argmax : -1;
   out->max_abs_err = have_abs ? max_abs : 0.0f;
+  out->max_rel_err = max_rel;
+  out->pass = (mism == 0) ? 1u : 0u;
+  out->reserved = 0;
+  return 0;
+}
+
+/* ---- the gate for binary64 tensors ---------------------------------------- */
+
+typedef struct {
+  uint64_t mismatch_count;
+  uint64_t nan_count;
+  uint64_t inf_count;
+  int64_t argmax_idx;
+  double max_abs_err;
+  double max_rel_err;
+  uint32_t pass;
+  uint32_t reserved;
+} kbo_screen_result_f64;
+
+static uint64_t double_to_bits(double f) {
+  uint64_t u;
+  memcpy(&u, &f, sizeof u);
+  return u;
+}
+static int is_nan64(double f) { return (double_to_bits(f) & 0x7FFFFFFFFFFFFFFFull) > 0x7FF0000000000000ull; }
+static int is_inf64(double f) { return (double_to_bits(f) & 0x7FFFFFFFFFFFFFFFull) == 0x7FF0000000000000ull; }
+static int is_finite64(double f) { return (double_to_bits(f) & 0x7FFFFFFFFFFFFFFFull) < 0x7FF0000000000000ull; }
+
+/*
+ * The same gate as kbo_screen (Sec. 3.1 K(p); Sec. 3.4 Verifier) for a reference and a
+ * candidate stored in binary64.  The seven steps are those of kbo_screen with every
+ * operation in binary64: a double-precision output is judged in its own precision, and the
+ * record carries the two errors as doubles.
+ */
+int kbo_screen_f64(const double* ref, const double* cand, uint64_t N, double atol, double rtol,
+                   int mask_kind, uint32_t log2_tile, uint32_t stride, uint32_t phase,
+                   const uint64_t* bits, kbo_screen_result_f64* out) {
+  uint64_t i;
+  uint64_t mism = 0, nans = 0, infs = 0;
+  int have_abs = 0;
+  double max_abs = 0.0, max_rel = 0.0;
+  int64_t argmax = -1;
+  if (!ref || !cand || !out || N == 0) return -1;
+  if (mask_kind == KBO_MASK_STRIDED && (stride == 0 || phase >= stride)) return -1;
+  if (mask_kind == KBO_MASK_BITMAP && !bits) return -1;
+
+  for (i = 0; i < N; ++i) {
+    double r, c, d, prod, tol;
+    int match;
+    if (!selected(i, mask_kind, log2_tile, stride, phase, bits)) continue;
+    r = ref[i];
+    c = cand[i];
+    d = fabs(c - r);
+    prod = rtol * fabs(r);
+    tol = atol + prod;
+    match = (c == r) || (is_finite64(d) && d <= tol);
+    if (!match) ++mism;
+    if (is_nan64(c)) ++nans;
+    if (is_inf64(c)) ++infs;
+    if (is_finite64(d)) {
+      if (!have_abs || d > max_abs) {
+        max_abs = d;
+        argmax = (int64_t)i;
+        have_abs = 1;
+      }
+      if (r != 0.0) {
+        double q = d / fabs(r);
+        if (q > max_rel) max_rel = q;
+      }
+    }
+  }
+  out->mismatch_count = mism;
+  out->nan_count = nans;
+  out->inf_count = infs;
+  out->argmax_idx = have_abs ? argmax : -1;
+  out->max_abs_err = have_abs ? max_abs : 0.0;
   out->max_rel_err = max_rel;
   out->pass = (mism == 0) ? 1u : 0u;
   out->reserved = 0;
