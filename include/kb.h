@@ -39,8 +39,8 @@
  *     kb_ctx_poll reads back.
  *   - Determinism: every output is a pure function of the inputs; it does not
  *     depend on grid size, scheduling or call history.
- *   - Arithmetic: IEEE-754 binary32, round-to-nearest-even, no fused
- *     multiply-add, subnormals honoured.
+ *   - Arithmetic: IEEE-754 binary32 (binary64 in kb_screen_f64),
+ *     round-to-nearest-even, no fused multiply-add, subnormals honoured.
  */
 #ifndef KB_H_
 #define KB_H_
@@ -221,6 +221,31 @@ kb_status kb_screen_multi(kb_ctx* ctx, uint32_t G, const void* const* h_refs,
                           const void* const* h_cands, const uint32_t* h_K, const uint64_t* h_N,
                           kb_dtype dtype, float atol, float rtol, kb_screen_result* d_out,
                           void* stream);
+
+/* ---- the gate for double-precision tensors ---------------------------------
+ * The same gate with the reference and the candidates stored in binary64 and
+ * EVERY operation of the record (d, tol, the comparison, d/|r|) in binary64,
+ * round-to-nearest-even, no fused multiply-add: a double-precision output is
+ * judged in its own precision.  56 bytes per record, 8-byte aligned; field
+ * meanings as in kb_screen_result. */
+typedef struct {
+  uint64_t mismatch_count;
+  uint64_t nan_count;
+  uint64_t inf_count;
+  int64_t argmax_idx;
+  double max_abs_err;
+  double max_rel_err;
+  uint32_t pass;
+  uint32_t reserved;
+} kb_screen_result_f64;
+
+/* Arguments as for kb_screen (DEVICE d_ref, HOST array of K DEVICE pointers, all
+ * 16-byte aligned; atol, rtol finite and >= 0; mask NULL or created for the
+ * same N; DEVICE d_out of K records, fully overwritten).  Asynchronous on
+ * `stream`. */
+kb_status kb_screen_f64(kb_ctx* ctx, const double* d_ref, const double* const* h_cands, uint32_t K,
+                        uint64_t N, double atol, double rtol, const kb_mask* mask,
+                        kb_screen_result_f64* d_out, void* stream);
 
 /* ---- the same gate for callers that must not allocate ----------------------
  * (The paper has no counterpart; this entry point exists for integration.)

@@ -34,12 +34,18 @@ RESULT_DTYPE = np.dtype([
     ("max_abs_err", "<f4"), ("max_rel_err", "<f4"), ("pass", "<u4"), ("reserved", "<u4"),
 ])
 RESULT_BYTES = 48
+# kb_screen_result_f64 (56 bytes)
+RESULT_F64_DTYPE = np.dtype([
+    ("mismatch_count", "<u8"), ("nan_count", "<u8"), ("inf_count", "<u8"), ("argmax_idx", "<i8"),
+    ("max_abs_err", "<f8"), ("max_rel_err", "<f8"), ("pass", "<u4"), ("reserved", "<u4"),
+])
+RESULT_F64_BYTES = 56
 
 EXPORTS = [
     "kb_ctx_create", "kb_ctx_destroy", "kb_last_error", "kb_ctx_poll", "kb_ctx_set_grid",
     "kb_ctx_enable_timing", "kb_ctx_read_timer", "kb_ctx_launch_count", "kb_ctx_set_wins_algo", "kb_ctx_set_small_path",
     "kb_mask_create_strided", "kb_mask_create_bitmap", "kb_mask_count", "kb_mask_destroy",
-    "kb_screen", "kb_screen_host", "kb_screen_static", "kb_screen_indexed", "kb_screen_multi", "kb_adjudicate", "kb_adjudicate_ragged", "kb_select",
+    "kb_screen", "kb_screen_f64", "kb_screen_host", "kb_screen_static", "kb_screen_indexed", "kb_screen_multi", "kb_adjudicate", "kb_adjudicate_ragged", "kb_select",
     "kb_select_by_score", "kb_tail_ratios", "kb_copeland", "kb_confirm",
 ]
 
@@ -82,6 +88,7 @@ def load() -> ctypes.CDLL:
     L.kb_mask_count.argtypes = [vp, ctypes.POINTER(u64)]
     L.kb_mask_destroy.argtypes = [vp]
     L.kb_screen.argtypes = [vp, vp, vp, u32, u64, i32, f32, f32, vp, vp, vp]
+    L.kb_screen_f64.argtypes = [vp, vp, vp, u32, u64, ctypes.c_double, ctypes.c_double, vp, vp, vp]
     L.kb_screen_host.argtypes = [vp, vp, vp, u32, u64, i32, f32, f32, vp, vp, vp]
     L.kb_screen_indexed.argtypes = [vp, vp, vp, u32, vp, vp, u32, u64, i32, f32, f32, vp, vp, vp]
     L.kb_screen_multi.argtypes = [vp, u32, vp, vp, vp, vp, i32, f32, f32, vp, vp]
@@ -232,6 +239,24 @@ class Context:
                               mask._h if mask is not None else None, out.data_ptr(),
                               _stream_ptr(ref.device))
         self._check(rc, "kb_screen")
+        return out
+
+    def screen_f64(self, ref: torch.Tensor, cands: Sequence[torch.Tensor], atol: float, rtol: float,
+                   mask: Optional[Mask] = None) -> torch.Tensor:
+        """kb_screen_f64 on float64 CUDA tensors.  Returns a uint8 CUDA tensor [K, 56] of
+        kb_screen_result_f64 records (see ``records_f64``); asynchronous on the current stream."""
+        K = len(cands)
+        N = ref.numel()
+        for c in list(cands) + [ref]:
+            if c.dtype != torch.float64 or c.numel() != N or not c.is_cuda or not c.is_contiguous():
+                raise KbError(1, "kb_screen_f64", "tensors must be contiguous CUDA float64 tensors of "
+                                                  "one element count")
+        out = torch.empty((K, RESULT_F64_BYTES), dtype=torch.uint8, device=ref.device)
+        ptrs = (ctypes.c_void_p * max(K, 1))(*[c.data_ptr() for c in cands])
+        rc = load().kb_screen_f64(self._h, ref.data_ptr(), ptrs, K, N, float(atol), float(rtol),
+                                  mask._h if mask is not None else None, out.data_ptr(),
+                                  _stream_ptr(ref.device))
+        self._check(rc, "kb_screen_f64")
         return out
 
     def screen_host(self, ref: torch.Tensor, cands: Sequence[torch.Tensor], atol: float,
@@ -422,6 +447,11 @@ def confirm(self, first: torch.Tensor, second: torch.Tensor, prev: torch.Tensor,
                            _stream_ptr(first.device))
     self._check(rc, "kb_confirm")
     return status, score
+
+
+def records_f64(screen_out: torch.Tensor) -> np.ndarray:
+    """Copy a [K, 56] uint8 result tensor of kb_screen_f64 to the host as K numpy records."""
+    return screen_out.cpu().numpy().view(RESULT_F64_DTYPE).reshape(-1)
 
 
 def records(screen_out: torch.Tensor) -> np.ndarray:

@@ -12,6 +12,7 @@
 #include "kb_adjudicate.cuh"
 #include "kb_common.cuh"
 #include "kb_screen.cuh"
+#include "kb_screen64.cuh"
 #include "kb_select.cuh"
 
 using namespace kb;
@@ -118,8 +119,8 @@ struct ScopedTimer {
   }
 };
 
-kb_status ensure_ws(kb_ctx* ctx, uint32_t K) {
-  const size_t need = round_up((size_t)K * sizeof(Acc), 256) + (size_t)K * sizeof(void*);
+kb_status ensure_ws(kb_ctx* ctx, uint32_t K, size_t acc_bytes = sizeof(Acc)) {
+  const size_t need = round_up((size_t)K * acc_bytes, 256) + (size_t)K * sizeof(void*);
   if (need <= ctx->ws_bytes) return KB_OK;
   if (ctx->ws) cudaFree(ctx->ws);   // waits for enqueued work that still uses it
   ctx->ws = nullptr;
@@ -195,6 +196,15 @@ kb_status set_stream_attr(kb_ctx* ctx) {
   return KB_OK;
 }
 
+constexpr uint32_t kStages64 = 6;
+kb_status set_stream64_attr(kb_ctx* ctx) {
+  KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)stream64_smem_bytes(kStages64)));
+  KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream64_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                    (int)cudaSharedmemCarveoutMaxShared));
+  return KB_OK;
+}
+
 template <int R>
 void launch_wins(const WinsParams& wp, unsigned int grid, size_t smem, cudaStream_t st) {
   wins_kernel<R><<<grid, kWinsThreads, smem, st>>>(wp);
@@ -250,6 +260,7 @@ extern "C" kb_status kb_ctx_create(int device, kb_ctx** out) {
   if ((st = set_stream_attr<KB_BF16>(ctx)) != KB_OK) return bail(st);
   if ((st = set_stream_attr<KB_F8E4M3>(ctx)) != KB_OK) return bail(st);
   if ((st = set_stream_attr<KB_F8E5M2>(ctx)) != KB_OK) return bail(st);
+  if ((st = set_stream64_attr(ctx)) != KB_OK) return bail(st);
   if (cudaFuncSetAttribute(rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)(KB_MAX_S * sizeof(float))) != cudaSuccess) {
     fail(ctx, KB_ERR_CUDA, "cannot raise the shared-memory limit of the row kernel");
@@ -679,6 +690,122 @@ extern "C" kb_status kb_screen(kb_ctx* ctx, const void* d_ref, const void* const
   DeviceGuard g(ctx->device);
   return screen_dispatch(ctx, d_ref, h_cands, K, N, dtype, atol, rtol, mask, d_out,
                          reinterpret_cast<cudaStream_t>(stream));
+}
+
+// ---------------------------------------------------------------------------
+// kb_screen_f64: the gate in binary64
+// ---------------------------------------------------------------------------
+extern "C" kb_status kb_screen_f64(kb_ctx* ctx, const double* d_ref, const double* const* h_cands,
+                                   uint32_t K, uint64_t N, double atol, double rtol,
+                                   const kb_mask* mask, kb_screen_result_f64* d_out, void* stream) {
+  if (!ctx) return KB_ERR_INVALID_ARG;
+  if (!d_ref || !h_cands || !d_out) return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen_f64: null pointer");
+  if (K == 0 || K > KB_MAX_K) return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen_f64: K=%u outside [1, %u]", K, KB_MAX_K);
+  if (N == 0 || N > KB_MAX_N) return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen_f64: N outside [1, 2^32]");
+  if (!(atol >= 0.0) || !(rtol >= 0.0) || std::isinf(atol) || std::isinf(rtol))
+    return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen_f64: atol and rtol must be finite and >= 0");
+  if (mask && (mask->N != N || mask->ctx != ctx))
+    return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen_f64: the mask was created for another N or context");
+  if (!aligned16(d_ref)) return fail(ctx, KB_ERR_ALIGNMENT, "kb_screen_f64: reference not 16-byte aligned");
+  if ((reinterpret_cast<uintptr_t>(d_out) & 7u) != 0)
+    return fail(ctx, KB_ERR_ALIGNMENT, "kb_screen_f64: output not 8-byte aligned");
+  for (uint32_t k = 0; k < K; ++k) {
+    if (!h_cands[k]) return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen_f64: candidate %u is NULL", k);
+    if (!aligned16(h_cands[k]))
+      return fail(ctx, KB_ERR_ALIGNMENT, "kb_screen_f64: candidate %u not 16-byte aligned", k);
+  }
+  DeviceGuard g(ctx->device);
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  kb_status rc = ensure_ws(ctx, K, sizeof(Acc64));
+  if (rc != KB_OK) return rc;
+  Acc64* acc = reinterpret_cast<Acc64*>(ctx->ws);
+  const void** table = reinterpret_cast<const void**>(ctx->ws + round_up((size_t)K * sizeof(Acc64), 256));
+  for (uint32_t off = 0; off < K; off += kPtrsPerLaunch) {
+    PtrChunk ch;
+    const uint32_t cnt = (K - off < (uint32_t)kPtrsPerLaunch) ? K - off : (uint32_t)kPtrsPerLaunch;
+    memcpy(ch.p, h_cands + off, cnt * sizeof(void*));
+    screen_prep64_kernel<<<(cnt + 127) / 128, 128, 0, st>>>(ch, table, acc, ctx->d_status + 1, off, cnt);
+    ++ctx->launches;
+    KB_CUDA(ctx, cudaGetLastError());
+  }
+  MaskDev md;
+  md.kind = mask ? mask->kind : 0;
+  md.log2_tile = mask ? mask->log2_tile : 0;
+  md.stride = mask ? mask->stride : 1;
+  md.phase = mask ? mask->phase : 0;
+  md.bits = mask ? mask->d_bits : nullptr;
+  auto generic = [&](uint64_t e0, uint64_t e1) -> kb_status {
+    if (e1 <= e0) return KB_OK;
+    uint64_t bx = (e1 - e0 + 255) / 256;
+    const uint64_t cap = (uint64_t)ctx->sm_count * 8;
+    if (bx > cap) bx = cap;
+    dim3 grid((unsigned int)bx, K);
+    screen_generic64_kernel<<<grid, 256, 0, st>>>(d_ref, table, acc, e0, e1, atol, rtol, md);
+    ++ctx->launches;
+    KB_CUDA(ctx, cudaGetLastError());
+    return KB_OK;
+  };
+  if (mask && !mask->coarse) {
+    if ((rc = generic(0, N)) != KB_OK) return rc;
+  } else {
+    const uint64_t nfull = N / kTile;
+    uint32_t ntiles = mask ? mask->n_tiles : (uint32_t)nfull;
+    const uint32_t* tile_list = mask ? mask->d_tiles : nullptr;
+    uint32_t nscout = 0;
+    if (ntiles >= 2) {
+      nscout = ntiles / 128;
+      if (nscout < 1) nscout = 1;
+      if (nscout > 8) nscout = 8;
+      dim3 sg(nscout * 4, K);
+      screen_scout64_kernel<<<sg, 256, 0, st>>>(d_ref, table, acc, tile_list, atol, rtol);
+      ++ctx->launches;
+      KB_CUDA(ctx, cudaGetLastError());
+    }
+    if ((rc = generic(nfull * kTile, N)) != KB_OK) return rc;
+    ntiles -= nscout;
+    if (ntiles) {
+      Stream64Params sp;
+      sp.ref = d_ref;
+      sp.cands = table;
+      sp.acc = acc;
+      sp.tile_list = tile_list;
+      sp.nhalf = 2 * ntiles;
+      sp.half0 = 2 * nscout;
+      sp.K = K;
+      uint32_t nchunks = (K + kMaxKC64 - 1) / kMaxKC64;
+      const uint64_t grid_want = ctx->forced_grid ? ctx->forced_grid : 2ull * ctx->sm_count;
+      const uint64_t want_items = 8 * grid_want;
+      if ((uint64_t)nchunks * sp.nhalf < want_items) {
+        uint64_t nc = (want_items + sp.nhalf - 1) / sp.nhalf;
+        const uint64_t max_nc = (K + 7) / 8;
+        if (nc > max_nc) nc = max_nc;
+        if (nc > nchunks) nchunks = (uint32_t)nc;
+      }
+      sp.KC = (K + nchunks - 1) / nchunks;
+      sp.nchunks = (K + sp.KC - 1) / sp.KC;
+      sp.stages = kStages64;
+      sp.atol = atol;
+      sp.rtol = rtol;
+      sp.status = ctx->d_status;
+      sp.done = ctx->d_status + 1;
+      sp.sched = reinterpret_cast<unsigned long long*>(ctx->d_status + 2);
+      sp.out = d_out;
+      const unsigned long long nitems = (unsigned long long)sp.nchunks * sp.nhalf;
+      unsigned long long grid = grid_want;
+      if (grid > nitems) grid = nitems;
+      {
+        ScopedTimer tm(ctx, KB_TIMER_SCREEN_STREAM, st);
+        screen_stream64_kernel<<<(unsigned int)grid, kStreamThreads, stream64_smem_bytes(kStages64), st>>>(sp);
+      }
+      ++ctx->launches;
+      KB_CUDA(ctx, cudaGetLastError());
+      return KB_OK;
+    }
+  }
+  screen_finalize64_kernel<<<(K + 127) / 128, 128, 0, st>>>(acc, d_out, K);
+  ++ctx->launches;
+  KB_CUDA(ctx, cudaGetLastError());
+  return KB_OK;
 }
 
 extern "C" kb_status kb_screen_indexed(kb_ctx* ctx, const void* d_ref, const void* const* d_table,
