@@ -15,15 +15,18 @@ namespace kb {
 // so a larger key is a larger |c - r| and, at equal error, a lower index;
 // 0 means "no finite difference seen".  rel: integer max of the bits of a
 // non-negative float (monotone, +Inf included).
-struct Acc {
+struct alignas(16) Acc {
   unsigned long long mism;
   unsigned long long nan;
   unsigned long long inf;
+  unsigned long long spare;
+  // the two maxima share one aligned 16-byte block, so that one asynchronous 16-byte copy
+  // brings both into shared memory
   unsigned long long key;
   unsigned int rel;
   unsigned int pad;
 };
-static_assert(sizeof(Acc) == 40, "Acc layout");
+static_assert(sizeof(Acc) == 48, "Acc layout");
 
 __device__ __forceinline__ unsigned long long pack_key(float d, unsigned long long idx) {
   return (((unsigned long long)__float_as_uint(d) << 32) |
@@ -229,6 +232,15 @@ __device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src_gmem, u
       "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar)), "l"(policy)
       : "memory");
 }
+
+// 16-byte asynchronous copy global -> shared that bypasses L1 (the source is updated by other
+// CTAs' atomics) and needs no register for the data.
+__device__ __forceinline__ void cp_async16(void* dst_smem, const void* src_gmem) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst_smem)), "l"(src_gmem)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 
 __device__ __forceinline__ unsigned int warp_max_u32(unsigned int v) {
   return __reduce_max_sync(0xFFFFFFFFu, v);

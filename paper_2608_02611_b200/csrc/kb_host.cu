@@ -20,7 +20,7 @@ using namespace kb;
 struct kb_ctx {
   int device = 0;
   int sm_count = 0;
-  unsigned char* ws = nullptr;      // [acc K*40 | pad | pointer table K*8]
+  unsigned char* ws = nullptr;      // [acc K*48 | pad | pointer table K*8]
   size_t ws_bytes = 0;
   unsigned int* d_status = nullptr;
   uint32_t forced_grid = 0;

@@ -124,10 +124,12 @@ __device__ __forceinline__ float max2_nan(float a, float b) {
 // Shared-memory carve-up (dynamic): stage buffers first (128-byte aligned).
 struct StreamSmem {
   unsigned char* buf;
+  uint4* xg;                 // [kMaxKC] landing slots of the global (key, rel) blocks (exchange)
   uint64_t* full;
   uint64_t* empty;
   uint64_t* sync_bar;        // consumer-wide barrier with a bounded wait (flush)
-  unsigned long long* item_id;   // [stages] work item whose reference tile a stage holds
+  unsigned long long* item_id;   // [stages] (chunk << 32 | position) of the work item whose reference
+                                 // tile a stage holds; all ones: no more work
   unsigned long long* cnt;   // [3][kMaxKC] mism, nan, inf
   unsigned long long* key;   // [kMaxKC]
   const void** ptrs;         // [kMaxKC] candidate pointers of the current chunk (producer only)
@@ -139,6 +141,7 @@ struct StreamSmem {
 
 __host__ __device__ inline size_t stream_smem_bytes(uint32_t stages, uint32_t tile_bytes) {
   size_t b = (size_t)stages * tile_bytes;
+  b += (size_t)kMaxKC * 16;
   b += 3 * (size_t)stages * 8 + 8;
   b += 3 * (size_t)kMaxKC * 8 + (size_t)kMaxKC * 8 + (size_t)kMaxKC * 8 + (size_t)kMaxKC * 4;
   b += (size_t)kMaxKC * kWarps * 8;
@@ -174,6 +177,8 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
     unsigned char* q = reinterpret_cast<unsigned char*>(base);
     s.buf = q;
     q += (size_t)p.stages * TILE_BYTES;
+    s.xg = reinterpret_cast<uint4*>(q);
+    q += (size_t)kMaxKC * 16;
     s.full = reinterpret_cast<uint64_t*>(q);
     q += (size_t)p.stages * 8;
     s.empty = reinterpret_cast<uint64_t*>(q);
@@ -260,7 +265,8 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
             ok = false;
             break;
           }
-          if (kk < 0) s.item_id[stage] = item;   // visible to the consumers with the phase
+          // (chunk, position in the visit order), visible to the consumers with the phase
+          if (kk < 0) s.item_id[stage] = ((unsigned long long)chunk << 32) | (unsigned long long)(slot - p.slot0);
           const unsigned char* src =
               reinterpret_cast<const unsigned char*>(kk < 0 ? p.ref : s.ptrs[kk]) + off;
           mbar_arrive_expect_tx(&s.full[stage], TILE_BYTES);
@@ -339,37 +345,45 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
 
     // Exchange of running maxima with the other CTAs.  Every merge is a maximum, so the
     // exchange needs no ordering: lane (warp, lane) owns candidate warp + 8*lane of the
-    // chunk, pushes this CTA's maxima with atomicMax and gets everyone's back.  The values
-    // that come back are applied one tile later (the round trip to L2 is then hidden),
-    // except on a chunk's first tile, where the scout's seeds are wanted at once.
+    // chunk, pushes this CTA's maxima with atomicMax (no return value) and fetches the
+    // global (key, rel) block with an asynchronous copy into shared memory.  What comes
+    // back is applied one tile later (the round trip to L2 is then hidden and no register
+    // waits for it), except on a chunk's first tile, where the scout's seeds are wanted at once.
     const int xkk = warp + kWarps * lane;
-    unsigned long long xmine_k = 0ull, xold_k = 0ull;
-    unsigned int xmine_r = 0u, xold_r = 0u;
     bool xpending = false;
     auto exchange_issue = [&]() {
       if (xkk < cur_kc) {
-        xmine_k = *reinterpret_cast<volatile unsigned long long*>(&s.key[xkk]);
-        xmine_r = *reinterpret_cast<volatile unsigned int*>(&s.rel[xkk]);
+        const unsigned long long mk = *reinterpret_cast<volatile unsigned long long*>(&s.key[xkk]);
+        const unsigned int mr = *reinterpret_cast<volatile unsigned int*>(&s.rel[xkk]);
         Acc* a = &p.acc[cur_k0 + xkk];
-        xold_k = atomicMax(&a->key, xmine_k);
-        xold_r = atomicMax(&a->rel, xmine_r);
+        if (mk) atomicMax(&a->key, mk);
+        if (mr) atomicMax(&a->rel, mr);
+        cp_async16(&s.xg[xkk], &a->key);
       }
+      cp_async_commit();
     };
-    auto exchange_apply = [&](unsigned long long tile_base) {
+    // `safe_base`: every element any warp of this CTA may still look at has an index >= it
+    // (warps drift apart by less than the ring depth, i.e. by less than one work item).
+    auto exchange_apply = [&](unsigned long long safe_base) {
+      cp_async_wait_all();
       if (xkk < cur_kc) {
+        const volatile uint4* slot = &s.xg[xkk];
+        const unsigned long long gk0 = ((unsigned long long)slot->y << 32) | slot->x;
+        const unsigned int gr = slot->z;
+        const unsigned long long mk = *reinterpret_cast<volatile unsigned long long*>(&s.key[xkk]);
         int* row = reinterpret_cast<int*>(&s.thr2[xkk * kWarps]);
-        if (xold_r > xmine_r) {
-          atomicMax(&s.rel[xkk], xold_r);
+        if (gr > *reinterpret_cast<volatile unsigned int*>(&s.rel[xkk])) {
+          atomicMax(&s.rel[xkk], gr);
 #pragma unroll
-          for (int w2 = 0; w2 < kWarps; ++w2) atomicMax(row + 2 * w2 + 1, (int)xold_r);
+          for (int w2 = 0; w2 < kWarps; ++w2) atomicMax(row + 2 * w2 + 1, (int)gr);
         }
-        const unsigned long long gk = xold_k > xmine_k ? xold_k : xmine_k;
+        const unsigned long long gk = gk0 > mk ? gk0 : mk;
         if (gk != 0ull) {
           // An error equal to one recorded at a lower index, or strictly below one
           // recorded anywhere, can never become the maximum.
           const unsigned int db = (unsigned int)((gk - 1ull) >> 32);
           const unsigned long long gidx = 0xFFFFFFFFull - ((gk - 1ull) & 0xFFFFFFFFull);
-          const int lim = gidx < tile_base ? (int)db : (int)db - 1;   // db == 0: -1 is below every float >= -1
+          const int lim = gidx < safe_base ? (int)db : (int)db - 1;   // db == 0: -1 is below every float >= -1
           if (lim >= 0) {
 #pragma unroll
             for (int w2 = 0; w2 < kWarps; ++w2) atomicMax(row + 2 * w2, lim);
@@ -378,6 +392,7 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
       }
       __syncwarp();
     };
+    uint32_t prev_tile = 0;
 
     for (;;) {
       // the next stage holds a reference tile and names its work item (or the end)
@@ -387,8 +402,8 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
       }
       const unsigned long long item = *reinterpret_cast<volatile unsigned long long*>(&s.item_id[stage]);
       if (item == kNoItem) break;
-      const uint32_t chunk = (uint32_t)(item / p.ntiles);
-      const uint32_t slot = p.slot0 + (uint32_t)(item % p.ntiles);
+      const uint32_t chunk = (uint32_t)(item >> 32);
+      const uint32_t slot = p.slot0 + (uint32_t)item;
       const uint32_t tile = p.tile_list ? p.tile_list[slot] : slot;
       const bool first_of_chunk = (int)chunk != cur_chunk;
       if (first_of_chunk) {
@@ -403,7 +418,13 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
       }
       const unsigned long long tile_base = (unsigned long long)tile * kTile;
 
-      if (xpending) exchange_apply(tile_base);
+      // Not all warps are in this item yet: the slowest may still be up to (ring depth - 1)
+      // stages back, inside the previous item if items are at least that long, so only what
+      // lies below the previous item's tile is "earlier" for everyone.  (On a chunk's first
+      // item the flush barrier has just lined the warps up.)
+      if (xpending)
+        exchange_apply((uint32_t)cur_kc + 1u >= stages ? (unsigned long long)prev_tile * kTile : 0ull);
+      prev_tile = tile;
       exchange_issue();
       xpending = !first_of_chunk;
 
@@ -425,10 +446,8 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
 #pragma unroll
         for (int j = 0; j < NV; ++j) E::decode(w[j], &r[j * VEC]);
 #pragma unroll
-        for (int e = 0; e < kEPT; ++e) {
-          const float ar = fabsf(r[e]);
-          extreme |= (ar > 0.0f && ar < 7.888609052e-31f);
-        }
+        for (int e = 0; e < kEPT; ++e)   // 0 < |r| < 2^-100 on the bit pattern (zero wraps to the top)
+          extreme |= ((__float_as_uint(r[e]) & 0x7FFFFFFFu) - 1u) < (0x0D800000u - 1u);
       }
       if (first_of_chunk) exchange_apply(tile_base);
 
@@ -802,6 +821,7 @@ __device__ __forceinline__ void small_block(const void* ref, const void* cand, u
     a.key = s_key;
     a.rel = s_rel;
     a.pad = 0u;
+    a.spare = 0ull;
     partials[bx] = a;
     __threadfence();
     s_ticket = atomicAdd(ticket, 1u);
@@ -837,6 +857,7 @@ __device__ __forceinline__ void small_block(const void* ref, const void* cand, u
       a.key = key;
       a.rel = rel;
       a.pad = 0u;
+      a.spare = 0ull;
       unpack_record(a, out);
       *ticket = 0u;   // ready for the next launch
     }
@@ -909,7 +930,7 @@ __global__ void screen_prep_kernel(const PtrChunk chunk, const void** table, Acc
   if (i < count) {
     table[offset + i] = chunk.p[i];
     Acc z;
-    z.mism = z.nan = z.inf = z.key = 0ull;
+    z.mism = z.nan = z.inf = z.spare = z.key = 0ull;
     z.rel = z.pad = 0u;
     acc[offset + i] = z;
   }
@@ -949,7 +970,7 @@ __global__ void screen_prep_indexed_kernel(const void* const* __restrict__ all, 
     }
     table[j] = ptr;
     Acc z;
-    z.mism = z.nan = z.inf = z.key = 0ull;
+    z.mism = z.nan = z.inf = z.spare = z.key = 0ull;
     z.rel = z.pad = 0u;
     acc[j] = z;
   }

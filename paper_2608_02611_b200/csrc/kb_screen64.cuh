@@ -387,6 +387,7 @@ __global__ void __maxnreg__(112) screen_stream64_kernel(const Stream64Params p) 
     const int xkk = warp + kWarps * lane;
     unsigned long long xk = 0ull, xl = 0ull, xr = 0ull, xr_applied = 0ull;
     long long xlim_applied = -1ll;
+    unsigned long long prev_base = 0ull;
     auto exchange_issue = [&]() {
       if (xkk < cur_kc) {
         Acc64* a = &p.acc[cur_k0 + xkk];
@@ -398,7 +399,8 @@ __global__ void __maxnreg__(112) screen_stream64_kernel(const Stream64Params p) 
         xr = *reinterpret_cast<const volatile unsigned long long*>(&a->rel);
       }
     };
-    auto exchange_apply = [&](unsigned long long elem_base) {
+    // `safe_base`: every element any warp of this CTA may still look at has an index >= it.
+    auto exchange_apply = [&](unsigned long long safe_base) {
       if (xkk < cur_kc) {
         long long* row = &s.thr[(size_t)xkk * kWarps * 2];
         if (xr > xr_applied) {
@@ -409,7 +411,7 @@ __global__ void __maxnreg__(112) screen_stream64_kernel(const Stream64Params p) 
         if (xk != 0ull) {
           const long long db = (long long)(xk - 1ull);
           const unsigned long long gidx = 0xFFFFFFFFull - xl;
-          const long long lim = gidx < elem_base ? db : db - 1;
+          const long long lim = gidx < safe_base ? db : db - 1;
           if (lim > xlim_applied) {
             xlim_applied = lim;
 #pragma unroll
@@ -445,7 +447,12 @@ __global__ void __maxnreg__(112) screen_stream64_kernel(const Stream64Params p) 
       const unsigned long long elem_base =
           (unsigned long long)tile * kTile + (unsigned long long)(slot & 1u) * kTile64;
 
-      if (!first_of_chunk) exchange_apply(elem_base);
+      // The slowest warp may still be up to (ring depth - 1) stages back, inside the previous
+      // item if items are at least that long: only what lies below the previous item's
+      // elements is "earlier" for every warp.  (On a chunk's first item the flush barrier has
+      // just lined the warps up.)
+      if (!first_of_chunk) exchange_apply((uint32_t)cur_kc + 1u >= stages ? prev_base : 0ull);
+      prev_base = elem_base;
       exchange_issue();
 
       // ---- reference stage: 8 elements per thread stay in registers ----
