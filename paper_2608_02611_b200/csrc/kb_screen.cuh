@@ -220,6 +220,7 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
     s.cnt[2 * kMaxKC + i] = 0ull;
     s.key[i] = 0ull;
     s.rel[i] = 0u;
+    s.xg[i] = make_uint4(0u, 0u, 0u, 0u);
   }
   for (int i = tid; i < kMaxKC * kWarps; i += kStreamThreads) s.thr2[i] = make_float2(-1.0f, 0.0f);
   __syncthreads();
@@ -339,6 +340,7 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
         s.key[i] = 0ull;
         s.rel[i] = 0u;
       }
+      for (int i = tid; i < kMaxKC; i += kConsumers) s.xg[i] = make_uint4(0u, 0u, 0u, 0u);
       for (int i = tid; i < kMaxKC * kWarps; i += kConsumers) s.thr2[i] = make_float2(-1.0f, 0.0f);
       return consumers_barrier();
     };
@@ -356,8 +358,12 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
         const unsigned long long mk = *reinterpret_cast<volatile unsigned long long*>(&s.key[xkk]);
         const unsigned int mr = *reinterpret_cast<volatile unsigned int*>(&s.rel[xkk]);
         Acc* a = &p.acc[cur_k0 + xkk];
-        if (mk) atomicMax(&a->key, mk);
-        if (mr) atomicMax(&a->rel, mr);
+        // push only what exceeds the last fetched global values (maxima only grow): once the
+        // maxima have settled nobody writes, and the accumulator's line is only read
+        const volatile uint4* slot = &s.xg[xkk];
+        const unsigned long long seen_k = ((unsigned long long)slot->y << 32) | slot->x;
+        if (mk > seen_k) atomicMax(&a->key, mk);
+        if (mr > slot->z) atomicMax(&a->rel, mr);
         cp_async16(&s.xg[xkk], &a->key);
       }
       cp_async_commit();
