@@ -324,6 +324,7 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
     };
     // Move the chunk's shared-memory accumulators to global memory and reset them.
     auto flush = [&]() -> bool {
+      cp_async_wait_all();   // this thread's last fetch has landed before the slots are cleared
       if (!consumers_barrier()) return false;
       for (int i = tid; i < cur_kc; i += kConsumers) {
         Acc* a = &p.acc[cur_k0 + i];
