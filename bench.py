@@ -189,6 +189,60 @@ def run_adjudicate(args):
     ctx.close()
 
 
+def run_screen(args):
+    """One kb_screen / kb_screen_f64 call on a seeded synthetic batch: a standard-normal
+    reference and K candidates that differ from it by one unit in the last place on a fraction
+    of the elements (two kernels that round differently).  Secondary measurement: the streaming
+    kernel's bytes/s against the measured HBM peak, for other dtypes and batch sizes than the
+    benchmark line's."""
+    import torch
+    from paper_2608_02611_b200 import binding
+    dev = torch.device("cuda", 0)
+    ctx = binding.Context(0)
+    ctx.set_small_path(False)
+    K, N = args.K, 1 << args.log2n
+    tdt = {"f64": torch.float64, "f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16}[args.dtype]
+    idt = {8: torch.int64, 4: torch.int32, 2: torch.int16}[torch.empty(0, dtype=tdt).element_size()]
+    g = torch.Generator(device=dev)
+    g.manual_seed(20260802)
+    ref = torch.randn(N, dtype=torch.float32, device=dev, generator=g).to(tdt)
+    cands = []
+    for _ in range(K):
+        flip = torch.rand(N, device=dev, generator=g) < args.flip_frac
+        cands.append(torch.where(flip, (ref.view(idt) + 1).view(tdt), ref))
+    atol, rtol = (1e-12, 1e-12) if args.dtype == "f64" else (1e-2, 1.6e-2)
+    call = (lambda: ctx.screen_f64(ref, cands, atol, rtol)) if args.dtype == "f64" else \
+        (lambda: ctx.screen(ref, cands, atol, rtol))
+    steps, warmup = max(1, min(args.steps, 50)), max(3, args.warmup)
+    for _ in range(warmup):
+        call()
+    torch.cuda.synchronize()
+    ctx.enable_timing(True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        call()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    k_ms = float(np.mean(ctx.read_timer(binding.KB_TIMER_SCREEN_STREAM)))
+    assert ctx.poll() == 0
+    ntiles = N // 4096
+    nscout = min(8, max(1, ntiles // 128)) if ntiles >= 2 else 0
+    esz = ref.element_size()
+    stream_bytes = (K + 1) * (ntiles - nscout) * 4096 * esz
+    peak, src = peaks()
+    line = {"workload": f"screen K={K} N=2^{args.log2n} {args.dtype}, one-ulp differences on "
+                        f"{args.flip_frac:.0%} of the elements",
+            "ms_per_call": ms, "stream_kernel_ms": k_ms, "steps": steps,
+            "call_gbs": (K + 1) * N * esz / (ms * 1e-3) / 1e9,
+            "roofline": {"bound": "hbm", "achieved": stream_bytes / (k_ms * 1e-3) / 1e9, "peak": peak,
+                         "unit": "GB/s", "frac": stream_bytes / (k_ms * 1e-3) / 1e9 / peak,
+                         "traffic": None, "peak_source": src}}
+    print(json.dumps(line), flush=True)
+    ctx.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -197,10 +251,14 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--workload", default="step", choices=["step", "adjudicate"],
+    ap.add_argument("--workload", default="step", choices=["step", "adjudicate", "screen"],
                     help="'adjudicate' times kb_adjudicate alone on timings[K][S] (config 5 tier 1 by "
                          "default) and reports pairwise comparisons/s against the ALU roofline; it is a "
                          "secondary measurement, not the benchmark line")
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "f16", "f32", "f64"],
+                    help="storage type of the 'screen' workload")
+    ap.add_argument("--log2n", type=int, default=24, help="elements per tensor of the 'screen' workload")
+    ap.add_argument("--flip-frac", type=float, default=0.25)
     ap.add_argument("--K", type=int, default=512)
     ap.add_argument("--S", type=int, default=200)
     ap.add_argument("--wins-algo", type=int, default=0, choices=[0, 1, 2])
@@ -212,6 +270,8 @@ def main():
         return run_reference(args)
     if args.workload == "adjudicate":
         return run_adjudicate(args)
+    if args.workload == "screen":
+        return run_screen(args)
 
     import torch
     import torch.distributed as dist

@@ -196,7 +196,7 @@ kb_status set_stream_attr(kb_ctx* ctx) {
   return KB_OK;
 }
 
-constexpr uint32_t kStages64 = 6;
+constexpr uint32_t kStages64 = 12;
 kb_status set_stream64_attr(kb_ctx* ctx) {
   KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     (int)stream64_smem_bytes(kStages64)));
@@ -773,7 +773,7 @@ extern "C" kb_status kb_screen_f64(kb_ctx* ctx, const double* d_ref, const doubl
       sp.half0 = 2 * nscout;
       sp.K = K;
       uint32_t nchunks = (K + kMaxKC64 - 1) / kMaxKC64;
-      const uint64_t grid_want = ctx->forced_grid ? ctx->forced_grid : 2ull * ctx->sm_count;
+      const uint64_t grid_want = ctx->forced_grid ? ctx->forced_grid : 1ull * ctx->sm_count;
       const uint64_t want_items = 8 * grid_want;
       if ((uint64_t)nchunks * sp.nhalf < want_items) {
         uint64_t nc = (want_items + sp.nhalf - 1) / sp.nhalf;

@@ -227,7 +227,7 @@ constexpr long long kThNone = (long long)0xBFF0000000000000ull;   // bits of -1.
 //   ad <= th,   ad - rel*|r| <= 0 (one fused multiply-add: its single rounding keeps the
 //   sign, so ad/|r| cannot round above rel),   ad <= atol + rtol*|r|,
 // and no NaN is involved (every comparison is written so that a NaN fires).
-__global__ void __maxnreg__(112) screen_stream64_kernel(const Stream64Params p) {
+__global__ void __maxnreg__(160) screen_stream64_kernel(const Stream64Params p) {
   extern __shared__ unsigned char smem_raw[];
   Stream64Smem s;
   {
