@@ -159,8 +159,9 @@ __host__ __device__ inline size_t stream_smem_bytes(uint32_t stages, uint32_t ti
 //   (a) ad <= atol + rtol*|r|              (match)
 // and no NaN is involved.  (c) is one fused multiply-add, whose single rounding
 // keeps the sign; a NaN-propagating max carries any NaN (a NaN or Inf candidate,
-// Inf - Inf) to the decision.  While rel <= rtol*(1-2^-20), (c) implies (a) and
-// the "lean" form drops the tolerance test: ad <= rel*|r| <= RN(rtol*|r|) <= tol.
+// Inf - Inf) to the decision.  While rel <= rtol*(1-2^-20), (c) implies (a):
+// ad <= rel*|r| <= RN(rtol*|r|) <= tol ("lean").  Beyond that the same loop runs with rel
+// clamped to that bound, and only threads for which it fails compare element by element.
 template <int DT>
 __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
   using E = Elem<DT>;
@@ -480,34 +481,29 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
         }
         const unsigned int* words = reinterpret_cast<const unsigned int*>(w);
 
-        bool bad = false;
-        float mabs = 0.0f, mrel = 0.0f;
+        // One loop for every case: (b) on the largest error, (c) with rel_f = min(rel, rtol_lean).
+        //   rel <= rtol_lean ("lean"): rel_f = rel; (c) implies (a).
+        //   rel  > rtol_lean: (c) with the smaller rel_f still implies both (a) and the real (c);
+        //     a thread for which it fails looks again element by element below (it holds an
+        //     element whose relative error exceeds rtol: a mismatch, or one that passes by atol).
+        //   no lean bound (rtol < 2^-20): rel_f = rel, and (a) is pre-tested per thread on the
+        //     largest error against atol alone.
+        const bool has_lean = p.rtol_lean >= 0.0f;
         const bool lean = rel <= p.rtol_lean;
-        if (lean) {
-          // lean filter: (b) and (c); (a) is implied
+        const float rel_f = (has_lean && !lean) ? p.rtol_lean : rel;
+        float mabs = 0.0f, mrel = 0.0f;
 #pragma unroll
-          for (int e = 0; e < kEPT; e += 2) {
-            float d0, d1;
-            E::pair_diff(words, e, r[e], r[e + 1], d0, d1);
-            const float t0 = fmaf(-rel, fabsf(r[e]), fabsf(d0));
-            const float t1 = fmaf(-rel, fabsf(r[e + 1]), fabsf(d1));
-            mabs = max3(mabs, fabsf(d0), fabsf(d1));
-            mrel = max3_nan(mrel, t0, t1);
-          }
-        } else {
-#pragma unroll
-          for (int e = 0; e < kEPT; e += 2) {
-            float d0, d1;
-            E::pair_diff(words, e, r[e], r[e + 1], d0, d1);
-            const float a0 = fabsf(d0), a1 = fabsf(d1);
-            const float tol0 = __fadd_rn(p.atol, __fmul_rn(p.rtol, fabsf(r[e])));
-            const float tol1 = __fadd_rn(p.atol, __fmul_rn(p.rtol, fabsf(r[e + 1])));
-            bad |= !(a0 <= tol0) || !(a1 <= tol1);   // also true for NaN / Inf differences
-            mabs = max3(mabs, a0, a1);
-            mrel = max3_nan(mrel, fmaf(-rel, fabsf(r[e]), a0), fmaf(-rel, fabsf(r[e + 1]), a1));
-          }
+        for (int e = 0; e < kEPT; e += 2) {
+          float d0, d1;
+          E::pair_diff(words, e, r[e], r[e + 1], d0, d1);
+          const float t0 = fmaf(-rel_f, fabsf(r[e]), fabsf(d0));
+          const float t1 = fmaf(-rel_f, fabsf(r[e + 1]), fabsf(d1));
+          mabs = max3(mabs, fabsf(d0), fabsf(d1));
+          mrel = max3_nan(mrel, t0, t1);
         }
-        bool trig = (mabs > th) || !(mrel <= 0.0f) || extreme;
+        const bool fire_c = !(mrel <= 0.0f);
+        const bool bad = has_lean ? (!lean && fire_c) : (mabs > p.atol);
+        bool trig = (mabs > th) || extreme || (fire_c && (lean || !has_lean));
         // Every vote below is reached by all 32 lanes: no warp-synchronous call sits under a
         // condition that could differ between lanes.
         if (!__any_sync(0xFFFFFFFFu, trig || bad)) continue;
@@ -516,7 +512,7 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
         // difference still does.
         unsigned int mis_fast = 0u;
         if (bad) {
-          bool nonfin = false;
+          bool again = false;   // a NaN or Inf difference, or the real (c) fails
 #pragma unroll
           for (int e = 0; e < kEPT; e += 2) {
             float d0, d1;
@@ -525,11 +521,12 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
             const float tol0 = __fadd_rn(p.atol, __fmul_rn(p.rtol, fabsf(r[e])));
             const float tol1 = __fadd_rn(p.atol, __fmul_rn(p.rtol, fabsf(r[e + 1])));
             const bool f0 = a0 <= kFltMax, f1 = a1 <= kFltMax;
-            nonfin |= !f0 || !f1;
+            again |= !f0 || !f1;
+            again |= !(fmaf(-rel, fabsf(r[e]), a0) <= 0.0f) || !(fmaf(-rel, fabsf(r[e + 1]), a1) <= 0.0f);
             mis_fast += ((a0 > tol0) && f0) ? 1u : 0u;   // (c == r would give a0 = 0 <= tol0)
             mis_fast += ((a1 > tol1) && f1) ? 1u : 0u;
           }
-          trig = trig || nonfin;
+          trig = trig || again;
         }
         if (!__any_sync(0xFFFFFFFFu, trig)) {
           const unsigned int tot = warp_add_u32(mis_fast);
