@@ -218,6 +218,29 @@ def test_awkward_values_and_ragged_sizes(ctx, kb, dtype_code, N):
         assert_records_equal(got, want, f"N={N} dtype={dtype_code} tol=({atol},{rtol})")
 
 
+@pytest.mark.parametrize("dtype_code", [synth.F32, synth.F16, synth.BF16])
+@pytest.mark.parametrize("atol,rtol", [(1e-3, 0.0), (0.0, 1e-2), (1e-2, 1e-7), (0.0, 3e-3), (1e30, 0.0),
+                                       (1e-4, 5e-4), (0.0, 1.0), (6e-8, 9.5367431640625e-07)])
+def test_tolerance_regimes_on_dense_small_differences(ctx, kb, dtype_code, atol, rtol):
+    """Differences of a unit or two in the last place on a third of the elements, values near zero
+    included (their relative error is large, so they pass by atol or not at all): relative error
+    below, around and above rtol; rtol too small for the filter's shortcut; atol only; rtol only."""
+    rng = np.random.default_rng(int(atol * 1e9) + int(rtol * 1e9) + dtype_code)
+    dev = torch.device("cuda", 0)
+    N = 48 * 4096 + 77
+    x = rng.standard_normal(N) * np.exp(2 * rng.standard_normal(N))
+    x[rng.random(N) < 0.05] *= 1e-6
+    x[rng.random(N) < 0.01] = 0.0
+    ref = torch.from_numpy(x).to(synth.TORCH_DTYPE[dtype_code]).to(dev)
+    cands = [perturbed(ref, dtype_code, rng, dev, p_flip=0.33, p_big=0.0, p_special=0.0) for _ in range(5)]
+    cands.append(perturbed(ref, dtype_code, rng, dev, p_flip=0.33, p_big=0.001, p_special=0.0))
+    cands.append(perturbed(ref, dtype_code, rng, dev, p_flip=0.33, p_big=0.0, p_special=0.0005))
+    cands.append(ref.clone())
+    got = run_screen(ctx, kb, ref, cands, atol, rtol)
+    want = oracle_screen(dtype_code, ref, cands, atol, rtol)
+    assert_records_equal(got, want, f"dtype={dtype_code} tol=({atol},{rtol})")
+
+
 @pytest.mark.parametrize("K", [1, 3, 33, 127, 128, 129, 300])
 def test_candidate_counts_around_chunk_size(ctx, kb, K):
     rng = np.random.default_rng(K)
