@@ -483,9 +483,9 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
 
         // One loop for every case: (b) on the largest error, (c) with rel_f = min(rel, rtol_lean).
         //   rel <= rtol_lean ("lean"): rel_f = rel; (c) implies (a).
-        //   rel  > rtol_lean: (c) with the smaller rel_f still implies both (a) and the real (c);
-        //     a thread for which it fails looks again element by element below (it holds an
-        //     element whose relative error exceeds rtol: a mismatch, or one that passes by atol).
+        //   rel  > rtol_lean: (c) with the smaller rel_f still implies both (a) and the real (c)
+        //     (a thread for which it fails holds an element whose relative error exceeds rtol: a
+        //     mismatch, or one that passes by atol).
         //   no lean bound (rtol < 2^-20): rel_f = rel, and (a) is pre-tested per thread on the
         //     largest error against atol alone.
         const bool has_lean = p.rtol_lean >= 0.0f;
@@ -501,9 +501,12 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
           mabs = max3(mabs, fabsf(d0), fabsf(d1));
           mrel = max3_nan(mrel, t0, t1);
         }
-        const bool fire_c = !(mrel <= 0.0f);
-        const bool bad = has_lean ? (!lean && fire_c) : (mabs > p.atol);
-        bool trig = (mabs > th) || extreme || (fire_c && (lean || !has_lean));
+        // A thread whose (c) fails, or (no lean bound) whose largest error exceeds atol, looks
+        // again element by element below before its warp is sent down the exact path.
+        // A thread whose (c) fails, or (no lean bound) whose largest error exceeds atol, looks
+        // again element by element below before its warp is sent down the exact path.
+        const bool bad = !(mrel <= 0.0f) || (!has_lean && mabs > p.atol);
+        bool trig = (mabs > th) || extreme;
         // Every vote below is reached by all 32 lanes: no warp-synchronous call sits under a
         // condition that could differ between lanes.
         if (!__any_sync(0xFFFFFFFFu, trig || bad)) continue;
@@ -511,8 +514,42 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
         // that a failing candidate does not send every step down the exact path; a NaN or Inf
         // difference still does.
         unsigned int mis_fast = 0u;
-        if (bad) {
-          bool again = false;   // a NaN or Inf difference, or the real (c) fails
+        if (bad && lean) {
+          // The second look while lean: the warp goes on to the exact path only for a NaN or Inf
+          // difference or a quotient that can round above rel.  That test is sharper than (c):
+          // with t = fl(ad - rel*|r|) > 0 the quotient still rounds to at most rel while
+          // ad/|r| < rel + ulp(rel)/2, which t <= g*|r| with g = (ulp(rel)/2)*(1 - 2^-20)
+          // guarantees for a normal t (t carries a relative error of 2^-24 at most).  So elements
+          // whose quotient was rounded DOWN to the running maximum (every element of the same
+          // significand class, if the maximum comes from one-ulp differences) stop here instead
+          // of taking the exact path each time.  Such an element is within tolerance as well:
+          // ad < (rel + ulp(rel)/2)*|r| < rtol*(1 - 2^-21)*|r| <= RN(rtol*|r|) <= tol.
+          const unsigned int rb = __float_as_uint(rel);
+          const float g = rb >= (30u << 23)
+                              ? __uint_as_float((rb & 0x7F800000u) - (24u << 23)) * 0.99999904632568359375f
+                              : 0.0f;
+          // (A failure that is large against the thread's errors is a real new maximum: no
+          // need to look.  An element of the kind above fails by 2^-24 of its error at most.)
+          bool again = !(mrel <= mabs * 9.5367431640625e-07f);
+          if (!again) {
+#pragma unroll
+          for (int e = 0; e < kEPT; e += 2) {
+            float d0, d1;
+            E::pair_diff(words, e, r[e], r[e + 1], d0, d1);
+            const float ar0 = fabsf(r[e]), ar1 = fabsf(r[e + 1]);
+            const float t0 = fmaf(-rel, ar0, fabsf(d0)), t1 = fmaf(-rel, ar1, fabsf(d1));
+            // (a NaN or Inf difference makes t NaN or Inf: neither clause holds)
+            const bool c0 = (t0 <= 0.0f) || (t0 >= 7.888609052e-31f && fmaf(-g, ar0, t0) <= 0.0f);
+            const bool c1 = (t1 <= 0.0f) || (t1 >= 7.888609052e-31f && fmaf(-g, ar1, t1) <= 0.0f);
+            again |= !c0 || !c1;
+          }
+          }
+          trig = trig || again;
+        } else if (bad) {
+          // The second look beyond the lean bound: finite mismatches are counted here, so that
+          // a failing candidate does not send every step down the exact path; a NaN or Inf
+          // difference, or a failure of the real (c), still does.
+          bool again = false;
 #pragma unroll
           for (int e = 0; e < kEPT; e += 2) {
             float d0, d1;

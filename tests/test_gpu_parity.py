@@ -241,6 +241,38 @@ def test_tolerance_regimes_on_dense_small_differences(ctx, kb, dtype_code, atol,
     assert_records_equal(got, want, f"dtype={dtype_code} tol=({atol},{rtol})")
 
 
+def test_many_quotients_within_units_in_the_last_place_of_the_max_rel_err(ctx, kb):
+    """Relative errors packed within a few units in the last place of each other: the running
+    maximum is challenged from both sides of every rounding boundary.  fp32: c = r*(1 + q0*(1+u)),
+    |u| < 2^-21.  bf16 / fp16: one-ulp differences everywhere except on the powers of two, so that
+    the largest quotient (1/129, 1/1025) is inexact and shared by a whole significand class."""
+    rng = np.random.default_rng(99)
+    dev = torch.device("cuda", 0)
+    N = 64 * 4096 + 333
+    r64 = rng.standard_normal(N) * np.exp(rng.standard_normal(N))
+    r32 = r64.astype(np.float32)
+    cands = []
+    for q0 in (0.01, 0.0123456, 2.0 ** -7 * 1.5, 0.3):
+        u = rng.uniform(-2.0 ** -21, 2.0 ** -21, N)
+        cands.append(torch.from_numpy((r32.astype(np.float64) * (1 + q0 * (1 + u))).astype(np.float32)).to(dev))
+    ref = torch.from_numpy(r32).to(dev)
+    for atol, rtol in [(1e-2, 1.6e-2), (0.0, 0.5), (1e-3, 1e-3)]:
+        got = run_screen(ctx, kb, ref, cands, atol, rtol)
+        want = oracle_screen(synth.F32, ref, cands, atol, rtol)
+        assert_records_equal(got, want, f"fp32 near ties tol=({atol},{rtol})")
+    for code in (synth.BF16, synth.F16):
+        tdt = synth.TORCH_DTYPE[code]
+        ref = torch.from_numpy(r64).to(tdt).to(dev)
+        eps = 2.0 ** -8 if code == synth.BF16 else 2.0 ** -11
+        cands = []
+        for k in range(6):
+            flip = torch.from_numpy(rng.random(N) < (0.25 if k < 4 else 0.01)).to(dev)
+            cands.append(torch.where(flip, (ref.float() * (1 + eps)).to(tdt), ref))   # ties-to-even spares 2^k
+        got = run_screen(ctx, kb, ref, cands, 1e-2, 1.6e-2)
+        want = oracle_screen(code, ref, cands, 1e-2, 1.6e-2)
+        assert_records_equal(got, want, f"dtype={code} shared inexact maximum")
+
+
 @pytest.mark.parametrize("K", [1, 3, 33, 127, 128, 129, 300])
 def test_candidate_counts_around_chunk_size(ctx, kb, K):
     rng = np.random.default_rng(K)
