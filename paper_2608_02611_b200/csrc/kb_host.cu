@@ -904,6 +904,8 @@ extern "C" kb_status kb_screen_multi(kb_ctx* ctx, uint32_t G, const void* const*
 // table].  In host code this name is only a handle for cudaGetSymbolAddress; it is not a
 // device address and must never be passed to a kernel as it stands.
 static __device__ __align__(256) unsigned char g_static_scratch[KB_STATIC_SCRATCH_BYTES];
+static_assert(KB_STATIC_SCRATCH_BYTES == 256 + KB_STATIC_MAX_K * sizeof(Acc) + KB_STATIC_MAX_K * sizeof(void*),
+              "the header's scratch size must match the accumulator layout");
 
 namespace {
 
