@@ -37,7 +37,7 @@ K_CANDS, SIDE, S_TIMINGS, BUDGET = 64, 4096, 100, 32
 # DRAM bytes moved per algorithmic byte by the streaming screen kernel, from the ncu capture
 # summarised in profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over (K+1)*N*2 bytes);
 # captured at side 2048 (545 MB) and scaled by the bytes a full launch processes.
-DRAM_BYTES_PER_ALGORITHMIC_BYTE = 1.0083
+DRAM_BYTES_PER_ALGORITHMIC_BYTE = 1.0076
 
 WORKLOAD = ("config2: screen K=64 bf16 4096x4096 (atol=1e-2, rtol=1.6e-2) + adjudicate "
             "timings[64][100] + select top 32")
