@@ -144,3 +144,53 @@ def test_random_small_and_medium(ctx, kb, block):
 def test_random_large(ctx, kb, block):
     for i in range(5):
         one_case(ctx, kb, 9_000_000 + block * 1000 + i, 20, 24)
+
+
+def fbits(a):
+    return np.ascontiguousarray(a, dtype=np.float32).view(np.uint32)
+
+
+@pytest.mark.parametrize("block", range(4))
+def test_random_adjudicate_and_select(ctx, kb, block):
+    """Random [K][S] timings (log-normal, rounded to create ties, with zero and negative values
+    now and then), both win-count algorithms, then selection by both policies and by score."""
+    dev = torch.device("cuda", 0)
+    for i in range(12):
+        rng = np.random.default_rng(11_000_000 + block * 1000 + i)
+        K = int(rng.choice([1, 2, 3, 7, 8, 9, 21, 40, 64, 100, 257]))
+        S = int(rng.choice([1, 2, 3, 4, 5, 16, 31, 32, 33, 60, 100, 200, 257, 700]))
+        t = rng.lognormal(0, rng.choice([0.02, 0.3]), (K, S)) * np.exp(rng.normal(0, 0.2, (K, 1)))
+        if rng.random() < 0.5:
+            t = np.round(t, int(rng.choice([1, 2])))
+        if rng.random() < 0.2:
+            t[rng.random((K, S)) < 0.05] = 0.0
+        if rng.random() < 0.1:
+            t = t - 1.0
+        t = t.astype(np.float32)
+        omed, oiqr, owins = oracle.adjudicate(t, threads=8)
+        for algo in (1, 2):
+            try:
+                ctx.set_wins_algo(algo)
+                med, iqr, wins = ctx.adjudicate(torch.from_numpy(t).to(dev))
+            finally:
+                ctx.set_wins_algo(0)
+            assert ctx.poll() == 0
+            label = f"seed block={block} i={i} K={K} S={S} algo={algo}"
+            assert (med.cpu().numpy() == omed).all(), label          # values: the sign of a zero is free
+            assert (iqr.cpu().numpy() == oiqr).all(), label
+            assert (wins.cpu().numpy().view(np.uint32) == owins).all(), label
+        rec = np.zeros(K, dtype=oracle.RESULT_DTYPE)
+        rec["pass"] = rng.random(K) < 0.7
+        rec["mismatch_count"] = 1 - rec["pass"]
+        rec["max_rel_err"] = rng.choice(np.float32([0.0, 2.0 ** -7, 2.0 ** -8, 0.01]), K)
+        d_rec = torch.from_numpy(rec.view(np.uint8).reshape(K, 48).copy()).to(dev)
+        budget = int(rng.integers(1, K + 3))
+        for policy in (0, 1):
+            surv, n = ctx.select(d_rec, med, policy, budget)
+            osurv, on = oracle.select(rec, omed, policy, budget)
+            assert int(n.item()) == on and surv.cpu().numpy().tolist() == osurv.tolist()
+        if (omed > 0).all():
+            sc, surv, n = ctx.select_by_score(d_rec, med, 1, 16, 0.02, 0.01, budget)
+            osc, osurv, on = oracle.select_by_score(rec, omed, 1, 16, 0.02, 0.01, budget)
+            assert (fbits(sc.cpu().numpy()) == fbits(osc)).all()
+            assert int(n.item()) == on and surv.cpu().numpy().tolist() == osurv.tolist()
