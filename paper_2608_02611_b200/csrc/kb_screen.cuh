@@ -836,10 +836,23 @@ __device__ __forceinline__ void small_block(const void* ref, const void* cand, u
   }
   __syncthreads();
   ExactAcc x;
-#pragma unroll 4
-  for (unsigned int j = 0; j < kSmallPerBlock / 256; ++j) {
-    const unsigned long long i = base + j * 256 + threadIdx.x;
-    if (i < N && mask_selected(mask, i)) x.add(E::load(ref, i), E::load(cand, i), i, atol, rtol);
+  {
+    // all loads first (one round trip to memory instead of one per unrolled group), then the
+    // arithmetic
+    constexpr unsigned int kPer = kSmallPerBlock / 256;
+    float rv[kPer], cv[kPer];
+    unsigned int sel = 0u;
+#pragma unroll
+    for (unsigned int j = 0; j < kPer; ++j) {
+      const unsigned long long i = base + j * 256 + threadIdx.x;
+      const bool on = i < N && mask_selected(mask, i);
+      sel |= on ? (1u << j) : 0u;
+      rv[j] = on ? E::load(ref, i) : 0.0f;
+      cv[j] = on ? E::load(cand, i) : 0.0f;
+    }
+#pragma unroll
+    for (unsigned int j = 0; j < kPer; ++j)
+      if (sel & (1u << j)) x.add(rv[j], cv[j], base + j * 256 + threadIdx.x, atol, rtol);
   }
   x.n_mis = warp_add_u32(x.n_mis);
   x.n_nan = warp_add_u32(x.n_nan);
