@@ -182,9 +182,12 @@ def run_adjudicate(args):
         R = ((S + nj - 1) // nj + 31) // 32
         evals = KB * (KB + 1) // 2 * 64 * S * (nj * R * 32)
         peak = 148 * 64 * 1.965e9 / 2          # sample-pair evaluations/s at 64 ALU lanes/clk/SM
+        probe = ctx.alu_probe(20000)           # the same instruction mix on registers only, measured
         line["roofline"] = {"bound": "alu", "achieved": evals / (wins_ms * 1e-3), "peak": peak,
                             "unit": "sample-pair evaluations/s", "frac": evals / (wins_ms * 1e-3) / peak,
-                            "traffic": None}
+                            "traffic": None, "peak_source": "derived: 148 SMs x 64 ALU lanes x 1.965 GHz / 2 "
+                            "compares per pair", "measured_probe": probe,
+                            "frac_of_probe": evals / (wins_ms * 1e-3) / probe}
     print(json.dumps(line), flush=True)
     ctx.close()
 

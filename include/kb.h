@@ -136,6 +136,12 @@ kb_status kb_ctx_enable_timing(kb_ctx* ctx, int on);
  * durations in milliseconds (oldest first, at most `cap`) to h_ms (HOST) and
  * their number to *n (HOST); the record is then cleared. */
 kb_status kb_ctx_read_timer(kb_ctx* ctx, kb_timer which, float* h_ms, uint32_t cap, uint32_t* n);
+/* Register-only probe of the instruction mix of the direct win count (two compares and two
+ * predicated increments per sample pair, values held in registers): runs it on every SM for
+ * `iters` (<= 2^23) rounds of 128 sample pairs per thread, times it with CUDA events on
+ * `stream`, and writes the rate in sample pairs per second to *pairs_per_s (HOST).  This is
+ * the measured ceiling the direct win-count kernel is compared with.  Synchronous. */
+kb_status kb_alu_probe(kb_ctx* ctx, uint32_t iters, double* pairs_per_s, void* stream);
 /* Choose how kb_adjudicate counts wins: 0 = automatic (binary search on the
  * sorted rows when 8 rows fit shared memory, i.e. S <= 4096, else direct
  * comparison), 1 = always direct comparison of all sample pairs, 2 = always

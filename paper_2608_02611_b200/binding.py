@@ -43,7 +43,7 @@ RESULT_F64_BYTES = 56
 
 EXPORTS = [
     "kb_ctx_create", "kb_ctx_destroy", "kb_last_error", "kb_ctx_poll", "kb_ctx_set_grid",
-    "kb_ctx_enable_timing", "kb_ctx_read_timer", "kb_ctx_launch_count", "kb_ctx_set_wins_algo", "kb_ctx_set_small_path",
+    "kb_ctx_enable_timing", "kb_ctx_read_timer", "kb_alu_probe", "kb_ctx_launch_count", "kb_ctx_set_wins_algo", "kb_ctx_set_small_path",
     "kb_mask_create_strided", "kb_mask_create_bitmap", "kb_mask_count", "kb_mask_destroy",
     "kb_screen", "kb_screen_f64", "kb_screen_host", "kb_screen_static", "kb_screen_indexed", "kb_screen_multi", "kb_adjudicate", "kb_adjudicate_ragged", "kb_select",
     "kb_select_by_score", "kb_tail_ratios", "kb_copeland", "kb_confirm",
@@ -80,6 +80,7 @@ def load() -> ctypes.CDLL:
     L.kb_ctx_set_grid.argtypes = [vp, u32]
     L.kb_ctx_enable_timing.argtypes = [vp, i32]
     L.kb_ctx_read_timer.argtypes = [vp, i32, vp, u32, ctypes.POINTER(u32)]
+    L.kb_alu_probe.argtypes = [vp, u32, ctypes.POINTER(ctypes.c_double), vp]
     L.kb_ctx_launch_count.argtypes = [vp, ctypes.POINTER(u64)]
     L.kb_ctx_set_wins_algo.argtypes = [vp, i32]
     L.kb_ctx_set_small_path.argtypes = [vp, i32]
@@ -203,6 +204,13 @@ class Context:
         n = ctypes.c_uint64(0)
         self._check(load().kb_ctx_launch_count(self._h, ctypes.byref(n)), "kb_ctx_launch_count")
         return int(n.value)
+
+    def alu_probe(self, iters: int = 20000) -> float:
+        """kb_alu_probe: measured sample pairs per second of the direct win count's inner loop."""
+        v = ctypes.c_double(0.0)
+        self._check(load().kb_alu_probe(self._h, iters, ctypes.byref(v), _stream_ptr(self.device)),
+                    "kb_alu_probe")
+        return float(v.value)
 
     # -- masks --------------------------------------------------------------
     def mask_strided(self, N: int, log2_tile: int, stride: int, phase: int) -> Mask:

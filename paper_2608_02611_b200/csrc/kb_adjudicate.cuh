@@ -152,6 +152,37 @@ __device__ __forceinline__ void count_pair(unsigned int& cnt, float a, float b) 
       : "f"(a), "f"(b));
 }
 
+// Register-only probe of the direct win count's instruction mix (no paper counterpart): every
+// thread runs count_pair on values that never leave its registers, 8 b-values against a
+// stream of a-values, as wins_kernel<8> does between two shared-memory reads.  The rate it
+// reaches is the measured ceiling for "sample pairs per second" of that kernel on this GPU at
+// the clock it holds.  The result is stored only if it has a value it cannot have, which is
+// enough to keep the loop alive.
+__global__ void __launch_bounds__(256) alu_probe_kernel(unsigned int iters, float seed,
+                                                        unsigned int* __restrict__ sink) {
+  float b[8];
+  unsigned int cnt[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    b[i] = seed + 0.37f * (float)i + 0.001f * (float)threadIdx.x;
+    cnt[i] = 0u;
+  }
+  float a = 0.5f * seed + 0.01f * (float)(threadIdx.x & 31);
+  for (unsigned int it = 0; it < iters; ++it) {
+#pragma unroll
+    for (int u = 0; u < 16; ++u) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) count_pair(cnt[i], a, b[i]);
+      a = fmaf(a, 1.0000001f, 0.03125f);   // one more instruction per 8 pairs keeps a moving
+      if (a > 4.0f * seed) a -= 4.0f * seed;
+    }
+  }
+  unsigned int tot = 0u;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) tot += cnt[i];
+  if (tot == 0xFFFFFFFFu) *sink = tot;   // 2 * 16 * 8 * iters < 2^32 - 1: never taken
+}
+
 template <int R>
 __global__ void __launch_bounds__(kWinsThreads) wins_kernel(const WinsParams p) {
   extern __shared__ float as[];   // [TA][IC]

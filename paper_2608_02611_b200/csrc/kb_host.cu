@@ -375,6 +375,31 @@ extern "C" kb_status kb_ctx_read_timer(kb_ctx* ctx, kb_timer which, float* h_ms,
   return KB_OK;
 }
 
+extern "C" kb_status kb_alu_probe(kb_ctx* ctx, uint32_t iters, double* pairs_per_s, void* stream) {
+  if (!ctx) return KB_ERR_INVALID_ARG;
+  if (!pairs_per_s || iters == 0) return fail(ctx, KB_ERR_INVALID_ARG, "kb_alu_probe: null pointer or iters = 0");
+  DeviceGuard g(ctx->device);
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const unsigned int blocks = (unsigned int)ctx->sm_count * 8u, threads = 256u;
+  if (iters > (1u << 23)) return fail(ctx, KB_ERR_INVALID_ARG, "kb_alu_probe: iters above 2^23");
+  unsigned int* sink = ctx->d_status + 60;   // a spare status word; never written in practice
+  cudaEvent_t e0, e1;
+  KB_CUDA(ctx, cudaEventCreate(&e0));
+  KB_CUDA(ctx, cudaEventCreate(&e1));
+  alu_probe_kernel<<<blocks, threads, 0, st>>>(iters / 8 + 1, 1.5f, sink);   // warm-up
+  KB_CUDA(ctx, cudaEventRecord(e0, st));
+  alu_probe_kernel<<<blocks, threads, 0, st>>>(iters, 1.5f, sink);
+  KB_CUDA(ctx, cudaEventRecord(e1, st));
+  ctx->launches += 2;
+  KB_CUDA(ctx, cudaEventSynchronize(e1));
+  float ms = 0.0f;
+  KB_CUDA(ctx, cudaEventElapsedTime(&ms, e0, e1));
+  cudaEventDestroy(e0);
+  cudaEventDestroy(e1);
+  *pairs_per_s = (double)blocks * threads * (double)iters * 16.0 * 8.0 / ((double)ms * 1e-3);
+  return KB_OK;
+}
+
 extern "C" kb_status kb_ctx_launch_count(const kb_ctx* ctx, uint64_t* n) {
   if (!ctx || !n) return KB_ERR_INVALID_ARG;
   *n = ctx->launches;

@@ -748,3 +748,9 @@ def test_fp8_large_with_masks_and_grids(ctx, kb, dtype_code):
             got = run_screen(ctx, kb, ref, cands, 1e-2, 7e-2, mask_spec)
             ctx.set_grid(0)
             assert_records_equal(got, want, f"fp8 {dtype_code} mask={mask_spec} grid={grid}")
+
+
+def test_alu_probe_reports_a_rate(ctx, kb):
+    rate = ctx.alu_probe(2000)
+    assert 1e11 < rate < 1e14          # sample pairs per second; 148 SMs x 64 lanes x 2 GHz / 2 = 9.3e12
+    assert ctx.poll() == 0
