@@ -383,19 +383,25 @@ extern "C" kb_status kb_alu_probe(kb_ctx* ctx, uint32_t iters, double* pairs_per
   const unsigned int blocks = (unsigned int)ctx->sm_count * 8u, threads = 256u;
   if (iters > (1u << 23)) return fail(ctx, KB_ERR_INVALID_ARG, "kb_alu_probe: iters above 2^23");
   unsigned int* sink = ctx->d_status + 60;   // a spare status word; never written in practice
-  cudaEvent_t e0, e1;
-  KB_CUDA(ctx, cudaEventCreate(&e0));
-  KB_CUDA(ctx, cudaEventCreate(&e1));
+  struct Events {   // released on every path
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    ~Events() {
+      if (e0) cudaEventDestroy(e0);
+      if (e1) cudaEventDestroy(e1);
+    }
+  } ev;
+  KB_CUDA(ctx, cudaEventCreate(&ev.e0));
+  KB_CUDA(ctx, cudaEventCreate(&ev.e1));
   alu_probe_kernel<<<blocks, threads, 0, st>>>(iters / 8 + 1, 1.5f, sink);   // warm-up
-  KB_CUDA(ctx, cudaEventRecord(e0, st));
+  KB_CUDA(ctx, cudaEventRecord(ev.e0, st));
   alu_probe_kernel<<<blocks, threads, 0, st>>>(iters, 1.5f, sink);
-  KB_CUDA(ctx, cudaEventRecord(e1, st));
+  KB_CUDA(ctx, cudaEventRecord(ev.e1, st));
   ctx->launches += 2;
-  KB_CUDA(ctx, cudaEventSynchronize(e1));
+  KB_CUDA(ctx, cudaGetLastError());
+  KB_CUDA(ctx, cudaEventSynchronize(ev.e1));
   float ms = 0.0f;
-  KB_CUDA(ctx, cudaEventElapsedTime(&ms, e0, e1));
-  cudaEventDestroy(e0);
-  cudaEventDestroy(e1);
+  KB_CUDA(ctx, cudaEventElapsedTime(&ms, ev.e0, ev.e1));
+  if (!(ms > 0.0f)) return fail(ctx, KB_ERR_CUDA, "kb_alu_probe: the probe took no measurable time");
   *pairs_per_s = (double)blocks * threads * (double)iters * 16.0 * 8.0 / ((double)ms * 1e-3);
   return KB_OK;
 }
