@@ -55,3 +55,29 @@ def test_product_does_not_import_the_oracle():
                 text = open(os.path.join(dirpath, f)).read()
                 assert "import oracle" not in text and "from oracle" not in text, f
                 assert "kb_oracle" not in text, f
+
+
+def test_header_is_plain_c99_and_a_c_program_links(tmp_path):
+    """include/kb.h compiles as C99 (no C++ or CUDA types in the boundary) with the record
+    sizes it documents, and a C translation unit that calls an entry point links against the
+    library.  The program is not run: without a GPU kb_ctx_create would only report that."""
+    import subprocess
+    from paper_2608_02611_b200 import build
+    lib_path = build.build()
+    src = tmp_path / "use_kb.c"
+    src.write_text(
+        '#include "kb.h"\n'
+        "typedef char rec32[sizeof(kb_screen_result) == 48 ? 1 : -1];\n"
+        "typedef char rec64[sizeof(kb_screen_result_f64) == 56 ? 1 : -1];\n"
+        "int main(void) {\n"
+        "  kb_ctx* ctx = 0;\n"
+        "  kb_status st = kb_ctx_create(0, &ctx);\n"
+        "  if (st == KB_OK) kb_ctx_destroy(ctx);\n"
+        "  return (int)st;\n"
+        "}\n")
+    exe = tmp_path / "use_kb"
+    cmd = ["gcc", "-std=c99", "-pedantic", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"),
+           str(src), lib_path, "-o", str(exe), "-Wl,-rpath," + os.path.dirname(lib_path),
+           "-Wl,--allow-shlib-undefined"]
+    done = subprocess.run(cmd, capture_output=True, text=True)
+    assert done.returncode == 0, done.stderr
