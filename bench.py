@@ -264,7 +264,7 @@ def main():
     ap.add_argument("--flip-frac", type=float, default=0.25)
     ap.add_argument("--K", type=int, default=512)
     ap.add_argument("--S", type=int, default=200)
-    ap.add_argument("--wins-algo", type=int, default=0, choices=[0, 1, 2])
+    ap.add_argument("--wins-algo", type=int, default=0, choices=[0, 1, 2, 3])
     ap.add_argument("--side", type=int, default=SIDE,
                     help="tensor side; anything but 4096 is for profiler captures only and is "
                          "not a benchmark configuration")

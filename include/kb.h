@@ -142,10 +142,11 @@ kb_status kb_ctx_read_timer(kb_ctx* ctx, kb_timer which, float* h_ms, uint32_t c
  * `stream`, and writes the rate in sample pairs per second to *pairs_per_s (HOST).  This is
  * the measured ceiling the direct win-count kernel is compared with.  Synchronous. */
 kb_status kb_alu_probe(kb_ctx* ctx, uint32_t iters, double* pairs_per_s, void* stream);
-/* Choose how kb_adjudicate counts wins: 0 = automatic (binary search on the
- * sorted rows when 8 rows fit shared memory, i.e. S <= 4096, else direct
- * comparison), 1 = always direct comparison of all sample pairs, 2 = always
- * binary search (S <= 4096 only).  The integers produced are identical. */
+/* Choose how kb_adjudicate counts wins: 0 = automatic (on the sorted rows when they fit shared
+ * memory: a lane-per-row merge for K >= 225 and S <= 1024, else a binary search and walk per
+ * row pair for S <= 4096; direct comparison beyond), 1 = always direct comparison of all
+ * sample pairs, 2 = always binary search (S <= 4096 only), 3 = always the lane-per-row merge
+ * (S <= 1024 only).  The integers produced are identical. */
 kb_status kb_ctx_set_wins_algo(kb_ctx* ctx, int algo);
 /* Number of kernels this context has launched since it was created (HOST out). */
 kb_status kb_ctx_launch_count(const kb_ctx* ctx, uint64_t* n);

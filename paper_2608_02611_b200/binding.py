@@ -185,7 +185,8 @@ class Context:
         self._check(load().kb_ctx_set_small_path(self._h, 1 if on else 0), "kb_ctx_set_small_path")
 
     def set_wins_algo(self, algo: int):
-        """0 automatic, 1 direct comparison of all sample pairs, 2 binary search on sorted rows."""
+        """0 automatic, 1 direct comparison of all sample pairs, 2 binary search on sorted rows,
+        3 lane-per-row merge of sorted rows."""
         self._check(load().kb_ctx_set_wins_algo(self._h, int(algo)), "kb_ctx_set_wins_algo")
 
     def enable_timing(self, on: bool = True):

@@ -11,6 +11,8 @@
 //                     one binary search, then a merge walk.  O(K^2 (S + 32 log S))
 //                     instead of O(K^2 S^2); the default when a
 //                     block of 8 sorted rows fits shared memory (S <= 4096).
+// wins_merge_kernel   the same integers again, for many candidates with short rows: a warp
+//                     walks one a row against 32 b rows, one per lane (see below).
 // wins_kernel         pairwise doubled Mann-Whitney counts by direct comparison.  A CTA takes a
 //                     block of 8 "a" rows x 8 "b" rows and a chunk of samples
 //                     of each; the a-chunk is staged in shared memory, each
@@ -324,6 +326,102 @@ __global__ void __launch_bounds__(kWinsThreads) wins_rank_kernel(const WinsRankP
       p.wins[(size_t)a * p.K + b] = 2u * p.S * p.S - sum;
       if (Ab != Bb) p.wins[(size_t)b * p.K + a] = sum;
     }
+  }
+}
+
+// ---------------------------------------------------------------------------
+// The same integers by a lane-per-row merge, for many candidates with short rows.  A CTA
+// stages a tile of 32 sorted b rows and 8 sorted a rows in shared memory (odd row stride,
+// every row closed by +Inf); warp w walks a row w against the 32 b rows at once, lane l
+// against b row l, with three pointers that only grow: i over a's samples, jl = #{b < a_i},
+// ju = #{b <= a_i}.  At most 3S steps of a dozen instructions serve 32 row pairs, against a
+// binary search and a walk per pair and lane in wins_rank_kernel.  Tiles (TA <= TB) of 32 x 32
+// rows; the mirrored entry comes from W[a][b] + W[b][a] = 2*S*S.
+// ---------------------------------------------------------------------------
+constexpr int kMergeTile = 32;    // b rows per CTA (one per lane) and rows per tile
+constexpr int kMergeARows = 8;    // a rows per CTA (one per warp)
+struct WinsMergeParams {
+  const float* sorted;   // [K][S] rows sorted ascending
+  unsigned int* wins;
+  unsigned int K, S, stride, nT;   // stride: odd, > S; nT: tiles of 32 rows
+};
+
+__global__ void __launch_bounds__(256) wins_merge_kernel(const WinsMergeParams p) {
+  extern __shared__ float ms[];   // [32][stride] b rows, then [8][stride] a rows
+  float* Bs = ms;
+  float* As = ms + (size_t)kMergeTile * p.stride;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const unsigned int nsub = kMergeTile / kMergeARows;
+  const unsigned int sub = blockIdx.x % nsub;
+  unsigned int TA = 0, rem = blockIdx.x / nsub;
+  while (rem >= p.nT - TA) {
+    rem -= p.nT - TA;
+    ++TA;
+  }
+  const unsigned int TB = TA + rem;
+  const unsigned int b0 = TB * kMergeTile;
+  const unsigned int a0 = TA * kMergeTile + sub * kMergeARows;
+  const float inf = __uint_as_float(0x7F800000u);
+  // stage the rows; rows past K and the closing element of every row are +Inf
+  for (unsigned int r = warp; r < kMergeTile + kMergeARows; r += 8) {
+    const bool is_b = r < kMergeTile;
+    const unsigned int row = is_b ? b0 + r : a0 + (r - kMergeTile);
+    float* dst = (is_b ? Bs + (size_t)r * p.stride : As + (size_t)(r - kMergeTile) * p.stride);
+    const float* src = p.sorted + (size_t)row * p.S;
+    for (unsigned int j = lane; j <= p.S; j += 32) dst[j] = (row < p.K && j < p.S) ? src[j] : inf;
+  }
+  __syncthreads();
+  const unsigned int a = a0 + warp, b = b0 + lane;
+  if (a >= p.K) return;   // the whole warp
+  const float* ar = As + (size_t)warp * p.stride;
+  const float* br = Bs + (size_t)lane * p.stride;
+  const bool live = b < p.K;
+  // The three current values live in registers; a step reloads only the one whose pointer moved.
+  // Pointers are byte addresses in shared memory, so that a step is 16 instructions: the sum of
+  // the two b pointers is accumulated as it stands and rebased at the end.
+  const unsigned int a_end = smem_u32(ar) + 4u * p.S;
+  const unsigned int b_base = smem_u32(br);
+  unsigned int ia = live ? smem_u32(ar) : a_end, il = b_base, iu = b_base, sum = 0u;
+  float x = ar[0], yl = br[0], yu = yl;
+  while (__any_sync(0xFFFFFFFFu, ia < a_end)) {
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      asm volatile(
+          "{\n"
+          ".reg .pred on, pl, pu, tk;\n"
+          ".reg .u32 ad;\n"
+          ".reg .f32 v;\n"
+          "setp.lt.u32 on, %0, %7;\n"              // rows left in a?
+          "setp.lt.and.f32 pl, %4, %3, on;\n"      // b[jl] <  x: the closing +Inf stops both pointers
+          "setp.le.and.f32 pu, %5, %3, on;\n"      // b[ju] <= x
+          "and.pred pu, pu, !pl;\n"
+          "or.pred tk, pl, pu;\n"
+          "and.pred tk, on, !tk;\n"                // neither moves: x is counted
+          "@pl add.u32 %1, %1, 4;\n"
+          "@pu add.u32 %2, %2, 4;\n"
+          "@tk add.u32 %6, %6, %1;\n"
+          "@tk add.u32 %6, %6, %2;\n"
+          "@tk add.u32 %0, %0, 4;\n"
+          "selp.u32 ad, %1, %2, pl;\n"
+          "selp.u32 ad, %0, ad, tk;\n"
+          "ld.shared.f32 v, [ad];\n"               // a[S] = +Inf is loaded but never used
+          "@pl mov.f32 %4, v;\n"
+          "@pu mov.f32 %5, v;\n"
+          "@tk mov.f32 %3, v;\n"
+          "}\n"
+          : "+r"(ia), "+r"(il), "+r"(iu), "+f"(x), "+f"(yl), "+f"(yu), "+r"(sum)
+          : "r"(a_end)
+          : "memory");
+    }
+  }
+  const unsigned int acc = (sum - 2u * p.S * b_base) >> 2;
+  if (!live) return;
+  // acc = sum over a's samples of (#{b < x} + #{b <= x}) = W[b][a]
+  if (TA == TB) {
+    p.wins[(size_t)b * p.K + a] = acc;   // a diagonal tile computes every ordered pair itself
+  } else {
+    p.wins[(size_t)a * p.K + b] = 2u * p.S * p.S - acc;
+    p.wins[(size_t)b * p.K + a] = acc;
   }
 }
 

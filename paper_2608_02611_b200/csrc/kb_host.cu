@@ -26,7 +26,8 @@ struct kb_ctx {
   uint32_t forced_grid = 0;
   unsigned char* small_ws = nullptr; // single-launch path: [tickets 2 KB | partial records 80 KB]
   bool small_on = true;
-  int wins_algo = 0;                // 0 auto, 1 direct comparison, 2 binary search on sorted rows
+  int wins_algo = 0;                // 0 auto, 1 direct comparison, 2 binary search on sorted rows,
+                                    // 3 lane-per-row merge of sorted rows
   float* srt = nullptr;             // [K][S] sorted timings (binary-search win count)
   size_t srt_bytes = 0;
   char err[512] = {0};
@@ -205,6 +206,8 @@ kb_status set_stream64_attr(kb_ctx* ctx) {
   return KB_OK;
 }
 
+constexpr uint32_t kMergeMaxS = 1024;   // 40 rows of S + 2 floats in shared memory: 164 KB
+
 template <int R>
 void launch_wins(const WinsParams& wp, unsigned int grid, size_t smem, cudaStream_t st) {
   wins_kernel<R><<<grid, kWinsThreads, smem, st>>>(wp);
@@ -264,6 +267,11 @@ extern "C" kb_status kb_ctx_create(int device, kb_ctx** out) {
   if (cudaFuncSetAttribute(rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)(KB_MAX_S * sizeof(float))) != cudaSuccess) {
     fail(ctx, KB_ERR_CUDA, "cannot raise the shared-memory limit of the row kernel");
+    return bail(KB_ERR_CUDA);
+  }
+  if (cudaFuncSetAttribute(wins_merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)((kMergeTile + kMergeARows) * ((kMergeMaxS + 1) | 1u) * sizeof(float))) != cudaSuccess) {
+    fail(ctx, KB_ERR_CUDA, "cannot raise the shared-memory limit of the merge win-count kernel");
     return bail(KB_ERR_CUDA);
   }
   if (cudaFuncSetAttribute(tails_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -338,7 +346,7 @@ extern "C" kb_status kb_ctx_set_small_path(kb_ctx* ctx, int on) {
 }
 
 extern "C" kb_status kb_ctx_set_wins_algo(kb_ctx* ctx, int algo) {
-  if (!ctx || algo < 0 || algo > 2) return KB_ERR_INVALID_ARG;
+  if (!ctx || algo < 0 || algo > 3) return KB_ERR_INVALID_ARG;
   ctx->wins_algo = algo;
   return KB_OK;
 }
@@ -1080,11 +1088,13 @@ extern "C" kb_status kb_adjudicate(kb_ctx* ctx, const float* d_timings, uint32_t
   bool rank = d_wins && S <= 4096 && ctx->wins_algo != 1;
   if (ctx->wins_algo == 2 && d_wins && S > 4096)
     return fail(ctx, KB_ERR_UNSUPPORTED, "kb_adjudicate: the binary-search win count needs S <= 4096");
+  if (ctx->wins_algo == 3 && d_wins && S > kMergeMaxS)
+    return fail(ctx, KB_ERR_UNSUPPORTED, "kb_adjudicate: the merge win count needs S <= %u", kMergeMaxS);
   if (rank) {
     size_t have = ctx->srt_bytes;
     if (ensure_buf(ctx, &ctx->srt, &have, (size_t)K * S * sizeof(float)) == KB_OK) {
       ctx->srt_bytes = have;
-    } else if (ctx->wins_algo == 2) {
+    } else if (ctx->wins_algo >= 2) {
       return KB_ERR_WORKSPACE;
     } else {
       ctx->srt_bytes = 0;
@@ -1100,6 +1110,28 @@ extern "C" kb_status kb_adjudicate(kb_ctx* ctx, const float* d_timings, uint32_t
   ++ctx->launches;
   KB_CUDA(ctx, cudaGetLastError());
   if (!d_wins) return KB_OK;
+
+  // many candidates with short rows: one warp walks a row against 32 rows at once
+  const unsigned int nT = (K + kMergeTile - 1) / kMergeTile;
+  if (rank && S <= kMergeMaxS && (ctx->wins_algo == 3 || (ctx->wins_algo == 0 && nT >= 8))) {
+    WinsMergeParams mp;
+    mp.sorted = ctx->srt;
+    mp.wins = d_wins;
+    mp.K = K;
+    mp.S = S;
+    mp.stride = (S + 1) | 1u;
+    mp.nT = nT;
+    const unsigned long long grid_m = (unsigned long long)nT * (nT + 1) / 2 * (kMergeTile / kMergeARows);
+    if (grid_m > 0x7FFFFFFFull) return fail(ctx, KB_ERR_UNSUPPORTED, "kb_adjudicate: K too large for one launch");
+    {
+      ScopedTimer tm(ctx, KB_TIMER_WINS, st);
+      wins_merge_kernel<<<(unsigned int)grid_m, 256,
+                          (size_t)(kMergeTile + kMergeARows) * mp.stride * sizeof(float), st>>>(mp);
+    }
+    ++ctx->launches;
+    KB_CUDA(ctx, cudaGetLastError());
+    return KB_OK;
+  }
 
   if (rank) {
     WinsRankParams rp;

@@ -433,7 +433,9 @@ def test_adjudicate_matches_oracle(ctx, kb, K, S):
             t = np.round(t, 2)
         t = t.astype(np.float32)
         omed, oiqr, owins = oracle.adjudicate(t)
-        for algo in (1, 2, 0):
+        for algo in (1, 2, 3, 0):
+            if algo == 3 and S > 1024:
+                continue
             try:
                 ctx.set_wins_algo(algo)
                 med, iqr, wins = ctx.adjudicate(torch.from_numpy(t).to(dev))

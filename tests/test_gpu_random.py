@@ -168,7 +168,7 @@ def test_random_adjudicate_and_select(ctx, kb, block):
             t = t - 1.0
         t = t.astype(np.float32)
         omed, oiqr, owins = oracle.adjudicate(t, threads=8)
-        for algo in (1, 2):
+        for algo in (1, 2, 3):
             try:
                 ctx.set_wins_algo(algo)
                 med, iqr, wins = ctx.adjudicate(torch.from_numpy(t).to(dev))
