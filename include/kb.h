@@ -229,7 +229,7 @@ kb_status kb_screen_multi(kb_ctx* ctx, uint32_t G, const void* const* h_refs,
                           kb_dtype dtype, float atol, float rtol, kb_screen_result* d_out,
                           void* stream);
 
-/* ---- the gate for double-precision tensors ---------------------------------
+/* ---- the gate for double-precision tensors (Sec. 3.1 K(p); Sec. 3.4 Verifier) ----
  * The same gate with the reference and the candidates stored in binary64 and
  * EVERY operation of the record (d, tol, the comparison, d/|r|) in binary64,
  * round-to-nearest-even, no fused multiply-add: a double-precision output is
@@ -249,7 +249,7 @@ typedef struct {
 /* Arguments as for kb_screen (DEVICE d_ref, HOST array of K DEVICE pointers, all
  * 16-byte aligned; atol, rtol finite and >= 0; mask NULL or created for the
  * same N; DEVICE d_out of K records, fully overwritten).  Asynchronous on
- * `stream`. */
+ * `stream`.  1 <= K <= KB_MAX_K, 1 <= N <= KB_MAX_N.  Errors as for kb_screen. */
 kb_status kb_screen_f64(kb_ctx* ctx, const double* d_ref, const double* const* h_cands, uint32_t K,
                         uint64_t N, double atol, double rtol, const kb_mask* mask,
                         kb_screen_result_f64* d_out, void* stream);
