@@ -414,7 +414,8 @@ def main():
                 "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
                 "kernel": "screen_stream_kernel<bf16>", "launch_ms_avg": avg_stream_ms,
                 "launch_ms_min": float(np.min(stream_ms)) if len(stream_ms) else None,
-                "algorithmic_bytes_per_launch": stream_bytes, "launches_timed": int(len(stream_ms))}
+                "algorithmic_bytes_per_launch": stream_bytes, "launches_timed": int(len(stream_ms)),
+                "share_of_step": avg_stream_ms / ms_per_step}
 
     # ---- CPU baseline: the oracle as it stands on a bounded sample (rank 0, N=1 only) ----
     cpu_baseline = None
