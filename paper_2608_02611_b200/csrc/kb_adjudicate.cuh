@@ -368,7 +368,17 @@ __global__ void __launch_bounds__(256) wins_merge_kernel(const WinsMergeParams p
     const unsigned int row = is_b ? b0 + r : a0 + (r - kMergeTile);
     float* dst = (is_b ? Bs + (size_t)r * p.stride : As + (size_t)(r - kMergeTile) * p.stride);
     const float* src = p.sorted + (size_t)row * p.S;
-    for (unsigned int j = lane; j <= p.S; j += 32) dst[j] = (row < p.K && j < p.S) ? src[j] : inf;
+    for (unsigned int j = lane; j <= p.S; j += 32) {
+      float v = inf;
+      if (row < p.K && j < p.S) {
+        v = src[j];
+        // A non-finite timing voids the call (rows_kernel has set KB_ERR_NONFINITE); here it
+        // must only not reach the closing +Inf's role: the walk below stops at the first value
+        // that is above every sample, so no staged sample may be +Inf or NaN.
+        if (!(fabsf(v) <= 3.402823466e38f)) v = 3.402823466e38f;
+      }
+      dst[j] = v;
+    }
   }
   __syncthreads();
   const unsigned int a = a0 + warp, b = b0 + lane;

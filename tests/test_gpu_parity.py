@@ -487,6 +487,24 @@ def test_adjudicate_flags_nonfinite(ctx, kb):
         assert ctx.poll() == 0          # the status word is cleared by the read
 
 
+def test_adjudicate_flags_nonfinite_with_many_candidates(ctx, kb):
+    """The lane-per-row merge (K >= 225) stages its rows with non-finite samples replaced, so
+    that its walk stays inside the rows; the call is flagged and the other rows' medians hold."""
+    dev = torch.device("cuda", 0)
+    rng = np.random.default_rng(3)
+    base = rng.lognormal(0, 0.1, (300, 50)).astype(np.float32)
+    omed = oracle.adjudicate(base, want_wins=False)[0]
+    for bad in (float("nan"), float("inf"), float("-inf")):
+        t = torch.from_numpy(base).to(dev)
+        t[7, 3] = bad
+        t[250, 49] = bad
+        med, iqr, wins = ctx.adjudicate(t)
+        assert ctx.poll() == 6          # KB_ERR_NONFINITE
+        keep = np.ones(300, dtype=bool)
+        keep[[7, 250]] = False
+        assert (med.cpu().numpy()[keep] == omed[keep]).all()
+
+
 @pytest.mark.parametrize("policy", [0, 1])
 @pytest.mark.parametrize("K,budget", [(1, 1), (7, 3), (33, 8), (64, 64), (40, 100), (300, 32), (1000, 7)])
 def test_select_matches_oracle(ctx, kb, policy, K, budget):
