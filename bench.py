@@ -202,7 +202,8 @@ def run_screen(args):
     from paper_2608_02611_b200 import binding
     dev = torch.device("cuda", 0)
     ctx = binding.Context(0)
-    ctx.set_small_path(False)
+    if not args.default_dispatch:
+        ctx.set_small_path(False)      # time the streaming path whatever the size
     K, N = args.K, 1 << args.log2n
     tdt = {"f64": torch.float64, "f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16}[args.dtype]
     idt = {8: torch.int64, 4: torch.int32, 2: torch.int16}[torch.empty(0, dtype=tdt).element_size()]
@@ -228,7 +229,8 @@ def run_screen(args):
     e1.record()
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / steps
-    k_ms = float(np.mean(ctx.read_timer(binding.KB_TIMER_SCREEN_STREAM)))
+    tk = ctx.read_timer(binding.KB_TIMER_SCREEN_STREAM)
+    k_ms = float(np.mean(tk)) if len(tk) else float("nan")   # no streaming launch on the small path
     assert ctx.poll() == 0
     ntiles = N // 4096
     nscout = min(8, max(1, ntiles // 128)) if ntiles >= 2 else 0
@@ -262,6 +264,8 @@ def main():
                     help="storage type of the 'screen' workload")
     ap.add_argument("--log2n", type=int, default=24, help="elements per tensor of the 'screen' workload")
     ap.add_argument("--flip-frac", type=float, default=0.25)
+    ap.add_argument("--default-dispatch", action="store_true",
+                    help="'screen' workload: let small problems take the single-launch kernel")
     ap.add_argument("--K", type=int, default=512)
     ap.add_argument("--S", type=int, default=200)
     ap.add_argument("--wins-algo", type=int, default=0, choices=[0, 1, 2, 3])

@@ -221,8 +221,8 @@ kb_status kb_screen_indexed(kb_ctx* ctx, const void* d_ref, const void* const* d
  *   h_refs   HOST array of G DEVICE pointers.
  *   h_cands  HOST array of sum(h_K) DEVICE pointers, group after group.
  *   d_out    DEVICE records in the order of h_cands.
- * 1 <= G <= 64, sum(h_K) <= 1024, and the tensors together at most 2048
- * blocks of 4096 elements (sum over candidates of ceil(N_g / 4096)); no mask.
+ * 1 <= G <= 64, sum(h_K) <= 1024, and the tensors together at most 8192
+ * blocks of 1024 elements (sum over candidates of ceil(N_g / 1024)); no mask.
  * Larger jobs: call kb_screen per group. */
 kb_status kb_screen_multi(kb_ctx* ctx, uint32_t G, const void* const* h_refs,
                           const void* const* h_cands, const uint32_t* h_K, const uint64_t* h_N,

@@ -24,7 +24,7 @@ struct kb_ctx {
   size_t ws_bytes = 0;
   unsigned int* d_status = nullptr;
   uint32_t forced_grid = 0;
-  unsigned char* small_ws = nullptr; // single-launch path: [tickets 2 KB | partial records 80 KB]
+  unsigned char* small_ws = nullptr; // single-launch path: [tickets 4 KB | partial records 384 KB]
   bool small_on = true;
   int wins_algo = 0;                // 0 auto, 1 direct comparison, 2 binary search on sorted rows,
                                     // 3 lane-per-row merge of sorted rows
@@ -100,7 +100,7 @@ inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline int elem_bytes(kb_dtype dt) { return dt == KB_F32 ? 4 : (dt == KB_F8E4M3 || dt == KB_F8E5M2) ? 1 : 2; }
 inline bool known_dtype(int dt) { return dt >= KB_F32 && dt <= KB_F8E5M2; }
 constexpr size_t kSmallTicketBytes = 4096;
-constexpr size_t kSmallMaxPartials = 2048;
+constexpr size_t kSmallMaxPartials = 8192;
 constexpr size_t kSmallWsBytes = kSmallTicketBytes + kSmallMaxPartials * sizeof(Acc);
 
 // Event pair around one launch of an instrumented kernel (no-op unless timing is on).
@@ -902,7 +902,7 @@ extern "C" kb_status kb_screen_multi(kb_ctx* ctx, uint32_t G, const void* const*
     for (uint32_t k = 0; k < h_K[g]; ++k) {
       if (rows >= (uint32_t)kMultiMaxRows || blocks + nb > kSmallMaxPartials)
         return fail(ctx, KB_ERR_UNSUPPORTED,
-                    "kb_screen_multi: more than %d candidates or %zu blocks of 4096 elements; "
+                    "kb_screen_multi: more than %d candidates or %zu blocks of 1024 elements; "
                     "call kb_screen per group", kMultiMaxRows, kSmallMaxPartials);
       const void* c = h_cands[rows];
       if (!c) return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen_multi: candidate %u is NULL", rows);

@@ -798,12 +798,12 @@ __global__ void __launch_bounds__(256) screen_scout_kernel(const void* __restric
 // ---------------------------------------------------------------------------
 // Small problems (the latency-bound regime: a few candidates of at most a few hundred
 // thousand elements, e.g. 21 candidates of a 2048-element mat-vec output): ONE launch.
-// Candidate pointers travel as kernel arguments; block (bx, k) classifies 4096 elements
+// Candidate pointers travel as kernel arguments; block (bx, k) classifies 1024 elements
 // exactly and writes a partial record; the last block of candidate k to finish (a
 // self-resetting ticket per candidate) merges the partials and writes the result.
 // Nothing has to be zeroed beforehand and no atomics touch the accumulators.
 // ---------------------------------------------------------------------------
-constexpr unsigned int kSmallPerBlock = 4096;
+constexpr unsigned int kSmallPerBlock = 1024;
 struct SmallParams {
   const void* ref;
   Acc* partials;            // [K][nb]
@@ -897,7 +897,7 @@ __device__ __forceinline__ void small_block(const void* ref, const void* cand, u
       const unsigned int rv = __ldcg(&q->rel);
       rel = rv > rel ? rv : rel;
     }
-    // each partial count is <= 4096 and nb <= 2048: the 32-bit adds below cannot overflow
+    // each partial count is <= 1024 and nb <= 8192: the 32-bit adds below cannot overflow
     const unsigned long long tm = warp_add_u32((unsigned int)mism);
     const unsigned long long tn = warp_add_u32((unsigned int)nan);
     const unsigned long long ti = warp_add_u32((unsigned int)inf);
