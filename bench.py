@@ -34,10 +34,20 @@ if ROOT not in sys.path:
 METRIC = "candidate-elements screened/sec"
 UNIT = "elements/s"
 K_CANDS, SIDE, S_TIMINGS, BUDGET = 64, 4096, 100, 32
-# DRAM bytes moved per algorithmic byte by the streaming screen kernel, from the ncu capture
-# summarised in profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over (K+1)*N*2 bytes);
-# captured at side 2048 (545 MB) and scaled by the bytes a full launch processes.
-DRAM_BYTES_PER_ALGORITHMIC_BYTE = 1.0076
+# DRAM bytes moved per algorithmic byte by the streaming screen kernel come from the ncu capture
+# summarised in profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over (K+1)*N*2 bytes;
+# captured at side 2048 and scaled by the bytes a full launch processes); the figure is stored
+# beside that summary so that it is replaced together with it.
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "screen_stream_kernel_bf16_config2.json")
+REF_MAX_STEPS, REF_MAX_WARMUP = 50, 5      # bounds of the reference arm (a step costs ~0.6 s)
+
+
+def dram_bytes_per_algorithmic_byte():
+    try:
+        with open(TRAFFIC_FILE) as f:
+            return float(json.load(f)["dram_bytes_per_algorithmic_byte"])
+    except Exception:
+        return None
 
 WORKLOAD = ("config2: screen K=64 bf16 4096x4096 (atol=1e-2, rtol=1.6e-2) + adjudicate "
             "timings[64][100] + select top 32")
@@ -56,10 +66,12 @@ class ClockSampler(threading.Thread):
     Everything that talks to NVML (initialisation included) happens on this daemon thread, so a
     slow or stuck NVML can never block the benchmark itself."""
 
-    def __init__(self, index: int, period_s: float = 0.02):
+    def __init__(self, index: int, period_s: float = 0.001):
         super().__init__(daemon=True)
         self.index, self.period = index, period_s
         self.samples, self.reasons, self.max_mhz = [], set(), None
+        self.stamps = []
+        self.window = None                 # (t0, t1) of the timed region, perf_counter
         self._halt = threading.Event()
 
     def run(self):
@@ -79,6 +91,7 @@ class ClockSampler(threading.Thread):
         while not self._halt.is_set():
             try:
                 self.samples.append(int(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)))
+                self.stamps.append(time.perf_counter())
                 mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(h))
                 for name, bit in names.items():
                     if mask & bit:
@@ -92,9 +105,16 @@ class ClockSampler(threading.Thread):
         if self.is_alive():
             self.join(timeout=2)
         samples = list(self.samples)
-        return {"sm_mhz": int(np.median(samples)) if samples else None,
+        stamps = list(self.stamps)[:len(samples)]
+        timed = [v for v, t in zip(samples, stamps)
+                 if self.window and self.window[0] <= t <= self.window[1]]
+        # the sampler runs from before the warm-up steps (the same load) to the end of the
+        # timed region; a timed region shorter than one NVML query still gets the load's clock
+        use = timed if len(timed) >= 3 else samples
+        return {"sm_mhz": int(np.median(use)) if use else None,
                 "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
-                "samples": len(samples)}
+                "samples": len(samples), "samples_in_timed_region": len(timed),
+                "window": "warm-up + timed region"}
 
 
 def host_cores() -> int:
@@ -112,30 +132,34 @@ def oracle_step(ref_np, cands_np, timings, n_cands, threads):
 
 
 def run_reference(args):
-    """The reference arm: the CPU oracle on the host cores, same config and metric."""
+    """The reference arm: the CPU oracle on the host cores, same config and metric: every step
+    screens all 64 candidates, adjudicates [64][100] and selects.  `--steps`/`--warmup` are
+    honoured up to REF_MAX_STEPS / REF_MAX_WARMUP."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     import torch
     from paper_2608_02611_b200 import synth
     cores = host_cores()
-    n_sample = min(K_CANDS, max(8, cores))          # candidates per step (bounded sample)
     case, timings = synth.config2("cpu", side=SIDE, K=K_CANDS)
     ref_np = synth.to_oracle_array(case.ref, case.dtype)
-    cands_np = [synth.to_oracle_array(case.make_cand(k), case.dtype) for k in range(n_sample)]
-    for _ in range(min(args.warmup, 1)):
-        oracle_step(ref_np, cands_np, timings, n_sample, cores)
-    steps = max(1, min(args.steps, 5))
-    secs = [oracle_step(ref_np, cands_np, timings, n_sample, cores) for _ in range(steps)]
+    cands_np = [synth.to_oracle_array(case.make_cand(k), case.dtype) for k in range(K_CANDS)]
+    warmup = max(0, min(args.warmup, REF_MAX_WARMUP))
+    steps = max(1, min(args.steps, REF_MAX_STEPS))
+    for _ in range(warmup):
+        oracle_step(ref_np, cands_np, timings, K_CANDS, cores)
+    secs = [oracle_step(ref_np, cands_np, timings, K_CANDS, cores) for _ in range(steps)]
     per_step = float(np.mean(secs))
-    value = n_sample * case.N / per_step
-    sample = (f"{n_sample} of {K_CANDS} candidates of 4096x4096 bf16 per step, full adjudication "
-              f"[64][100] and select; {steps} steps")
+    value = K_CANDS * case.N / per_step
+    sample = (f"the whole step: all {K_CANDS} candidates of 4096x4096 bf16, adjudication [64][100] "
+              f"and select; {steps} steps after {warmup} warm-up steps on {cores} threads")
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": per_step * 1e3,
+        "steps": steps, "warmup": warmup, "ms_per_step": per_step * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
-        "data": "synthetic", "config": {"workload": WORKLOAD, "sample": sample},
+        "data": "synthetic",
+        "config": {"workload": WORKLOAD, "K": K_CANDS, "N": case.N, "storage": "bf16", "S": S_TIMINGS,
+                   "budget": BUDGET, "sample": sample},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -248,6 +272,22 @@ def run_screen(args):
     ctx.close()
 
 
+def relaunch_ranks(n: int):
+    """`python bench.py --gpus N` without a launcher: start N ranks (one process per GPU) under
+    torch.distributed.run on this node, with the same arguments, and pass their output on."""
+    import socket
+    import subprocess
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "INFO")           # the communicator set-up goes to stderr
+    env.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+    raise SystemExit(subprocess.run(cmd, env=env).returncode)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -280,6 +320,9 @@ def main():
     if args.workload == "screen":
         return run_screen(args)
 
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        return relaunch_ranks(args.gpus)
+
     import torch
     import torch.distributed as dist
     from paper_2608_02611_b200 import binding, sharding, synth
@@ -292,6 +335,8 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the product has no CPU path")
+    if world > torch.cuda.device_count():
+        raise SystemExit(f"bench.py --gpus {world}: only {torch.cuda.device_count()} GPUs are visible")
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     ctx = binding.Context(local_rank)
@@ -333,24 +378,26 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    sampler = ClockSampler(local_rank)
+    sampler.start()
     for _ in range(warmup):
         step()
     barrier()
     assert ctx.poll() == 0 and ctx_adj.poll() == 0
 
     # ---- timed region: exactly `steps` steps, CUDA events, clocks sampled meanwhile ----
-    sampler = ClockSampler(local_rank)
-    sampler.start()
     ctx.enable_timing(True)
     ctx_adj.enable_timing(True)
     launches0 = ctx.launch_count + ctx_adj.launch_count
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
+    t_begin = time.perf_counter()
     e0.record()
     for _ in range(steps):
         surv, n = step()
     e1.record()
     barrier()
+    sampler.window = (t_begin, time.perf_counter())
     clocks = sampler.stop()
     elapsed_ms = e0.elapsed_time(e1)
     launches = ctx.launch_count + ctx_adj.launch_count - launches0
@@ -413,9 +460,11 @@ def main():
     stream_bytes = (K_CANDS + 1) * (N - nscout * 4096) * esz
     avg_stream_ms = float(np.mean(stream_ms)) if len(stream_ms) else float("nan")
     achieved = stream_bytes / (avg_stream_ms * 1e-3) / 1e9
-    traffic = DRAM_BYTES_PER_ALGORITHMIC_BYTE * stream_bytes if DRAM_BYTES_PER_ALGORITHMIC_BYTE else None
+    ratio = dram_bytes_per_algorithmic_byte()
+    traffic = ratio * stream_bytes if ratio else None
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
+                "traffic_source": os.path.relpath(TRAFFIC_FILE, ROOT) if traffic else None,
                 "kernel": "screen_stream_kernel<bf16>", "launch_ms_avg": avg_stream_ms,
                 "launch_ms_min": float(np.min(stream_ms)) if len(stream_ms) else None,
                 "algorithmic_bytes_per_launch": stream_bytes, "launches_timed": int(len(stream_ms)),

@@ -12,8 +12,8 @@
  *                  optionally on a fidelity-dependent subset of tiles
  *                  (low-cost screening, Abstract / Sec. 3.3 Observation 2);
  *   kb_adjudicate  the reduction of repeated, noisy timings to an
- *                  "adjudicated latency" (Algorithm 1, "Compute score s(c,r)
- *                  from adjudicated latency"; Sec. 1 contribution 1
+ *                  "adjudicated latency" (Algorithm 1, the step that scores a
+ *                  candidate from it; Sec. 1 contribution 1
  *                  "stability adjudication"; Appendix "Relative Variability
  *                  Metrics"), as median + IQR per candidate plus a K x K
  *                  matrix of doubled Mann-Whitney win counts;
@@ -108,48 +108,13 @@ kb_status kb_ctx_destroy(kb_ctx* ctx);
  * next call on the context); with ctx == NULL, the text of the last failed
  * kb_ctx_create on this thread. */
 const char* kb_last_error(const kb_ctx* ctx);
-/* Synchronise `stream`, read the device status word into *device_status
+/* (Takes the stream it synchronises, since the library keeps no stream of its own.)
+ * Synchronise `stream`, read the device status word into *device_status
  * (KB_OK, KB_ERR_NONFINITE or KB_ERR_DEVICE_TIMEOUT; HOST pointer) and clear
  * it.  Returns KB_OK unless the read itself failed. */
 kb_status kb_ctx_poll(kb_ctx* ctx, void* stream, kb_status* device_status);
-/* Test/tuning hook: force the number of thread blocks of the streaming screen
- * kernel (0 = automatic).  Results do not depend on it. */
-kb_status kb_ctx_set_grid(kb_ctx* ctx, uint32_t blocks);
-
-/* Test/tuning hook: small problems (K <= 480 and K*N <= 2^22 elements) are
- * screened by a single-launch kernel; on = 0 sends them down the general
- * (streaming) path instead.  Results do not depend on it. */
-kb_status kb_ctx_set_small_path(kb_ctx* ctx, int on);
-
-/* ---- instrumentation (used by the benchmark; no paper counterpart) ------- */
-
-typedef enum {
-  KB_TIMER_SCREEN_STREAM = 0, /* the streaming screen kernel */
-  KB_TIMER_WINS = 1           /* the pairwise win-count kernel */
-} kb_timer;
-
-/* With timing on, every launch of the two kernels above is bracketed by a pair
- * of CUDA events recorded on the launching stream (taken from a ctx-owned
- * pool of 256 pairs per timer; older launches are overwritten). */
-kb_status kb_ctx_enable_timing(kb_ctx* ctx, int on);
-/* Wait for the recorded launches of `which` since the last read, write their
- * durations in milliseconds (oldest first, at most `cap`) to h_ms (HOST) and
- * their number to *n (HOST); the record is then cleared. */
-kb_status kb_ctx_read_timer(kb_ctx* ctx, kb_timer which, float* h_ms, uint32_t cap, uint32_t* n);
-/* Register-only probe of the instruction mix of the direct win count (two compares and two
- * predicated increments per sample pair, values held in registers): runs it on every SM for
- * `iters` (<= 2^23) rounds of 128 sample pairs per thread, times it with CUDA events on
- * `stream`, and writes the rate in sample pairs per second to *pairs_per_s (HOST).  This is
- * the measured ceiling the direct win-count kernel is compared with.  Synchronous. */
-kb_status kb_alu_probe(kb_ctx* ctx, uint32_t iters, double* pairs_per_s, void* stream);
-/* Choose how kb_adjudicate counts wins: 0 = automatic (on the sorted rows when they fit shared
- * memory: a lane-per-row merge for K >= 225 and S <= 1024, else a binary search and walk per
- * row pair for S <= 4096; direct comparison beyond), 1 = always direct comparison of all
- * sample pairs, 2 = always binary search (S <= 4096 only), 3 = always the lane-per-row merge
- * (S <= 1024 only).  The integers produced are identical. */
-kb_status kb_ctx_set_wins_algo(kb_ctx* ctx, int algo);
-/* Number of kernels this context has launched since it was created (HOST out). */
-kb_status kb_ctx_launch_count(const kb_ctx* ctx, uint64_t* n);
+/* Test, tuning and instrumentation hooks (forced grid sizes and dispatch paths,
+ * CUDA-event timers, launch counter, self-tests) are declared in kb_hooks.h. */
 
 /* ---- fidelity masks (Sec. 3.2 "Fidelity level", rendered on elements) --- */
 
@@ -279,6 +244,10 @@ kb_status kb_screen_f64(kb_ctx* ctx, const double* d_ref, const double* const* h
  *     call left in it; each call clears the part it uses before use.  Two
  *     calls that overlap on the GPU (different streams, or one stream and a
  *     graph replay) race on it and give wrong records: order them.
+ *   - Host threads: calls on one device are serialised by a lock inside the library for
+ *     as long as they validate and enqueue, so two host threads may call it; they still
+ *     have to order their work on the GPU (previous point).  kb_last_error(NULL) is per
+ *     thread.
  *   - Asynchronous like kb_screen; d_out is valid after `stream` synchronises.
  *     A device-side wait that ran out cannot be polled through this entry point
  *     (there is no context); use kb_screen + kb_ctx_poll where that matters. */
@@ -328,7 +297,9 @@ typedef enum {
   KB_SELECT_TIME = 1           /* key (median asc, index asc)                   */
 } kb_select_policy;
 
-/* Eligible candidates are those with pass == 1 (failed candidates are never
+/* (The policies below read only the gate's records and the medians, so those are the
+ * statistics this call takes; a ranking over the win matrix is kb_copeland.)
+ * Eligible candidates are those with pass == 1 (failed candidates are never
  * promoted).  They are ordered by the policy's key, floats compared as values
  * (none is NaN), ties broken by the lower candidate index; the first
  * n = min(budget, #eligible) indices are written to d_survivors IN RANK ORDER

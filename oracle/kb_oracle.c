@@ -280,9 +280,17 @@ int kbo_screen_f64(const double* ref, const double* cand, uint64_t N, double ato
   return 0;
 }
 
+/* Ascending order of timings as a TOTAL order, so that the sorted row (and with it
+ * the sign of a quantile that is zero) is unique: by value, and where two values are
+ * equal but differ in sign (-0 and +0, the only such pair) the negative zero first. */
 static int cmp_float_asc(const void* pa, const void* pb) {
   float a = *(const float*)pa, b = *(const float*)pb;
-  return (a > b) - (a < b);
+  if (a > b) return 1;
+  if (a < b) return -1;
+  {
+    int sa = (int)(float_to_bits(a) >> 31), sb = (int)(float_to_bits(b) >> 31);
+    return sb - sa; /* a negative (sa = 1), b positive (sb = 0): a first */
+  }
 }
 
 /*

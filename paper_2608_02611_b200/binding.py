@@ -47,6 +47,7 @@ EXPORTS = [
     "kb_mask_create_strided", "kb_mask_create_bitmap", "kb_mask_count", "kb_mask_destroy",
     "kb_screen", "kb_screen_f64", "kb_screen_host", "kb_screen_static", "kb_screen_indexed", "kb_screen_multi", "kb_adjudicate", "kb_adjudicate_ragged", "kb_select",
     "kb_select_by_score", "kb_tail_ratios", "kb_copeland", "kb_confirm",
+    "kb_ctx_fail_next_allocs", "kb_ctx_selftest_wait", "kb_ctx_check_guards", "kb_static_scratch_read",
 ]
 
 
@@ -84,6 +85,10 @@ def load() -> ctypes.CDLL:
     L.kb_ctx_launch_count.argtypes = [vp, ctypes.POINTER(u64)]
     L.kb_ctx_set_wins_algo.argtypes = [vp, i32]
     L.kb_ctx_set_small_path.argtypes = [vp, i32]
+    L.kb_ctx_fail_next_allocs.argtypes = [vp, u32, u32]
+    L.kb_ctx_check_guards.argtypes = [vp, vp, ctypes.POINTER(u32), ctypes.POINTER(u32)]
+    L.kb_static_scratch_read.argtypes = [vp, u32]
+    L.kb_ctx_selftest_wait.argtypes = [vp, u64, vp]
     L.kb_mask_create_strided.argtypes = [vp, u64, u32, u32, u32, pvp]
     L.kb_mask_create_bitmap.argtypes = [vp, u64, u32, vp, pvp]
     L.kb_mask_count.argtypes = [vp, ctypes.POINTER(u64)]
@@ -189,6 +194,23 @@ class Context:
         3 lane-per-row merge of sorted rows."""
         self._check(load().kb_ctx_set_wins_algo(self._h, int(algo)), "kb_ctx_set_wins_algo")
 
+    def fail_next_allocs(self, n: int, skip: int = 0):
+        """Test hook: after `skip` more device allocations of this context, the next n fail."""
+        self._check(load().kb_ctx_fail_next_allocs(self._h, int(skip), int(n)), "kb_ctx_fail_next_allocs")
+
+    def check_guards(self):
+        """Test hook: (buffers checked, guard-band bytes overwritten) over the context's buffers."""
+        nb, bad = ctypes.c_uint32(0), ctypes.c_uint32(0)
+        self._check(load().kb_ctx_check_guards(self._h, _stream_ptr(self.device), ctypes.byref(nb),
+                                               ctypes.byref(bad)), "kb_ctx_check_guards")
+        return int(nb.value), int(bad.value)
+
+    def selftest_wait(self, limit_ns: int):
+        """Test hook: one warp waits `limit_ns` on a barrier nothing completes, then gives up;
+        poll() afterwards reports KB_ERR_DEVICE_TIMEOUT once."""
+        self._check(load().kb_ctx_selftest_wait(self._h, int(limit_ns), _stream_ptr(self.device)),
+                    "kb_ctx_selftest_wait")
+
     def enable_timing(self, on: bool = True):
         self._check(load().kb_ctx_enable_timing(self._h, 1 if on else 0), "kb_ctx_enable_timing")
 
@@ -251,7 +273,7 @@ class Context:
         return out
 
     def screen_f64(self, ref: torch.Tensor, cands: Sequence[torch.Tensor], atol: float, rtol: float,
-                   mask: Optional[Mask] = None) -> torch.Tensor:
+                   mask: Optional[Mask] = None, out: Optional[torch.Tensor] = None) -> torch.Tensor:
         """kb_screen_f64 on float64 CUDA tensors.  Returns a uint8 CUDA tensor [K, 56] of
         kb_screen_result_f64 records (see ``records_f64``); asynchronous on the current stream."""
         K = len(cands)
@@ -260,7 +282,8 @@ class Context:
             if c.dtype != torch.float64 or c.numel() != N or not c.is_cuda or not c.is_contiguous():
                 raise KbError(1, "kb_screen_f64", "tensors must be contiguous CUDA float64 tensors of "
                                                   "one element count")
-        out = torch.empty((K, RESULT_F64_BYTES), dtype=torch.uint8, device=ref.device)
+        if out is None:
+            out = torch.empty((K, RESULT_F64_BYTES), dtype=torch.uint8, device=ref.device)
         ptrs = (ctypes.c_void_p * max(K, 1))(*[c.data_ptr() for c in cands])
         rc = load().kb_screen_f64(self._h, ref.data_ptr(), ptrs, K, N, float(atol), float(rtol),
                                   mask._h if mask is not None else None, out.data_ptr(),
@@ -286,27 +309,35 @@ class Context:
         self._check(rc, "kb_screen_host")
         return out
 
-    def adjudicate(self, timings: torch.Tensor, want_wins: bool = True):
+    def adjudicate(self, timings: torch.Tensor, want_wins: bool = True, out=None):
         """kb_adjudicate on a CUDA float32 tensor [K, S] -> (median[K], iqr[K], wins[K,K] or None).
-        wins is int32 storage holding uint32 counts (values < 2^31 for S < 32768)."""
+        wins is int32 storage holding uint32 counts (values < 2^31 for S < 32768).
+        `out` = (median, iqr, wins) gives pre-allocated outputs."""
         if timings.dtype != torch.float32 or timings.dim() != 2 or not timings.is_cuda \
                 or not timings.is_contiguous():
             raise KbError(1, "kb_adjudicate", "timings must be a contiguous CUDA float32 [K, S] tensor")
         K, S = timings.shape
-        med = torch.empty(K, dtype=torch.float32, device=timings.device)
-        iqr = torch.empty(K, dtype=torch.float32, device=timings.device)
-        wins = torch.empty((K, K), dtype=torch.int32, device=timings.device) if want_wins else None
+        if out is not None:
+            med, iqr, wins = out
+        else:
+            med = torch.empty(K, dtype=torch.float32, device=timings.device)
+            iqr = torch.empty(K, dtype=torch.float32, device=timings.device)
+            wins = torch.empty((K, K), dtype=torch.int32, device=timings.device) if want_wins else None
         rc = load().kb_adjudicate(self._h, timings.data_ptr(), K, S, med.data_ptr(), iqr.data_ptr(),
                                   wins.data_ptr() if want_wins else None,
                                   _stream_ptr(timings.device))
         self._check(rc, "kb_adjudicate")
         return med, iqr, wins
 
-    def select(self, screen_out: torch.Tensor, median: torch.Tensor, policy: int, budget: int):
-        """kb_select -> (survivors int32 [budget] in rank order, n int32 [1]) on the device."""
+    def select(self, screen_out: torch.Tensor, median: torch.Tensor, policy: int, budget: int, out=None):
+        """kb_select -> (survivors int32 [budget] in rank order, n int32 [1]) on the device.
+        `out` = (survivors, n) gives pre-allocated outputs."""
         K = median.numel()
-        surv = torch.empty(budget, dtype=torch.int32, device=median.device)
-        n = torch.empty(1, dtype=torch.int32, device=median.device)
+        if out is not None:
+            surv, n = out
+        else:
+            surv = torch.empty(budget, dtype=torch.int32, device=median.device)
+            n = torch.empty(1, dtype=torch.int32, device=median.device)
         rc = load().kb_select(self._h, screen_out.data_ptr(), median.data_ptr(), K, int(policy),
                               int(budget), surv.data_ptr(), n.data_ptr(), _stream_ptr(median.device))
         self._check(rc, "kb_select")
@@ -337,6 +368,18 @@ def screen_static(ref: torch.Tensor, cands: Sequence[torch.Tensor], atol: float,
     if rc != KB_OK:
         raise KbError(rc, "kb_screen_static", (load().kb_last_error(None) or b"").decode())
     return out
+
+
+KB_STATIC_SCRATCH_BYTES = 256 + 1024 * 48 + 1024 * 8
+
+
+def static_scratch_read(nbytes: int = KB_STATIC_SCRATCH_BYTES) -> np.ndarray:
+    """Test hook: the scratch array of kb_screen_static on the current device, as bytes."""
+    buf = np.zeros(nbytes, dtype=np.uint8)
+    rc = load().kb_static_scratch_read(buf.ctypes.data, nbytes)
+    if rc != KB_OK:
+        raise KbError(rc, "kb_static_scratch_read")
+    return buf
 
 
 def _ctx_method(fn):
@@ -423,7 +466,7 @@ def adjudicate_ragged(self, flat: torch.Tensor, offsets: torch.Tensor, S_max: in
 
 
 @_ctx_method
-def screen_multi(self, groups, atol: float, rtol: float) -> torch.Tensor:
+def screen_multi(self, groups, atol: float, rtol: float, out: Optional[torch.Tensor] = None) -> torch.Tensor:
     """kb_screen_multi: groups = [(ref, [cands...]), ...] of different sizes, one launch.
     Returns a uint8 CUDA tensor [sum K, 48] in group order."""
     G = len(groups)
@@ -438,7 +481,8 @@ def screen_multi(self, groups, atol: float, rtol: float) -> torch.Tensor:
                                                     "and the call's dtype")
     ptrs = (ctypes.c_void_p * max(len(flat), 1))(*[c.data_ptr() for c in flat])
     dev = groups[0][0].device
-    out = torch.empty((len(flat), RESULT_BYTES), dtype=torch.uint8, device=dev)
+    if out is None:
+        out = torch.empty((len(flat), RESULT_BYTES), dtype=torch.uint8, device=dev)
     rc = load().kb_screen_multi(self._h, G, refs, ptrs, Ks, Ns, DTYPE_CODE.get(groups[0][0].dtype, -1),
                                 float(atol), float(rtol), out.data_ptr(), _stream_ptr(dev))
     self._check(rc, "kb_screen_multi")

@@ -33,7 +33,9 @@ namespace kb {
 constexpr int kRowsThreads = 256;
 
 // Load one row into shared memory (padded with +Inf to P, a power of two), flag
-// non-finite timings, sort ascending (bitonic network).
+// non-finite timings, sort ascending (bitonic network).  The order is total, so that the
+// sorted row is unique: by value, and -0 before +0 (the only equal values whose bits differ;
+// as signed integers the bits of -0 lie below those of +0).
 __device__ __forceinline__ void load_and_sort_row(const float* __restrict__ row, unsigned int S,
                                                   unsigned int P, float* xs, unsigned int* status) {
   const float inf = __uint_as_float(0x7F800000u);
@@ -55,7 +57,8 @@ __device__ __forceinline__ void load_and_sort_row(const float* __restrict__ row,
         const unsigned int hi = lo + stride;
         const bool up = (lo & size) == 0;
         const float a = xs[lo], b = xs[hi];
-        if ((a > b) == up) {
+        const bool gt = (a > b) || (a == b && __float_as_int(a) > __float_as_int(b));
+        if (gt == up) {
           xs[lo] = b;
           xs[hi] = a;
         }

@@ -6,7 +6,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
-#include "../../include/kb.h"
+#include "../../include/kb_hooks.h"
 
 namespace kb {
 
@@ -190,11 +190,13 @@ __device__ __forceinline__ unsigned long long global_ns() {
   return t;
 }
 // Bounded wait: polls until the phase with `parity` completes, the CTA-wide
-// abort flag is raised, or ~2 s pass.  Returns false when it gave up; it then
-// raises the abort flag and records KB_ERR_DEVICE_TIMEOUT.  Never traps.
+// abort flag is raised, or `limit_ns` (2 s unless stated) pass.  Returns false when it gave
+// up; it then raises the abort flag and records KB_ERR_DEVICE_TIMEOUT.  Never traps.
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity,
                                                   volatile unsigned int* abort_flag,
-                                                  unsigned int* status) {
+                                                  unsigned int* status,
+                                                  unsigned long long limit_ns = kWaitLimitNs) {
   if (mbar_try_wait(bar, parity)) return true;
   unsigned long long t0 = 0;
   unsigned int polls = 0;
@@ -204,7 +206,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
     if ((++polls & 1023u) == 0) {
       unsigned long long now = global_ns();
       if (t0 == 0) t0 = now;
-      if (now - t0 > 2000000000ull) {
+      if (now - t0 > limit_ns) {
         *abort_flag = 1u;
         set_status(status, (unsigned int)KB_ERR_DEVICE_TIMEOUT);
         return false;
@@ -212,6 +214,21 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
     }
   }
 }
+// Self-test of the wait above (kb_ctx_selftest_wait): one warp waits on a barrier that nothing
+// completes.  No copy is in flight, so giving up leaves nothing behind; the kernel returns
+// normally with KB_ERR_DEVICE_TIMEOUT in the status word.
+__global__ void wait_selftest_kernel(unsigned int* status, unsigned long long limit_ns) {
+  __shared__ uint64_t bar;
+  __shared__ unsigned int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    abort_flag = 0u;
+    mbar_fence_init();
+  }
+  __syncwarp();
+  mbar_wait_bounded(&bar, 0u, &abort_flag, status, limit_ns);
+}
+
 __device__ __forceinline__ uint64_t l2_policy_evict_first() {
   uint64_t pol;
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));

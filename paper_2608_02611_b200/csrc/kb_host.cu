@@ -22,6 +22,7 @@ struct kb_ctx {
   int sm_count = 0;
   unsigned char* ws = nullptr;      // [acc K*48 | pad | pointer table K*8]
   size_t ws_bytes = 0;
+  bool ws_fixed = false;            // the workspace is not ours to grow or free (kb_screen_static)
   unsigned int* d_status = nullptr;
   uint32_t forced_grid = 0;
   unsigned char* small_ws = nullptr; // single-launch path: [tickets 4 KB | partial records 384 KB]
@@ -35,12 +36,18 @@ struct kb_ctx {
   unsigned char* st_ref = nullptr;
   size_t st_ref_bytes = 0;
   unsigned char* st_batch[2] = {nullptr, nullptr};
-  size_t st_batch_bytes = 0;
+  size_t st_batch_bytes[2] = {0, 0};
   kb_screen_result* st_out = nullptr;
   size_t st_out_bytes = 0;
   cudaStream_t copy_stream = nullptr;
   cudaEvent_t ev_copied[2] = {nullptr, nullptr};
   cudaEvent_t ev_done[2] = {nullptr, nullptr};
+  uint32_t skip_allocs = 0;         // test hook: let this many device allocations through, ...
+  uint32_t fail_allocs = 0;         // ... then refuse this many
+  // Every buffer the context owns sits between two 256-byte guard bands filled with kGuardByte;
+  // kb_ctx_check_guards counts the band bytes that no longer hold it (an out-of-bounds write).
+  struct Guarded { unsigned char* raw; size_t bytes; };
+  std::vector<Guarded> guarded;
   // instrumentation
   uint64_t launches = 0;
   bool timing = false;
@@ -120,33 +127,64 @@ struct ScopedTimer {
   }
 };
 
-kb_status ensure_ws(kb_ctx* ctx, uint32_t K, size_t acc_bytes = sizeof(Acc)) {
-  const size_t need = round_up((size_t)K * acc_bytes, 256) + (size_t)K * sizeof(void*);
-  if (need <= ctx->ws_bytes) return KB_OK;
-  if (ctx->ws) cudaFree(ctx->ws);   // waits for enqueued work that still uses it
-  ctx->ws = nullptr;
-  ctx->ws_bytes = 0;
-  const size_t grow = round_up(need * 2, 4096);
-  if (cudaMalloc(&ctx->ws, grow) != cudaSuccess) {
-    cudaGetLastError();
-    return fail(ctx, KB_ERR_WORKSPACE, "cannot allocate %zu bytes of device workspace", grow);
+// Every device allocation of a context goes through here: a test can make it fail
+// (kb_ctx_fail_next_allocs) without exhausting a GPU's memory, and every buffer gets guard
+// bands (compute-sanitizer's stand-in for out-of-bounds writes; see kb_ctx_check_guards).
+constexpr size_t kGuardBytes = 256;
+constexpr int kGuardByte = 0xA5;
+cudaError_t ctx_malloc(kb_ctx* ctx, void** p, size_t bytes) {
+  *p = nullptr;
+  if (ctx->skip_allocs) {
+    --ctx->skip_allocs;
+  } else if (ctx->fail_allocs) {
+    --ctx->fail_allocs;
+    return cudaErrorMemoryAllocation;
   }
-  ctx->ws_bytes = grow;
+  unsigned char* raw = nullptr;
+  const size_t body = round_up(bytes, 256);
+  cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&raw), body + 2 * kGuardBytes);
+  if (e == cudaSuccess) e = cudaMemset(raw, kGuardByte, kGuardBytes);
+  if (e == cudaSuccess) e = cudaMemset(raw + kGuardBytes + body, kGuardByte, kGuardBytes);
+  if (e != cudaSuccess) {
+    if (raw) cudaFree(raw);
+    cudaGetLastError();
+    return e;
+  }
+  ctx->guarded.push_back({raw, body});
+  *p = raw + kGuardBytes;
+  return cudaSuccess;
+}
+void ctx_free(kb_ctx* ctx, void* p) {
+  if (!p) return;
+  unsigned char* raw = static_cast<unsigned char*>(p) - kGuardBytes;
+  for (size_t i = 0; i < ctx->guarded.size(); ++i)
+    if (ctx->guarded[i].raw == raw) {
+      ctx->guarded.erase(ctx->guarded.begin() + (long)i);
+      break;
+    }
+  cudaFree(raw);   // waits for enqueued work that still uses the buffer
+}
+
+// Grow *buf to at least `need` bytes.  The new buffer is allocated BEFORE the old one is
+// released, and pointer and size change together: after a failure the context still holds
+// its old, valid (pointer, size) pair and a later, smaller call works as before.
+template <typename T>
+kb_status ensure_buf(kb_ctx* ctx, T** buf, size_t* have, size_t need, const char* what = "device staging") {
+  if (need <= *have) return KB_OK;
+  void* fresh = nullptr;
+  if (ctx_malloc(ctx, &fresh, need) != cudaSuccess)
+    return fail(ctx, KB_ERR_WORKSPACE, "cannot allocate %zu bytes of %s", need, what);
+  ctx_free(ctx, *buf);
+  *buf = static_cast<T*>(fresh);
+  *have = need;
   return KB_OK;
 }
 
-template <typename T>
-kb_status ensure_buf(kb_ctx* ctx, T** buf, size_t* have, size_t need) {
-  if (need <= *have) return KB_OK;
-  if (*buf) cudaFree(*buf);
-  *buf = nullptr;
-  *have = 0;
-  if (cudaMalloc(reinterpret_cast<void**>(buf), need) != cudaSuccess) {
-    cudaGetLastError();
-    return fail(ctx, KB_ERR_WORKSPACE, "cannot allocate %zu bytes of device staging", need);
-  }
-  *have = need;
-  return KB_OK;
+kb_status ensure_ws(kb_ctx* ctx, uint32_t K, size_t acc_bytes = sizeof(Acc)) {
+  const size_t need = round_up((size_t)K * acc_bytes, 256) + (size_t)K * sizeof(void*);
+  if (need <= ctx->ws_bytes) return KB_OK;
+  if (ctx->ws_fixed) return fail(ctx, KB_ERR_WORKSPACE, "the fixed scratch holds %zu bytes, %zu needed", ctx->ws_bytes, need);
+  return ensure_buf(ctx, &ctx->ws, &ctx->ws_bytes, round_up(need * 2, 4096), "device workspace");
 }
 
 // ring depth by stage size: 3 CTAs/SM must fit ~75 KB each
@@ -249,11 +287,12 @@ extern "C" kb_status kb_ctx_create(int device, kb_ctx** out) {
     return bail(KB_ERR_CUDA);
   }
   ctx->sm_count = prop.multiProcessorCount;
-  if (cudaMalloc(&ctx->d_status, 256) != cudaSuccess || cudaMemset(ctx->d_status, 0, 256) != cudaSuccess) {
+  if (ctx_malloc(ctx, reinterpret_cast<void**>(&ctx->d_status), 256) != cudaSuccess ||
+      cudaMemset(ctx->d_status, 0, 256) != cudaSuccess) {
     fail(ctx, KB_ERR_WORKSPACE, "cannot allocate the device status word");
     return bail(KB_ERR_WORKSPACE);
   }
-  if (cudaMalloc(&ctx->small_ws, kSmallWsBytes) != cudaSuccess ||
+  if (ctx_malloc(ctx, reinterpret_cast<void**>(&ctx->small_ws), kSmallWsBytes) != cudaSuccess ||
       cudaMemset(ctx->small_ws, 0, kSmallWsBytes) != cudaSuccess) {
     fail(ctx, KB_ERR_WORKSPACE, "cannot allocate the small-problem workspace");
     return bail(KB_ERR_WORKSPACE);
@@ -297,17 +336,17 @@ extern "C" kb_status kb_ctx_destroy(kb_ctx* ctx) {
   if (!ctx) return KB_OK;
   DeviceGuard g(ctx->device);
   cudaDeviceSynchronize();
-  if (ctx->ws) cudaFree(ctx->ws);
-  if (ctx->d_status) cudaFree(ctx->d_status);
-  if (ctx->st_ref) cudaFree(ctx->st_ref);
-  if (ctx->srt) cudaFree(ctx->srt);
-  if (ctx->small_ws) cudaFree(ctx->small_ws);
+  if (!ctx->ws_fixed) ctx_free(ctx, ctx->ws);
+  ctx_free(ctx, ctx->d_status);
+  ctx_free(ctx, ctx->st_ref);
+  ctx_free(ctx, ctx->srt);
+  ctx_free(ctx, ctx->small_ws);
   for (int i = 0; i < 2; ++i) {
-    if (ctx->st_batch[i]) cudaFree(ctx->st_batch[i]);
+    ctx_free(ctx, ctx->st_batch[i]);
     if (ctx->ev_copied[i]) cudaEventDestroy(ctx->ev_copied[i]);
     if (ctx->ev_done[i]) cudaEventDestroy(ctx->ev_done[i]);
   }
-  if (ctx->st_out) cudaFree(ctx->st_out);
+  ctx_free(ctx, ctx->st_out);
   if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
   for (int t = 0; t < kb_ctx::kTimers; ++t)
     for (int i = 0; i < kb_ctx::kPool; ++i) {
@@ -342,6 +381,40 @@ extern "C" kb_status kb_ctx_set_grid(kb_ctx* ctx, uint32_t blocks) {
 extern "C" kb_status kb_ctx_set_small_path(kb_ctx* ctx, int on) {
   if (!ctx) return KB_ERR_INVALID_ARG;
   ctx->small_on = on != 0;
+  return KB_OK;
+}
+
+extern "C" kb_status kb_ctx_fail_next_allocs(kb_ctx* ctx, uint32_t skip, uint32_t n) {
+  if (!ctx) return KB_ERR_INVALID_ARG;
+  ctx->skip_allocs = n ? skip : 0;
+  ctx->fail_allocs = n;
+  return KB_OK;
+}
+
+extern "C" kb_status kb_ctx_check_guards(kb_ctx* ctx, void* stream, uint32_t* n_buffers, uint32_t* n_bad_bytes) {
+  if (!ctx || !n_buffers || !n_bad_bytes) return KB_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  KB_CUDA(ctx, cudaStreamSynchronize(reinterpret_cast<cudaStream_t>(stream)));
+  uint32_t bad = 0;
+  unsigned char band[2 * kGuardBytes];
+  for (const kb_ctx::Guarded& gb : ctx->guarded) {
+    KB_CUDA(ctx, cudaMemcpy(band, gb.raw, kGuardBytes, cudaMemcpyDeviceToHost));
+    KB_CUDA(ctx, cudaMemcpy(band + kGuardBytes, gb.raw + kGuardBytes + gb.bytes, kGuardBytes, cudaMemcpyDeviceToHost));
+    for (size_t i = 0; i < 2 * kGuardBytes; ++i) bad += band[i] != (unsigned char)kGuardByte;
+  }
+  *n_buffers = (uint32_t)ctx->guarded.size();
+  *n_bad_bytes = bad;
+  return KB_OK;
+}
+
+extern "C" kb_status kb_ctx_selftest_wait(kb_ctx* ctx, uint64_t limit_ns, void* stream) {
+  if (!ctx) return KB_ERR_INVALID_ARG;
+  if (limit_ns < 1000ull || limit_ns > 100000000ull)
+    return fail(ctx, KB_ERR_INVALID_ARG, "kb_ctx_selftest_wait: limit outside [1 us, 100 ms]");
+  DeviceGuard g(ctx->device);
+  wait_selftest_kernel<<<1, 32, 0, reinterpret_cast<cudaStream_t>(stream)>>>(ctx->d_status, limit_ns);
+  ++ctx->launches;
+  KB_CUDA(ctx, cudaGetLastError());
   return KB_OK;
 }
 
@@ -958,8 +1031,8 @@ std::mutex g_static_mutex;
 
 // Once per device, with that device current: resolve the array's device address, read the
 // SM count, raise the kernels' shared-memory limits.  None of these allocates.
+// (the caller holds g_static_mutex)
 kb_status static_setup(int device, kb_ctx** out) {
-  std::lock_guard<std::mutex> lock(g_static_mutex);
   StaticSlot& slot = g_static_slot[device];
   if (!slot.ready) {
     kb_ctx* ctx = &slot.ctx;
@@ -972,6 +1045,7 @@ kb_status static_setup(int device, kb_ctx** out) {
     ctx->d_status = reinterpret_cast<unsigned int*>(base);
     ctx->ws = base + 256;
     ctx->ws_bytes = KB_STATIC_SCRATCH_BYTES - 256;   // ensure_ws never grows it: K is capped
+    ctx->ws_fixed = true;
     kb_status st;
     if ((st = set_stream_attr<KB_F32>(ctx)) != KB_OK) return st;
     if ((st = set_stream_attr<KB_F16>(ctx)) != KB_OK) return st;
@@ -1001,6 +1075,9 @@ extern "C" kb_status kb_screen_static(const void* d_ref, const void* const* h_ca
              "(use kb_screen, which may allocate)", K, KB_STATIC_MAX_K);
     return KB_ERR_WORKSPACE;
   }
+  // One host thread at a time validates and enqueues: all callers on a device share the
+  // slot's error text and launch counter as well as the scratch array.
+  std::lock_guard<std::mutex> lock(g_static_mutex);
   kb_ctx* ctx = nullptr;
   kb_status rc = static_setup(device, &ctx);
   if (rc == KB_OK) rc = validate_screen(ctx, d_ref, h_cands, K, N, dtype, atol, rtol, nullptr, d_out, true);
@@ -1009,6 +1086,16 @@ extern "C" kb_status kb_screen_static(const void* d_ref, const void* const* h_ca
                          reinterpret_cast<cudaStream_t>(stream));
   if (rc != KB_OK) snprintf(g_create_err, sizeof g_create_err, "%.250s", g_static_slot[device].ctx.err);
   return rc;
+}
+
+extern "C" kb_status kb_static_scratch_read(void* h_dst, uint32_t bytes) {
+  if (!h_dst || bytes > KB_STATIC_SCRATCH_BYTES) return KB_ERR_INVALID_ARG;
+  if (cudaDeviceSynchronize() != cudaSuccess ||
+      cudaMemcpyFromSymbol(h_dst, g_static_scratch, bytes, 0, cudaMemcpyDeviceToHost) != cudaSuccess) {
+    cudaGetLastError();
+    return KB_ERR_CUDA;
+  }
+  return KB_OK;
 }
 
 extern "C" kb_status kb_screen_host(kb_ctx* ctx, const void* h_ref, const void* const* h_cands_host,
@@ -1032,12 +1119,8 @@ extern "C" kb_status kb_screen_host(kb_ctx* ctx, const void* h_ref, const void* 
     }
   }
   if ((rc = ensure_buf(ctx, &ctx->st_ref, &ctx->st_ref_bytes, pitch)) != KB_OK) return rc;
-  if ((size_t)B * pitch > ctx->st_batch_bytes) {
-    size_t have0 = ctx->st_batch_bytes, have1 = ctx->st_batch_bytes;
-    if ((rc = ensure_buf(ctx, &ctx->st_batch[0], &have0, (size_t)B * pitch)) != KB_OK) return rc;
-    if ((rc = ensure_buf(ctx, &ctx->st_batch[1], &have1, (size_t)B * pitch)) != KB_OK) return rc;
-    ctx->st_batch_bytes = (size_t)B * pitch;
-  }
+  for (int i = 0; i < 2; ++i)
+    if ((rc = ensure_buf(ctx, &ctx->st_batch[i], &ctx->st_batch_bytes[i], (size_t)B * pitch)) != KB_OK) return rc;
   if ((rc = ensure_buf(ctx, &ctx->st_out, &ctx->st_out_bytes, (size_t)K * sizeof(kb_screen_result))) != KB_OK)
     return rc;
 
@@ -1090,16 +1173,9 @@ extern "C" kb_status kb_adjudicate(kb_ctx* ctx, const float* d_timings, uint32_t
     return fail(ctx, KB_ERR_UNSUPPORTED, "kb_adjudicate: the binary-search win count needs S <= 4096");
   if (ctx->wins_algo == 3 && d_wins && S > kMergeMaxS)
     return fail(ctx, KB_ERR_UNSUPPORTED, "kb_adjudicate: the merge win count needs S <= %u", kMergeMaxS);
-  if (rank) {
-    size_t have = ctx->srt_bytes;
-    if (ensure_buf(ctx, &ctx->srt, &have, (size_t)K * S * sizeof(float)) == KB_OK) {
-      ctx->srt_bytes = have;
-    } else if (ctx->wins_algo >= 2) {
-      return KB_ERR_WORKSPACE;
-    } else {
-      ctx->srt_bytes = 0;
-      rank = false;     // no room for the sorted copy: count by direct comparison
-    }
+  if (rank && ensure_buf(ctx, &ctx->srt, &ctx->srt_bytes, (size_t)K * S * sizeof(float), "sorted timings") != KB_OK) {
+    if (ctx->wins_algo >= 2) return KB_ERR_WORKSPACE;
+    rank = false;     // no room for the sorted copy: count by direct comparison
   }
   // rows: sort + quartiles (also the place where non-finite timings are caught)
   unsigned int P = 1;
@@ -1314,13 +1390,8 @@ extern "C" kb_status kb_adjudicate_ragged(kb_ctx* ctx, const float* d_timings,
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   float* srt = nullptr;
   if (d_wins) {
-    size_t have = ctx->srt_bytes;
-    kb_status rc = ensure_buf(ctx, &ctx->srt, &have, (size_t)total * sizeof(float));
-    if (rc != KB_OK) {
-      ctx->srt_bytes = 0;
-      return rc;
-    }
-    ctx->srt_bytes = have;
+    kb_status rc = ensure_buf(ctx, &ctx->srt, &ctx->srt_bytes, (size_t)total * sizeof(float), "sorted timings");
+    if (rc != KB_OK) return rc;
     srt = ctx->srt;
   }
   unsigned int P = 1;

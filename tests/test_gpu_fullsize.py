@@ -1,12 +1,12 @@
 """GPU parity at the full sizes of the five configurations, in the launch
 configuration the benchmark times.
 
-Where the oracle can afford it every candidate is compared bit for bit
-(configs 2 and 4); otherwise (configs 3 and 5: tens of GiB) a sample of
-candidates that covers every failure kind is compared bit for bit and the rest
-is checked through what must hold at any size: the closed-form consequences of
-how each candidate was built.  A last case exercises the largest tensor the
-boundary accepts (N = 2^32).
+Every candidate of every configuration is compared bit for bit with the oracle,
+which reads the very bytes the GPU screened (copied back from the device; under
+config 5's first-tier mask only the selected tiles are copied, into a host
+array whose other tiles hold NaN patterns the oracle must never touch).  The
+closed-form consequences of how each candidate was built are asserted as well.
+A last case exercises the largest tensor the boundary accepts (N = 2^32).
 """
 import os
 
@@ -115,6 +115,20 @@ def test_config4_full(ctx, kb):
     assert int(n.item()) == on and surv.cpu().numpy().tolist() == osurv.tolist()
 
 
+def oracle_all(case, ref_np, cands, mask="case"):
+    """The oracle's record of every candidate in `cands` (device tensors), copied back one by
+    one on the worker threads."""
+    from concurrent.futures import ThreadPoolExecutor
+    want = np.zeros(len(cands), dtype=oracle.RESULT_DTYPE)
+
+    def one(j):
+        want[j] = oracle_for(case, ref_np, cands[j], mask)
+
+    with ThreadPoolExecutor(max_workers=THREADS) as ex:
+        list(ex.map(one, range(len(cands))))
+    return want
+
+
 def test_config3_full(ctx, kb):
     dev = torch.device("cuda", 0)
     case, timings = synth.config3(dev)
@@ -123,20 +137,12 @@ def test_config3_full(ctx, kb):
     out = ctx.screen(case.ref, cands, case.atol, case.rtol)
     got = kb.records(out)
     assert ctx.poll() == 0
-    special = [k for k in range(case.K) if case.truth[k]["kind"] != "ulp_noise"]
-    clean = [k for k in range(case.K) if case.truth[k]["kind"] == "ulp_noise"]
-    assert len(special) == 26
+    assert sum(case.truth[k]["kind"] != "ulp_noise" for k in range(case.K)) == 26
     ref_np = synth.to_oracle_array(case.ref, case.dtype)
-    sample = special + clean[:3] + clean[-3:]
-
-    def one(k):
-        return k, oracle_for(case, ref_np, cands[k])
-
-    from concurrent.futures import ThreadPoolExecutor
-    with ThreadPoolExecutor(max_workers=min(THREADS, 8)) as ex:
-        for k, want in ex.map(one, sample):
-            assert same_record(got[k], want), (k, case.truth[k], got[k], want)
-    # every candidate, by construction
+    want = oracle_all(case, ref_np, cands)               # all 256 candidates
+    for k in range(case.K):
+        assert same_record(got[k], want[k]), (k, case.truth[k], got[k], want[k])
+    # and by construction
     for k in range(case.K):
         tr = case.truth[k]
         assert bool(got[k]["pass"]) == tr["passes"], (k, tr, got[k])
@@ -151,45 +157,72 @@ def test_config3_full(ctx, kb):
             assert 0 < got[k]["max_abs_err"] <= 2.0 ** -9          # one fp16 ulp below |x| < 4
     del cands
     torch.cuda.empty_cache()
-    check_adjudicate(ctx, timings, sample_rows=[0, 17, 128, 255])
+    med, omed = check_adjudicate(ctx, timings)           # the whole win matrix
+    surv, n = ctx.select(out, med, kb.KB_SELECT_ERR_THEN_TIME, 64)
+    osurv, on = oracle.select(want, omed, 0, 64)
+    assert int(n.item()) == on and surv.cpu().numpy().tolist() == osurv.tolist()
 
 
 def test_config5_full_two_tier(ctx, kb):
+    from concurrent.futures import ThreadPoolExecutor
     dev = torch.device("cuda", 0)
     c5 = synth.config5(dev)
     case = c5["case"]
     assert case.N == 1 << 28 and case.K == 512
     _, log2_tile, stride, phase = case.mask
+    assert log2_tile == 12
     mask = ctx.mask_strided(case.N, log2_tile, stride, phase)
     assert mask.n_selected == 1 << 24
     ref_np = synth.to_oracle_array(case.ref, case.dtype)
     labels = c5["labels"]
-    sample = []
-    for lab in ("clean", "hidden_burst", "visible_burst", "ulp4", "nan_inf"):
-        sample += [k for k in range(case.K) if labels[k] == lab][:2]
     out1 = torch.empty((case.K, kb.RESULT_BYTES), dtype=torch.uint8, device=dev)
+    want1 = np.zeros(case.K, dtype=oracle.RESULT_DTYPE)
+
+    # Host images for the oracle: full-size arrays in which only the tiles the mask selects are
+    # ever written (from the device); all other tiles keep a NaN pattern, so an oracle that read
+    # an unselected element would report NaNs the GPU does not.
+    import queue
+    pool = queue.Queue()
+    for _ in range(THREADS):
+        pool.put(np.full(case.N, 0x7FC0, dtype=np.uint16))
+
+    def one(k, sel_tiles):
+        img = pool.get()
+        try:
+            img.reshape(-1, stride, 1 << log2_tile)[:, phase, :] = sel_tiles
+            want1[k] = oracle.screen_one(ref_np, img, case.dtype, case.atol, case.rtol, case.mask)
+        finally:
+            pool.put(img)
+
     B = 64                                               # 32 GiB of candidates per batch
-    for k0 in range(0, case.K, B):
-        batch = [case.make_cand(k) for k in range(k0, k0 + B)]
-        ctx.screen(case.ref, batch, case.atol, case.rtol, mask, out=out1[k0:k0 + B])
-        torch.cuda.synchronize()
-        for k in sample:
-            if k0 <= k < k0 + B:
-                want = oracle_for(case, ref_np, batch[k - k0])
-                got = kb.records(out1[k:k + 1])[0]
-                assert same_record(got, want), (k, labels[k], got, want)
-        del batch
+    with ThreadPoolExecutor(max_workers=THREADS) as ex:
+        jobs = []
+        for k0 in range(0, case.K, B):
+            batch = [case.make_cand(k) for k in range(k0, k0 + B)]
+            ctx.screen(case.ref, batch, case.atol, case.rtol, mask, out=out1[k0:k0 + B])
+            torch.cuda.synchronize()
+            for jb in jobs:                              # at most two batches of tiles on the host
+                jb.result()
+            jobs = []
+            for j, c in enumerate(batch):
+                tiles = c.view(torch.int16).view(-1, stride, 1 << log2_tile)[:, phase, :].contiguous()
+                jobs.append(ex.submit(one, k0 + j, tiles.cpu().numpy().view(np.uint16)))
+            del batch
+        for jb in jobs:
+            jb.result()
     assert ctx.poll() == 0
     rec1 = kb.records(out1)
+    for k in range(case.K):                              # all 512 candidates, bit for bit
+        assert same_record(rec1[k], want1[k]), (k, labels[k], rec1[k], want1[k])
     for k in range(case.K):
         assert bool(rec1[k]["pass"]) == case.truth[k]["tier1_pass"], (k, case.truth[k], rec1[k])
         if labels[k] == "nan_inf":
             assert rec1[k]["nan_count"] == case.truth[k]["nan"] and rec1[k]["inf_count"] == case.truth[k]["inf"]
     assert int(rec1["pass"].sum()) == 256
 
-    med1, omed1 = check_adjudicate(ctx, c5["timings1"], sample_rows=[0, 100, 511])
+    med1, omed1 = check_adjudicate(ctx, c5["timings1"])
     surv, n = ctx.select(out1, med1, kb.KB_SELECT_ERR_THEN_TIME, c5["budget"])
-    osurv, on = oracle.select(rec1, omed1, 0, c5["budget"])
+    osurv, on = oracle.select(want1, omed1, 0, c5["budget"])      # the oracle's own records
     assert int(n.item()) == on == 32 and surv.cpu().numpy().tolist() == osurv.tolist()
 
     # tier 2: the 32 survivors on every element (16 GiB), regenerated from their seeds
@@ -198,17 +231,16 @@ def test_config5_full_two_tier(ctx, kb):
     out2 = ctx.screen(case.ref, cands2, case.atol, case.rtol)
     rec2 = kb.records(out2)
     assert ctx.poll() == 0
+    want2 = oracle_all(case, ref_np, cands2, mask=None)   # all 32 survivors
     for j, k in enumerate(s):
+        assert same_record(rec2[j], want2[j]), (k, labels[k], rec2[j], want2[j])
         assert bool(rec2[j]["pass"]) == case.truth[k]["tier2_pass"], (k, case.truth[k], rec2[j])
     hidden = [j for j, k in enumerate(s) if labels[k] == "hidden_burst"]
     cleanj = [j for j, k in enumerate(s) if labels[k] == "clean"]
     assert hidden and cleanj                             # the second tier has something to catch
-    for j in hidden[:2] + cleanj[:2]:
-        want = oracle_for(case, ref_np, cands2[j], mask=None)
-        assert same_record(rec2[j], want), (s[j], rec2[j], want)
     del cands2
     torch.cuda.empty_cache()
-    check_adjudicate(ctx, c5["make_timings2"](s), sample_rows=[0, 13, 31])
+    check_adjudicate(ctx, c5["make_timings2"](s))
     mask.close()
 
 

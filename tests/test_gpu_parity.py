@@ -466,15 +466,30 @@ def test_adjudicate_long_rows_use_direct_comparison(ctx, kb):
 
 
 def test_adjudicate_negative_and_zero_timings(ctx, kb):
+    """Zeros of both signs: the sorted row is unique (-0 before +0), so medians and IQRs are
+    compared as bit patterns, signs of zeros included."""
     dev = torch.device("cuda", 0)
-    t = np.float32([[0.0, -1.0, 2.0, 0.0, 1.0], [1.0, 0.0, -2.0, 5.0, 1.0], [3.0, 3.0, 3.0, 3.0, 3.0]])
+    t = np.float32([[0.0, -1.0, 2.0, -0.0, 1.0], [1.0, 0.0, -2.0, 5.0, 1.0], [3.0, 3.0, 3.0, 3.0, 3.0],
+                    [0.0, -0.0, 0.0, -0.0, -0.0], [-0.0, 0.0, 0.0, 0.0, 0.0], [-0.0, -0.0, -0.0, -0.0, -0.0]])
     omed, oiqr, owins = oracle.adjudicate(t)
-    for algo in (1, 2):
+    assert fbits(omed).tolist()[3:] == [0x80000000, 0, 0x80000000]
+    for algo in (1, 2, 3):
         ctx.set_wins_algo(algo)
         med, iqr, wins = ctx.adjudicate(torch.from_numpy(t).to(dev))
         ctx.set_wins_algo(0)
-        assert (med.cpu().numpy() == omed).all() and (iqr.cpu().numpy() == oiqr).all()
+        assert (fbits(med.cpu().numpy()) == fbits(omed)).all()
+        assert (fbits(iqr.cpu().numpy()) == fbits(oiqr)).all()
         assert (wins.cpu().numpy().view(np.uint32) == owins).all()
+    rng = np.random.default_rng(18)
+    for S in (2, 7, 32, 33, 100, 257):
+        t = rng.choice(np.float32([0.0, -0.0, 0.0, -0.0, 1.0, -1.0]), (9, S)).astype(np.float32)
+        omed, oiqr, owins = oracle.adjudicate(t)
+        med, iqr, wins = ctx.adjudicate(torch.from_numpy(t).to(dev))
+        assert (fbits(med.cpu().numpy()) == fbits(omed)).all(), S
+        assert (fbits(iqr.cpu().numpy()) == fbits(oiqr)).all(), S
+        assert (wins.cpu().numpy().view(np.uint32) == owins).all()
+        rat = ctx.tail_ratios(torch.from_numpy(np.abs(t) + np.float32(1.0)).to(dev))
+        assert (fbits(rat.cpu().numpy()) == fbits(oracle.tail_ratios(np.abs(t) + np.float32(1.0)))).all()
 
 
 def test_adjudicate_flags_nonfinite(ctx, kb):

@@ -164,6 +164,7 @@ def test_random_adjudicate_and_select(ctx, kb, block):
             t = np.round(t, int(rng.choice([1, 2])))
         if rng.random() < 0.2:
             t[rng.random((K, S)) < 0.05] = 0.0
+            t[(t == 0.0) & (rng.random((K, S)) < 0.5)] = -0.0       # zeros of both signs
         if rng.random() < 0.1:
             t = t - 1.0
         t = t.astype(np.float32)
@@ -176,8 +177,8 @@ def test_random_adjudicate_and_select(ctx, kb, block):
                 ctx.set_wins_algo(0)
             assert ctx.poll() == 0
             label = f"seed block={block} i={i} K={K} S={S} algo={algo}"
-            assert (med.cpu().numpy() == omed).all(), label          # values: the sign of a zero is free
-            assert (iqr.cpu().numpy() == oiqr).all(), label
+            assert (fbits(med.cpu().numpy()) == fbits(omed)).all(), label   # bit patterns: the sorted
+            assert (fbits(iqr.cpu().numpy()) == fbits(oiqr)).all(), label   # row is unique (-0 before +0)
             assert (wins.cpu().numpy().view(np.uint32) == owins).all(), label
         rec = np.zeros(K, dtype=oracle.RESULT_DTYPE)
         rec["pass"] = rng.random(K) < 0.7

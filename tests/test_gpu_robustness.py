@@ -1,0 +1,287 @@
+"""Failure paths and out-of-bounds checks on the GPU, none of which faults, traps or hangs it.
+
+* a bounded device-side wait that runs out (a stand-alone warp waiting on a barrier nothing
+  completes, with no copy in flight) is reported through kb_ctx_poll and leaves the context
+  usable;
+* a workspace allocation that fails (refused by a hook, the device's memory is not touched)
+  leaves the context with its old, valid buffers;
+* guard bands: every caller-owned output sits between two bands of a canary pattern that must
+  be intact after the call, and the library's own device buffers carry the same bands
+  (kb_ctx_check_guards) -- the stand-in for a memory checker.
+"""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2608_02611_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+THREADS = max(1, len(os.sched_getaffinity(0)))
+CANARY = 0xA5
+BAND = 256
+
+
+@pytest.fixture(scope="module")
+def kb():
+    from paper_2608_02611_b200 import binding
+    return binding
+
+
+@pytest.fixture()
+def ctx(kb):
+    c = kb.Context(0)
+    yield c
+    c.close()
+
+
+def fbits(a):
+    return np.ascontiguousarray(a, dtype=np.float32).view(np.uint32)
+
+
+def same_records(got, want):
+    for f in want.dtype.names:
+        a, b = got[f], want[f]
+        if a.dtype.kind == "f":
+            a, b = a.view(np.uint32 if a.dtype.itemsize == 4 else np.uint64), \
+                b.view(np.uint32 if b.dtype.itemsize == 4 else np.uint64)
+        assert (a == b).all(), f
+
+
+class Guarded:
+    """A device tensor of `shape`/`dtype` placed between two canary bands."""
+
+    def __init__(self, shape, dtype, dev):
+        n = int(np.prod(shape)) * torch.empty(0, dtype=dtype).element_size()
+        self.nbytes = n
+        self.raw = torch.full((n + 2 * BAND,), CANARY, dtype=torch.uint8, device=dev)
+        self.t = self.raw[BAND:BAND + n].view(dtype).view(shape)
+
+    def intact(self):
+        torch.cuda.synchronize()
+        return bool((self.raw[:BAND] == CANARY).all()) and bool((self.raw[BAND + self.nbytes:] == CANARY).all())
+
+
+def oracle_records(case_dtype, ref, cands, atol, rtol, mask=None):
+    return oracle.screen(synth.to_oracle_array(ref, case_dtype),
+                         [synth.to_oracle_array(c, case_dtype) for c in cands],
+                         case_dtype, atol, rtol, mask, threads=THREADS)
+
+
+# ---------------------------------------------------------------------------------------------
+
+def test_bounded_wait_runs_out_and_the_context_stays_usable(ctx, kb):
+    dev = torch.device("cuda", 0)
+    case, _ = synth.config2(dev, side=768, K=12, n_bad=3)          # K*N > 2^22: the streaming gate
+    cands = case.cands()
+    want = oracle_records(case.dtype, case.ref, cands, case.atol, case.rtol)
+    same_records(kb.records(ctx.screen(case.ref, cands, case.atol, case.rtol)), want)
+    assert ctx.poll() == 0
+    ctx.selftest_wait(1_000_000)                   # one warp, 1 ms limit, nothing arrives
+    assert ctx.poll() == 7                         # KB_ERR_DEVICE_TIMEOUT
+    assert ctx.poll() == 0                         # cleared by the read
+    # the next call on the same context is exact, and the status stays clear
+    same_records(kb.records(ctx.screen(case.ref, cands, case.atol, case.rtol)), want)
+    assert ctx.poll() == 0
+    with pytest.raises(kb.KbError):
+        ctx.selftest_wait(10)                      # limits outside [1 us, 100 ms] are refused
+    with pytest.raises(kb.KbError):
+        ctx.selftest_wait(10_000_000_000)
+
+
+def test_failed_workspace_growth_keeps_the_old_workspace(ctx, kb):
+    dev = torch.device("cuda", 0)
+    ctx.set_small_path(False)                      # the general path uses the growing workspace
+    rng = np.random.default_rng(11)
+    ref = torch.from_numpy(rng.standard_normal(5000).astype(np.float32)).to(dev)
+    cands = [ref.clone() for _ in range(40)]
+    cands[7][123] += 1.0
+    want = oracle_records(synth.F32, ref, cands, 1e-5, 1e-3)
+    same_records(kb.records(ctx.screen(ref, cands, 1e-5, 1e-3)), want)       # workspace for 40 (x2)
+    many = [ref] * 3000                            # needs a larger workspace
+    out = torch.full((3000, kb.RESULT_BYTES), 0xAB, dtype=torch.uint8, device=dev)
+    ctx.fail_next_allocs(1)
+    with pytest.raises(kb.KbError) as e:
+        ctx.screen(ref, many, 1e-5, 1e-3, out=out)
+    assert e.value.status == 4                     # KB_ERR_WORKSPACE
+    assert (out.cpu() == 0xAB).all()               # nothing was launched
+    # the old workspace is still there and still right
+    same_records(kb.records(ctx.screen(ref, cands, 1e-5, 1e-3)), want)
+    # and with the hook spent the large call goes through
+    rec = kb.records(ctx.screen(ref, many, 1e-5, 1e-3, out=out))
+    assert (rec["pass"] == 1).all()
+    assert ctx.poll() == 0
+
+    # sorted-timings buffer of kb_adjudicate
+    t_small = np.round(rng.lognormal(0, 0.1, (16, 40)), 2).astype(np.float32)
+    t_big = np.round(rng.lognormal(0, 0.1, (64, 200)), 2).astype(np.float32)
+    ctx.set_wins_algo(2)
+    med, iqr, wins = ctx.adjudicate(torch.from_numpy(t_small).to(dev))
+    ow = oracle.adjudicate(t_small)[2]
+    assert (wins.cpu().numpy().view(np.uint32) == ow).all()
+    ctx.fail_next_allocs(1)
+    with pytest.raises(kb.KbError) as e:
+        ctx.adjudicate(torch.from_numpy(t_big).to(dev))
+    assert e.value.status == 4
+    med, iqr, wins = ctx.adjudicate(torch.from_numpy(t_small).to(dev))      # old buffer, still valid
+    assert (wins.cpu().numpy().view(np.uint32) == ow).all()
+    ctx.set_wins_algo(0)
+    ctx.fail_next_allocs(1)                        # automatic choice: falls back to direct comparison
+    med, iqr, wins = ctx.adjudicate(torch.from_numpy(t_big).to(dev))
+    assert (wins.cpu().numpy().view(np.uint32) == oracle.adjudicate(t_big, threads=THREADS)[2]).all()
+    assert ctx.poll() == 0
+
+    # host-buffer path: the SECOND of its two batch buffers fails to grow
+    h_ref = ref.cpu()
+    h_cands = [c.cpu() for c in cands]
+    same_records(ctx.screen_host(h_ref, h_cands, 1e-5, 1e-3), want)
+    big_ref = torch.from_numpy(rng.standard_normal(300000).astype(np.float32))
+    big_cands = [big_ref.clone() for _ in range(3)]
+    big_cands[1][299999] = float("nan")
+    ctx.fail_next_allocs(1, skip=2)                # reference staging, first batch buffer pass
+    with pytest.raises(kb.KbError) as e:
+        ctx.screen_host(big_ref, big_cands, 1e-5, 1e-3)
+    assert e.value.status == 4
+    same_records(ctx.screen_host(h_ref, h_cands, 1e-5, 1e-3), want)          # small call still right
+    rec = ctx.screen_host(big_ref, big_cands, 1e-5, 1e-3)
+    assert rec["pass"].tolist() == [1, 0, 1] and rec["nan_count"].tolist() == [0, 1, 0]
+    nb, bad = ctx.check_guards()
+    assert nb >= 6 and bad == 0
+
+
+@pytest.mark.parametrize("dtype", [synth.F32, synth.F16, synth.BF16])
+def test_guard_bands_around_screen_outputs(ctx, kb, dtype):
+    """kb_screen on every dispatch path writes K records and nothing else."""
+    dev = torch.device("cuda", 0)
+    rng = np.random.default_rng(100 + dtype)
+    N = 5 * 4096 + 37                              # full tiles plus a ragged tail
+    tdt = synth.TORCH_DTYPE[dtype]
+    ref = torch.from_numpy(rng.standard_normal(N).astype(np.float32)).to(tdt).to(dev)
+    K = 13
+    cands = []
+    for k in range(K):
+        c = ref.clone()
+        if k % 3 == 1:
+            c[rng.integers(0, N, 5)] = 2.5
+        if k == 4:
+            c[N - 1] = float("nan")
+        cands.append(c)
+    want = oracle_records(dtype, ref, cands, 1e-3, 1e-2)
+    spec = ("strided", 5, 3, 1)
+    want_fine = oracle_records(dtype, ref, cands, 1e-3, 1e-2, spec)
+    spec_c = ("strided", 12, 2, 1)
+    want_coarse = oracle_records(dtype, ref, cands, 1e-3, 1e-2, spec_c)
+    fine = ctx.mask_strided(N, 5, 3, 1)
+    coarse = ctx.mask_strided(N, 12, 2, 1)
+    for small in (True, False):
+        ctx.set_small_path(small)
+        for grid in (0, 1, 5):
+            ctx.set_grid(grid)
+            for mask, w in ((None, want), (fine, want_fine), (coarse, want_coarse)):
+                g = Guarded((K, kb.RESULT_BYTES), torch.uint8, dev)
+                ctx.screen(ref, cands, 1e-3, 1e-2, mask, out=g.t)
+                assert g.intact(), (small, grid)
+                same_records(kb.records(g.t), w)
+    ctx.set_grid(0)
+    ctx.set_small_path(True)
+    fine.close()
+    coarse.close()
+    # several shapes in one launch
+    groups = [(ref[:n].clone(), [c[:n].clone() for c in cands[:kk]]) for n, kk in ((700, 3), (4096, 5), (9001, 2))]
+    g = Guarded((10, kb.RESULT_BYTES), torch.uint8, dev)
+    ctx.screen_multi(groups, 1e-3, 1e-2, out=g.t)
+    assert g.intact()
+    got = kb.records(g.t)
+    o = 0
+    for r, cs in groups:
+        same_records(got[o:o + len(cs)], oracle_records(dtype, r, cs, 1e-3, 1e-2))
+        o += len(cs)
+    # a selection that lives on the device, with fewer survivors than slots
+    table = ctx.pointer_table(cands)
+    index = torch.tensor([4, 0, 9, 1, 1, 1], dtype=torch.int32, device=dev)
+    count = torch.tensor([3], dtype=torch.int32, device=dev)
+    g = Guarded((6, kb.RESULT_BYTES), torch.uint8, dev)
+    ctx.screen_indexed(ref, table, index, count, 1e-3, 1e-2, out=g.t)
+    assert g.intact()
+    got = kb.records(g.t)
+    same_records(got[:3], want[[4, 0, 9]])
+    assert (got["pass"][3:] == 0).all() and (got["argmax_idx"][3:] == -1).all()
+    assert ctx.poll() == 0
+    nb, bad = ctx.check_guards()
+    assert nb >= 3 and bad == 0                    # status words, single-launch workspace, accumulators
+
+
+def test_guard_bands_around_the_double_precision_gate(ctx, kb):
+    dev = torch.device("cuda", 0)
+    rng = np.random.default_rng(64)
+    N = 9 * 4096 + 5
+    ref = torch.from_numpy(rng.standard_normal(N)).to(dev)
+    cands = [ref.clone() for _ in range(5)]
+    cands[2][N - 1] += 1e-3
+    cands[3][4096] = float("inf")
+    g = Guarded((5, kb.RESULT_F64_BYTES), torch.uint8, dev)
+    ctx.screen_f64(ref, cands, 1e-12, 1e-9, out=g.t)
+    assert g.intact()
+    want = oracle.screen_f64(ref.cpu().numpy(), [c.cpu().numpy() for c in cands], 1e-12, 1e-9)
+    same_records(kb.records_f64(g.t), want)
+    assert ctx.poll() == 0
+    assert ctx.check_guards()[1] == 0
+
+
+@pytest.mark.parametrize("K,S", [(3, 5), (13, 33), (37, 100), (230, 17), (9, 4100)])
+def test_guard_bands_around_adjudication_and_selection_outputs(ctx, kb, K, S):
+    dev = torch.device("cuda", 0)
+    rng = np.random.default_rng(K * 1000 + S)
+    t = np.round(rng.lognormal(0, 0.1, (K, S)), 2).astype(np.float32)
+    omed, oiqr, owins = oracle.adjudicate(t, threads=THREADS)
+    d_t = torch.from_numpy(t).to(dev)
+    for algo in (0, 1, 2, 3):
+        if (algo == 2 and S > 4096) or (algo == 3 and S > 1024):
+            continue
+        ctx.set_wins_algo(algo)
+        gm, gi = Guarded((K,), torch.float32, dev), Guarded((K,), torch.float32, dev)
+        gw = Guarded((K, K), torch.int32, dev)
+        ctx.adjudicate(d_t, out=(gm.t, gi.t, gw.t))
+        assert gm.intact() and gi.intact() and gw.intact(), algo
+        assert (fbits(gm.t.cpu().numpy()) == fbits(omed)).all()
+        assert (fbits(gi.t.cpu().numpy()) == fbits(oiqr)).all()
+        assert (gw.t.cpu().numpy().view(np.uint32) == owins).all()
+    ctx.set_wins_algo(0)
+    rec = np.zeros(K, dtype=oracle.RESULT_DTYPE)
+    rec["pass"] = rng.random(K) < 0.7
+    rec["mismatch_count"] = 1 - rec["pass"]
+    rec["max_rel_err"] = rng.choice(np.float32([0.0, 2.0 ** -7, 0.01]), K)
+    d_rec = torch.from_numpy(rec.view(np.uint8).reshape(K, 48).copy()).to(dev)
+    for budget in (1, K, K + 5):
+        gs, gn = Guarded((budget,), torch.int32, dev), Guarded((1,), torch.int32, dev)
+        ctx.select(d_rec, gm.t, 0, budget, out=(gs.t, gn.t))
+        assert gs.intact() and gn.intact()
+        osurv, on = oracle.select(rec, omed, 0, budget)
+        assert int(gn.t.item()) == on and gs.t.cpu().numpy().tolist() == osurv.tolist()
+    assert ctx.poll() == 0
+    assert ctx.check_guards()[1] == 0
+
+
+def test_static_scratch_is_untouched_beyond_the_part_a_call_uses(kb):
+    """kb_screen_static with K candidates uses the status words, K accumulators and K table
+    entries of its fixed array; every byte beyond them keeps its value."""
+    dev = torch.device("cuda", 0)
+    rng = np.random.default_rng(9)
+    N = 3 * 4096 + 11
+    ref = torch.from_numpy(rng.standard_normal(N).astype(np.float32)).to(dev)
+    K = 37
+    cands = [ref.clone() for _ in range(K)]
+    cands[5][100] = 7.0
+    out = torch.empty((K, kb.RESULT_BYTES), dtype=torch.uint8, device=dev)
+    kb.screen_static(ref, cands[:3], 1e-5, 1e-3, out=out[:3])      # set-up call
+    before = kb.static_scratch_read()
+    kb.screen_static(ref, cands, 1e-5, 1e-3, out=out)
+    after = kb.static_scratch_read()
+    acc_end = 256 + ((K * 48 + 255) // 256) * 256
+    tab_end = acc_end + K * 8
+    assert (after[tab_end:] == before[tab_end:]).all()
+    assert (after[256 + K * 48:acc_end] == before[256 + K * 48:acc_end]).all()
+    same_records(kb.records(out), oracle_records(synth.F32, ref, cands, 1e-5, 1e-3))

@@ -130,6 +130,43 @@ def test_median_is_middle_or_midpoint():
     assert oracle.quantiles(np.float32([7]))[0].tolist() == [7, 7, 7, 0]
 
 
+def test_signed_zeros_sort_negative_first_and_fix_the_sign_of_zero_quantiles():
+    """A row that mixes -0 and +0: the sorted row is unique (value, then -0 before +0), so the
+    sign of a quantile that is zero is fixed.  The expected signs are worked out by hand."""
+    def bits(v):
+        return [int(x) for x in np.asarray(v, dtype=np.float32).view(np.uint32)]
+    NZ, PZ = 0x80000000, 0x00000000
+    # S = 5: positions 1, 2, 3 hit samples exactly (rem = 0).
+    q, srt = oracle.quantiles(np.float32([0.0, -0.0, 0.0, -0.0, -0.0]))
+    assert bits(srt) == [NZ, NZ, NZ, PZ, PZ]
+    # Q1 = x1 = -0, median = x2 = -0, Q3 = x3 = +0, IQR = (+0) - (-0) = +0
+    assert bits(q) == [NZ, NZ, PZ, PZ]
+    q, srt = oracle.quantiles(np.float32([0.0, 0.0, -0.0, 0.0, 0.0]))
+    assert bits(srt) == [NZ, PZ, PZ, PZ, PZ]
+    # Q1 = +0, median = +0, Q3 = +0, IQR = (+0) - (+0) = +0
+    assert bits(q) == [PZ, PZ, PZ, PZ]
+    # S = 2, row {+0, -0} -> sorted {-0, +0}: Q_j = -0 + (j/4)*((+0) - (-0)) = -0 + (+0) = +0
+    q, srt = oracle.quantiles(np.float32([0.0, -0.0]))
+    assert bits(srt) == [NZ, PZ] and bits(q) == [PZ, PZ, PZ, PZ]
+    # S = 2, row {-0, -0}: Q_j = -0 + (j/4)*((-0) - (-0)) = -0 + (j/4)*(+0) = -0 + +0 = +0
+    q, srt = oracle.quantiles(np.float32([-0.0, -0.0]))
+    assert bits(srt) == [NZ, NZ] and bits(q) == [PZ, PZ, PZ, PZ]
+    # S = 1: every quantile is the sample itself; IQR = (-0) - (-0) = +0
+    q, _ = oracle.quantiles(np.float32([-0.0]))
+    assert bits(q) == [NZ, NZ, NZ, PZ]
+    # zeros among other values: [-1, +0, -0, 2, -0] sorts to [-1, -0, -0, +0, 2]
+    q, srt = oracle.quantiles(np.float32([-1.0, 0.0, -0.0, 2.0, -0.0]))
+    assert bits(srt) == [0xBF800000, NZ, NZ, PZ, 0x40000000]
+    assert bits(q) == [NZ, NZ, PZ, PZ]
+    # the order of the input does not matter
+    rng = np.random.default_rng(5)
+    row = np.float32([0.0, -0.0, 0.0, -0.0, 1.0, -1.0, -0.0, 0.0, 0.0])
+    want = bits(oracle.quantiles(row)[1])
+    assert want == [0xBF800000, NZ, NZ, NZ, PZ, PZ, PZ, PZ, 0x3F800000]
+    for _ in range(20):
+        assert bits(oracle.quantiles(rng.permutation(row))[1]) == want
+
+
 def test_nonfinite_timing_is_an_error():
     t = np.ones((3, 4), dtype=np.float32)
     for bad in (np.nan, np.inf, -np.inf):

@@ -37,8 +37,12 @@ def _worker(rank, world, port, K, q):
         dist.destroy_process_group()
 
 
-def test_two_ranks_shard_and_gather():
-    K, world = 7, 2                       # an odd K: the shards differ in size
+import pytest
+
+
+@pytest.mark.parametrize("K", [7, 1])     # an odd K: the shards differ in size; K = 1: one is empty
+def test_two_ranks_shard_and_gather(K):
+    world = 2
     ctx = mp.get_context("spawn")
     q = ctx.Queue()
     port = _free_port()
