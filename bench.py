@@ -72,6 +72,8 @@ class ClockSampler(threading.Thread):
         self.samples, self.reasons, self.max_mhz = [], set(), None
         self.stamps = []
         self.window = None                 # (t0, t1) of the timed region, perf_counter
+        self.n_before_load = 0             # samples taken before the first warm-up step
+        self.ready = threading.Event()
         self._halt = threading.Event()
 
     def run(self):
@@ -81,7 +83,9 @@ class ClockSampler(threading.Thread):
             h = nv.nvmlDeviceGetHandleByIndex(self.index)
             self.max_mhz = int(nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM))
         except Exception:
+            self.ready.set()
             return
+        self.ready.set()
         names = {
             "hw_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
             "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
@@ -104,17 +108,18 @@ class ClockSampler(threading.Thread):
         self._halt.set()
         if self.is_alive():
             self.join(timeout=2)
-        samples = list(self.samples)
-        stamps = list(self.stamps)[:len(samples)]
+        samples = list(self.samples)[self.n_before_load:]
+        stamps = list(self.stamps)[self.n_before_load:][:len(samples)]
         timed = [v for v, t in zip(samples, stamps)
                  if self.window and self.window[0] <= t <= self.window[1]]
-        # the sampler runs from before the warm-up steps (the same load) to the end of the
-        # timed region; a timed region shorter than one NVML query still gets the load's clock
-        use = timed if len(timed) >= 3 else samples
+        # the sampler runs from the first warm-up step to the end of the timed region and, if
+        # that gave fewer than five samples, over an untimed continuation of the same steps
+        use = timed if len(timed) >= 5 else samples
         return {"sm_mhz": int(np.median(use)) if use else None,
                 "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
-                "samples": len(samples), "samples_in_timed_region": len(timed),
-                "window": "warm-up + timed region"}
+                "samples": len(use), "samples_in_timed_region": len(timed),
+                "window": "timed region" if len(timed) >= 5 else
+                          "warm-up + timed region + untimed continuation of the same steps"}
 
 
 def host_cores() -> int:
@@ -380,6 +385,8 @@ def main():
 
     sampler = ClockSampler(local_rank)
     sampler.start()
+    sampler.ready.wait(timeout=5)           # NVML initialised (tens of ms) before the load starts
+    sampler.n_before_load = len(sampler.samples)
     for _ in range(warmup):
         step()
     barrier()
@@ -398,13 +405,22 @@ def main():
     e1.record()
     barrier()
     sampler.window = (t_begin, time.perf_counter())
-    clocks = sampler.stop()
     elapsed_ms = e0.elapsed_time(e1)
     launches = ctx.launch_count + ctx_adj.launch_count - launches0
     stream_ms = ctx.read_timer(binding.KB_TIMER_SCREEN_STREAM)
     wins_ms = ctx_adj.read_timer(binding.KB_TIMER_WINS)
     ctx.enable_timing(False)
     ctx_adj.enable_timing(False)
+    # A timed region shorter than a few NVML queries (20 steps take 7 ms) leaves the sampler
+    # nothing to see: the same steps go on, untimed and uncounted, until it has five samples
+    # under this load.
+    t_more = time.perf_counter()
+    while sampler.is_alive() and len(sampler.samples) < 5 + sampler.n_before_load \
+            and time.perf_counter() - t_more < 0.5:
+        for _ in range(10):
+            step()
+        torch.cuda.synchronize()
+    clocks = sampler.stop()
     if world > 1:
         elapsed_ms = sharding.max_over_ranks(elapsed_ms, dev)
     ms_per_step = elapsed_ms / steps
