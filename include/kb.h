@@ -252,7 +252,7 @@ kb_status kb_screen_f64(kb_ctx* ctx, const double* d_ref, const double* const* h
  *     A device-side wait that ran out cannot be polled through this entry point
  *     (there is no context); use kb_screen + kb_ctx_poll where that matters. */
 #define KB_STATIC_MAX_K 1024u
-#define KB_STATIC_SCRATCH_BYTES (256u + 1024u * 48u + 1024u * 8u)
+#define KB_STATIC_SCRATCH_BYTES (256u + 2u * 1024u * 48u + 1024u * 8u)
 kb_status kb_screen_static(const void* d_ref, const void* const* h_cands, uint32_t K, uint64_t N,
                            kb_dtype dtype, float atol, float rtol, kb_screen_result* d_out,
                            void* stream);

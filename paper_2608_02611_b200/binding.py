@@ -370,7 +370,7 @@ def screen_static(ref: torch.Tensor, cands: Sequence[torch.Tensor], atol: float,
     return out
 
 
-KB_STATIC_SCRATCH_BYTES = 256 + 1024 * 48 + 1024 * 8
+KB_STATIC_SCRATCH_BYTES = 256 + 2 * 1024 * 48 + 1024 * 8
 
 
 def static_scratch_read(nbytes: int = KB_STATIC_SCRATCH_BYTES) -> np.ndarray:

@@ -20,9 +20,22 @@ using namespace kb;
 struct kb_ctx {
   int device = 0;
   int sm_count = 0;
-  unsigned char* ws = nullptr;      // [acc K*48 | pad | pointer table K*8]
+  // Workspace for ws_cap_K candidates: [accumulators, set 0 | accumulators, set 1 | pointer table |
+  // accumulators of the binary64 gate]; no offset depends on a call's K.
+  unsigned char* ws = nullptr;
   size_t ws_bytes = 0;
+  uint32_t ws_cap_K = 0;
   bool ws_fixed = false;            // the workspace is not ours to grow or free (kb_screen_static)
+  // The binary32 gate keeps two sets of accumulators and counters.  A call works on set
+  // `ws_parity`, which is zero on entry, and its lead kernel zeroes the other set (as far as the
+  // last call on it got: `used_K`) for the next call.  `ws_dirty`: that may not hold (fresh
+  // memory, a call that failed half-way or ran out of time, a call captured into a graph, a path
+  // without a lead launch): the next call zeroes both sets with memsets first.
+  int ws_parity = 0;
+  uint32_t used_K[2] = {0, 0};
+  bool ws_dirty = true;
+  // [0] status, [1..3] counters of the binary64 gate, [4] effective K of an indexed call,
+  // [8..10] and [16..18] the two counter sets of the binary32 gate, [60] probe sink
   unsigned int* d_status = nullptr;
   uint32_t forced_grid = 0;
   unsigned char* small_ws = nullptr; // single-launch path: [tickets 4 KB | partial records 384 KB]
@@ -180,11 +193,24 @@ kb_status ensure_buf(kb_ctx* ctx, T** buf, size_t* have, size_t need, const char
   return KB_OK;
 }
 
-kb_status ensure_ws(kb_ctx* ctx, uint32_t K, size_t acc_bytes = sizeof(Acc)) {
-  const size_t need = round_up((size_t)K * acc_bytes, 256) + (size_t)K * sizeof(void*);
-  if (need <= ctx->ws_bytes) return KB_OK;
-  if (ctx->ws_fixed) return fail(ctx, KB_ERR_WORKSPACE, "the fixed scratch holds %zu bytes, %zu needed", ctx->ws_bytes, need);
-  return ensure_buf(ctx, &ctx->ws, &ctx->ws_bytes, round_up(need * 2, 4096), "device workspace");
+static_assert(sizeof(Acc) == sizeof(Acc64), "one region size serves both gates");
+inline size_t ws_region(uint32_t cap_K) { return round_up((size_t)cap_K * sizeof(Acc), 256); }
+inline size_t ws_table_offset(uint32_t cap_K) { return 2 * ws_region(cap_K); }
+inline size_t ws_acc64_offset(uint32_t cap_K) {
+  return 2 * ws_region(cap_K) + round_up((size_t)cap_K * sizeof(void*), 256);
+}
+inline unsigned int* counter_set(kb_ctx* ctx, int set) { return ctx->d_status + 8 + 8 * set; }
+kb_status ensure_ws(kb_ctx* ctx, uint32_t K) {
+  if (K <= ctx->ws_cap_K) return KB_OK;
+  if (ctx->ws_fixed)
+    return fail(ctx, KB_ERR_WORKSPACE, "the fixed scratch holds %u candidates, %u asked for", ctx->ws_cap_K, K);
+  const uint32_t cap = K < 32768u ? 2u * K : 65535u;
+  const kb_status rc =
+      ensure_buf(ctx, &ctx->ws, &ctx->ws_bytes, ws_acc64_offset(cap) + ws_region(cap), "device workspace");
+  if (rc != KB_OK) return rc;
+  ctx->ws_cap_K = cap;
+  ctx->ws_dirty = true;   // fresh memory
+  return KB_OK;
 }
 
 // ring depth by stage size: 3 CTAs/SM must fit ~75 KB each
@@ -369,6 +395,7 @@ extern "C" kb_status kb_ctx_poll(kb_ctx* ctx, void* stream, kb_status* device_st
   KB_CUDA(ctx, cudaMemsetAsync(ctx->d_status, 0, sizeof word, st));
   KB_CUDA(ctx, cudaStreamSynchronize(st));
   *device_status = (kb_status)word;
+  if (word != 0u) ctx->ws_dirty = true;   // a call may have been cut short: take nothing on trust
   return KB_OK;
 }
 
@@ -685,22 +712,61 @@ kb_status screen_impl(kb_ctx* ctx, const void* d_ref, const void* const* h_cands
   }
   kb_status rc = ensure_ws(ctx, K);
   if (rc != KB_OK) return rc;
-  Acc* acc = reinterpret_cast<Acc*>(ctx->ws);
-  const void** table = reinterpret_cast<const void**>(ctx->ws + round_up((size_t)K * sizeof(Acc), 256));
+  const void** table = reinterpret_cast<const void**>(ctx->ws + ws_table_offset(ctx->ws_cap_K));
+
+  // Two sets of accumulators and counters: this call's (zero on entry) and the one its lead
+  // kernel zeroes for the next call.  Whatever may have broken that is repaired with memsets.
+  // A call that is being captured into a graph takes nothing on trust (the graph may be
+  // replayed in any state) and leaves the workspace marked dirty for the calls after it.
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) {
+    cudaGetLastError();
+    cap = cudaStreamCaptureStatusActive;
+  }
+  const bool capturing = cap != cudaStreamCaptureStatusNone;
+  if (capturing || ctx->ws_dirty) {
+    KB_CUDA(ctx, cudaMemsetAsync(ctx->ws, 0, 2 * ws_region(ctx->ws_cap_K), st));
+    KB_CUDA(ctx, cudaMemsetAsync(counter_set(ctx, 0), 0, 16 * sizeof(unsigned int), st));   // both sets
+    ctx->used_K[0] = ctx->used_K[1] = 0;
+  }
+  const int set = ctx->ws_parity;
+  Acc* acc = reinterpret_cast<Acc*>(ctx->ws + (size_t)set * ws_region(ctx->ws_cap_K));
+  Acc* acc_next = reinterpret_cast<Acc*>(ctx->ws + (size_t)(set ^ 1) * ws_region(ctx->ws_cap_K));
+  unsigned int* counters = counter_set(ctx, set);
+  ctx->ws_dirty = true;      // until every launch of this call has been enqueued
+  bool lead_ran = false;
+  auto finished = [&]() {
+    // the lead kernel has cleaned the other set; without one (or under capture) the next call memsets
+    if (lead_ran && !capturing) {
+      ctx->used_K[set] = K;
+      ctx->used_K[set ^ 1] = 0;
+      ctx->ws_parity = set ^ 1;
+      ctx->ws_dirty = false;
+    }
+    return KB_OK;
+  };
+
+  // Candidate pointers: up to kPtrsPerLaunch travel in the lead kernel's own arguments (it puts
+  // them into the device table); more, or a selection that lives on the device, take a launch.
+  const bool fine_mask = mask && !mask->coarse;
+  const bool by_args = !sel && !fine_mask && K <= (uint32_t)kPtrsPerLaunch;
+  static thread_local PtrChunk chunk;   // 3.8 KB: kept off the stack
+  if (by_args) memcpy(chunk.p, h_cands, K * sizeof(void*));
 
   // with a device-resident selection the later kernels read the effective candidate count
-  const unsigned int* count = sel ? ctx->d_status + 4 : nullptr;
+  unsigned int* eff_count = ctx->d_status + 4;
+  const unsigned int* count = sel ? eff_count : nullptr;
   if (sel) {
     screen_prep_indexed_kernel<<<1, 256, 0, st>>>(sel->d_table, sel->K_all, sel->d_index, sel->d_count, K,
-                                                  table, acc, ctx->d_status, ctx->d_status);
+                                                  table, acc, counters, eff_count, ctx->d_status);
     ++ctx->launches;
     KB_CUDA(ctx, cudaGetLastError());
   }
-  for (uint32_t off = 0; !sel && off < K; off += kPtrsPerLaunch) {
+  for (uint32_t off = 0; !sel && !by_args && off < K; off += kPtrsPerLaunch) {
     PtrChunk ch;
     const uint32_t cnt = (K - off < (uint32_t)kPtrsPerLaunch) ? K - off : (uint32_t)kPtrsPerLaunch;
     memcpy(ch.p, h_cands + off, cnt * sizeof(void*));
-    screen_prep_kernel<<<(cnt + 127) / 128, 128, 0, st>>>(ch, table, acc, ctx->d_status + 1, off, cnt);
+    screen_prep_kernel<<<(cnt + 127) / 128, 128, 0, st>>>(ch, table, off, cnt);
     ++ctx->launches;
     KB_CUDA(ctx, cudaGetLastError());
   }
@@ -712,7 +778,7 @@ kb_status screen_impl(kb_ctx* ctx, const void* d_ref, const void* const* h_cands
   md.phase = mask ? mask->phase : 0;
   md.bits = mask ? mask->d_bits : nullptr;
 
-  if (mask && !mask->coarse) {
+  if (fine_mask) {
     // finer than a kernel tile: every sector is touched anyway
     rc = launch_generic<DT>(ctx, d_ref, table, acc, K, 0, N, atol, rtol, md, count, st);
     if (rc != KB_OK) return rc;
@@ -736,24 +802,42 @@ kb_status screen_impl(kb_ctx* ctx, const void* d_ref, const void* const* h_cands
       sp.rtol_lean = f;
     }
     sp.status = ctx->d_status;
-    // Scout a few leading tiles exactly (about 1% of the work at most); the streaming
-    // kernel starts behind them with its thresholds seeded.
+    // Lead launch: a few leading tiles scouted exactly (about 1% of the work at most; the
+    // streaming kernel starts behind them with its thresholds seeded), the ragged tail
+    // (elements past the last full kernel tile) and the call's housekeeping.
     uint32_t nscout = 0;
     if (sp.ntiles >= 2) {
       nscout = sp.ntiles / 128;
       if (nscout < 1) nscout = 1;
       if (nscout > 8) nscout = 8;
-      dim3 sg(nscout * (kTile / kScoutPerBlock), K);
-      screen_scout_kernel<DT><<<sg, 256, 0, st>>>(d_ref, table, acc, sp.tile_list, atol, rtol, count);
+    }
+    const uint64_t tail0 = nfull * kTile;
+    const unsigned int tail_blocks = (unsigned int)((N - tail0 + kScoutPerBlock - 1) / kScoutPerBlock);
+    const unsigned int lead_blocks = nscout * (kTile / kScoutPerBlock) + tail_blocks;
+    {
+      LeadParams lp;
+      lp.ref = d_ref;
+      lp.table = table;
+      lp.acc = acc;
+      lp.acc_next = acc_next;
+      lp.counters_next = counter_set(ctx, set ^ 1);
+      lp.tile_list = sp.tile_list;
+      lp.nscout = nscout;
+      lp.n_clear = ctx->used_K[set ^ 1];
+      lp.from_args = by_args ? 1u : 0u;
+      lp.tail0 = tail0;
+      lp.N = N;
+      lp.atol = atol;
+      lp.rtol = rtol;
+      lp.mask = md;
+      lp.count = count;
+      screen_lead_kernel<DT><<<dim3(lead_blocks ? lead_blocks : 1u, K), 256, 0, st>>>(lp, chunk);
       ++ctx->launches;
       KB_CUDA(ctx, cudaGetLastError());
+      lead_ran = true;
     }
     sp.slot0 = nscout;
     sp.ntiles -= nscout;
-    // ragged tail (elements past the last full kernel tile), before the streaming
-    // kernel so that its last CTA can unpack the finished records
-    rc = launch_generic<DT>(ctx, d_ref, table, acc, K, nfull * kTile, N, atol, rtol, md, count, st);
-    if (rc != KB_OK) return rc;
     if (sp.ntiles) {
       // chunk the candidates: shared-memory accumulators hold kMaxKC of them, and
       // small tensors need more, smaller items to fill the machine
@@ -768,16 +852,17 @@ kb_status screen_impl(kb_ctx* ctx, const void* d_ref, const void* const* h_cands
       }
       sp.KC = (K + nchunks - 1) / nchunks;
       sp.nchunks = (K + sp.KC - 1) / sp.KC;
-      sp.done = ctx->d_status + 1;
-      sp.sched = reinterpret_cast<unsigned long long*>(ctx->d_status + 2);
+      sp.done = counters;
+      sp.sched = reinterpret_cast<unsigned long long*>(counters + 2);
       sp.out = d_out;
-      return launch_stream<DT>(ctx, sp, st);
+      rc = launch_stream<DT>(ctx, sp, st);
+      return rc == KB_OK ? finished() : rc;
     }
   }
   screen_finalize_kernel<<<(K + 127) / 128, 128, 0, st>>>(acc, d_out, K, count);
   ++ctx->launches;
   KB_CUDA(ctx, cudaGetLastError());
-  return KB_OK;
+  return finished();
 }
 
 kb_status screen_dispatch(kb_ctx* ctx, const void* d_ref, const void* const* h_cands, uint32_t K,
@@ -828,10 +913,12 @@ extern "C" kb_status kb_screen_f64(kb_ctx* ctx, const double* d_ref, const doubl
   }
   DeviceGuard g(ctx->device);
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-  kb_status rc = ensure_ws(ctx, K, sizeof(Acc64));
+  kb_status rc = ensure_ws(ctx, K);
   if (rc != KB_OK) return rc;
-  Acc64* acc = reinterpret_cast<Acc64*>(ctx->ws);
-  const void** table = reinterpret_cast<const void**>(ctx->ws + round_up((size_t)K * sizeof(Acc64), 256));
+  // its own accumulator region and counters, zeroed by its prep kernel: independent of the
+  // binary32 gate's two sets
+  Acc64* acc = reinterpret_cast<Acc64*>(ctx->ws + ws_acc64_offset(ctx->ws_cap_K));
+  const void** table = reinterpret_cast<const void**>(ctx->ws + ws_table_offset(ctx->ws_cap_K));
   for (uint32_t off = 0; off < K; off += kPtrsPerLaunch) {
     PtrChunk ch;
     const uint32_t cnt = (K - off < (uint32_t)kPtrsPerLaunch) ? K - off : (uint32_t)kPtrsPerLaunch;
@@ -1012,11 +1099,11 @@ extern "C" kb_status kb_screen_multi(kb_ctx* ctx, uint32_t G, const void* const*
 // kb_screen_static: the gate without any allocation
 // ---------------------------------------------------------------------------
 
-// Scratch of the allocation-free entry point: [status words 256 B | accumulators | pointer
-// table].  In host code this name is only a handle for cudaGetSymbolAddress; it is not a
+// Scratch of the allocation-free entry point: [status words and counters 256 B | two sets of
+// accumulators | pointer table].  In host code this name is only a handle for cudaGetSymbolAddress; it is not a
 // device address and must never be passed to a kernel as it stands.
 static __device__ __align__(256) unsigned char g_static_scratch[KB_STATIC_SCRATCH_BYTES];
-static_assert(KB_STATIC_SCRATCH_BYTES == 256 + KB_STATIC_MAX_K * sizeof(Acc) + KB_STATIC_MAX_K * sizeof(void*),
+static_assert(KB_STATIC_SCRATCH_BYTES == 256 + 2 * KB_STATIC_MAX_K * sizeof(Acc) + KB_STATIC_MAX_K * sizeof(void*),
               "the header's scratch size must match the accumulator layout");
 
 namespace {
@@ -1045,6 +1132,7 @@ kb_status static_setup(int device, kb_ctx** out) {
     ctx->d_status = reinterpret_cast<unsigned int*>(base);
     ctx->ws = base + 256;
     ctx->ws_bytes = KB_STATIC_SCRATCH_BYTES - 256;   // ensure_ws never grows it: K is capped
+    ctx->ws_cap_K = KB_STATIC_MAX_K;
     ctx->ws_fixed = true;
     kb_status st;
     if ((st = set_stream_attr<KB_F32>(ctx)) != KB_OK) return st;
@@ -1081,6 +1169,11 @@ extern "C" kb_status kb_screen_static(const void* d_ref, const void* const* h_ca
   kb_ctx* ctx = nullptr;
   kb_status rc = static_setup(device, &ctx);
   if (rc == KB_OK) rc = validate_screen(ctx, d_ref, h_cands, K, N, dtype, atol, rtol, nullptr, d_out, true);
+  if (rc == KB_OK) {
+    // The array is shared by every caller on the device and keeps what the last call left:
+    // nothing is taken on trust, the part this call uses is cleared first.
+    ctx->ws_dirty = true;
+  }
   if (rc == KB_OK)
     rc = screen_dispatch(ctx, d_ref, h_cands, K, N, dtype, atol, rtol, nullptr, d_out,
                          reinterpret_cast<cudaStream_t>(stream));

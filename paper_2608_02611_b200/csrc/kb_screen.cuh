@@ -11,10 +11,16 @@
 //   exact path.  Merges are integer adds and integer maxima on packed keys, so
 //   the result does not depend on order.  The last CTA to finish unpacks the
 //   K records.
-// screen_scout_kernel   classifies a few leading tiles exactly before the
-//   streaming kernel starts; their maxima seed its thresholds.
+// screen_lead_kernel    classifies a few leading tiles exactly before the
+//   streaming kernel starts (their maxima seed its thresholds), and the ragged
+//   tail past the last full tile; it also does the call's housekeeping (pointer
+//   table from its own arguments, zeroing of the accumulators the NEXT call
+//   will use), so that a call of up to 480 candidates is two launches.
 // screen_generic_kernel plain loads, every element classified exactly; used
-//   for the ragged tail tile and for masks finer than a kernel tile.
+//   for masks finer than a kernel tile.
+// Accumulators and counters exist twice: a call works on one set while its
+//   lead kernel zeroes the other for the call after it, so no call needs a
+//   zeroing launch and the streaming kernel's epilogue stays a plain unpack.
 // screen_small_kernel / screen_multi_kernel  the latency regime: one launch
 //   for a small problem / for several small problems of different shapes.
 // screen_prep_kernel / screen_prep_indexed_kernel  pointer table, zeroed
@@ -90,6 +96,13 @@ __device__ __forceinline__ void unpack_record(const Acc& a, kb_screen_result* ds
   r.pass = a.mism == 0ull ? 1u : 0u;
   r.reserved = 0u;
   *dst = r;
+}
+
+__device__ __forceinline__ void clear_acc(Acc* a) {
+  Acc z;
+  z.mism = z.nan = z.inf = z.spare = z.key = 0ull;
+  z.rel = z.pad = 0u;
+  *a = z;
 }
 
 // record of a candidate slot that holds no candidate (indexed screening with fewer
@@ -735,22 +748,40 @@ __global__ void __launch_bounds__(256) screen_generic_kernel(const void* __restr
   x.commit(&acc[k]);
 }
 
-// Scout: the first `nscout` full tiles (of the list, or tiles 0..nscout-1) of every
-// candidate, classified exactly before the streaming kernel starts.  Their maxima
-// seed the streaming kernel's thresholds, so that its first tile does not have to
-// discover them.  A block takes 1024 elements of one tile of one candidate and issues
-// one set of atomics.  grid = (nscout * 4, K).
+// Lead kernel: (1) the first `nscout` full tiles (of the list, or tiles 0..nscout-1) of every
+// candidate, classified exactly before the streaming kernel starts: their maxima seed the
+// streaming kernel's thresholds, so that its first tile does not have to discover them;
+// (2) the ragged tail [tail0, N) past the last full tile, under the mask; (3) housekeeping by
+// the blocks with blockIdx.x == 0: candidate k's pointer goes from the kernel's arguments to
+// the device table the streaming kernel reads (when `from_args`), and the accumulators and
+// counters of the OTHER set -- the one the next call will work on -- are zeroed (nobody else
+// touches them during this call).  A block takes 1024 elements of one candidate and issues
+// one set of atomics.  grid = (max(1, nscout * 4 + ceil((N - tail0) / 1024)), K).
 constexpr unsigned int kScoutPerBlock = 1024;
+struct LeadParams {
+  const void* ref;
+  const void** table;           // device pointer table [K]
+  Acc* acc;                     // this call's accumulators (zero on entry)
+  Acc* acc_next;                // the other set: entries [0, n_clear) are zeroed here
+  unsigned int* counters_next;  // the other set's ticket and work counters (3 words)
+  const uint32_t* tile_list;
+  unsigned int nscout, n_clear, from_args;
+  unsigned long long tail0, N;
+  float atol, rtol;
+  MaskDev mask;
+  const unsigned int* count;
+};
 template <int DT>
-__global__ void __launch_bounds__(256) screen_scout_kernel(const void* __restrict__ ref,
-                                                           const void* const* __restrict__ cands,
-                                                           Acc* __restrict__ acc,
-                                                           const uint32_t* __restrict__ tile_list,
-                                                           float atol, float rtol,
-                                                           const unsigned int* __restrict__ count) {
+__global__ void __launch_bounds__(256) screen_lead_kernel(const LeadParams p, const __grid_constant__ PtrChunk chunk_ptrs) {
   using E = Elem<DT>;
   constexpr unsigned int kBlocksPerTile = kTile / kScoutPerBlock;
-  if (count && blockIdx.y >= *count) return;
+  const unsigned int k = blockIdx.y;
+  if (blockIdx.x == 0) {
+    if (threadIdx.x == 0 && p.from_args) p.table[k] = chunk_ptrs.p[k];
+    for (unsigned int j = k + gridDim.y * threadIdx.x; j < p.n_clear; j += gridDim.y * 256u) clear_acc(&p.acc_next[j]);
+    if (k == 0 && threadIdx.x < 3) p.counters_next[threadIdx.x] = 0u;
+  }
+  if (p.count && k >= *p.count) return;
   __shared__ unsigned int s_cnt[3];
   __shared__ unsigned int s_rel;
   __shared__ unsigned long long s_key;
@@ -760,16 +791,25 @@ __global__ void __launch_bounds__(256) screen_scout_kernel(const void* __restric
     s_key = 0ull;
   }
   __syncthreads();
-  const unsigned int k = blockIdx.y;
-  const unsigned int slot = blockIdx.x / kBlocksPerTile;
-  const unsigned long long tile = tile_list ? tile_list[slot] : slot;
-  const unsigned long long base = tile * kTile + (blockIdx.x % kBlocksPerTile) * kScoutPerBlock;
-  const void* cand = cands[k];
+  const void* cand = p.from_args ? chunk_ptrs.p[k] : p.table[k];
   ExactAcc x;
+  if (blockIdx.x < p.nscout * kBlocksPerTile) {
+    const unsigned int slot = blockIdx.x / kBlocksPerTile;
+    const unsigned long long tile = p.tile_list ? p.tile_list[slot] : slot;
+    const unsigned long long base = tile * kTile + (blockIdx.x % kBlocksPerTile) * kScoutPerBlock;
 #pragma unroll
-  for (unsigned int j = 0; j < kScoutPerBlock / 256; ++j) {
-    const unsigned long long i = base + j * 256 + threadIdx.x;
-    x.add(E::load(ref, i), E::load(cand, i), i, atol, rtol);
+    for (unsigned int j = 0; j < kScoutPerBlock / 256; ++j) {
+      const unsigned long long i = base + j * 256 + threadIdx.x;
+      x.add(E::load(p.ref, i), E::load(cand, i), i, p.atol, p.rtol);
+    }
+  } else {
+    const unsigned long long base =
+        p.tail0 + (unsigned long long)(blockIdx.x - p.nscout * kBlocksPerTile) * kScoutPerBlock;
+#pragma unroll
+    for (unsigned int j = 0; j < kScoutPerBlock / 256; ++j) {
+      const unsigned long long i = base + j * 256 + threadIdx.x;
+      if (i < p.N && mask_selected(p.mask, i)) x.add(E::load(p.ref, i), E::load(cand, i), i, p.atol, p.rtol);
+    }
   }
   // block-level merge in shared memory, then one set of global atomics
   x.n_mis = warp_add_u32(x.n_mis);
@@ -786,7 +826,7 @@ __global__ void __launch_bounds__(256) screen_scout_kernel(const void* __restric
   }
   __syncthreads();
   if (threadIdx.x == 0) {
-    Acc* a = &acc[k];
+    Acc* a = &p.acc[k];
     if (s_cnt[0]) atomicAdd(&a->mism, (unsigned long long)s_cnt[0]);
     if (s_cnt[1]) atomicAdd(&a->nan, (unsigned long long)s_cnt[1]);
     if (s_cnt[2]) atomicAdd(&a->inf, (unsigned long long)s_cnt[2]);
@@ -977,22 +1017,11 @@ __global__ void screen_finalize_kernel(const Acc* __restrict__ acc, kb_screen_re
     unpack_record(acc[k], &out[k]);
 }
 
-// Also zeroes the accumulators of the same candidates and the ticket counter.
-__global__ void screen_prep_kernel(const PtrChunk chunk, const void** table, Acc* acc,
-                                   unsigned int* done, unsigned int offset, unsigned int count) {
+// Candidate pointers of a call with more than kPtrsPerLaunch candidates go to the device table.
+__global__ void screen_prep_kernel(const PtrChunk chunk, const void** table, unsigned int offset,
+                                   unsigned int count) {
   const unsigned int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < count) {
-    table[offset + i] = chunk.p[i];
-    Acc z;
-    z.mism = z.nan = z.inf = z.spare = z.key = 0ull;
-    z.rel = z.pad = 0u;
-    acc[offset + i] = z;
-  }
-  if (i == 0) {
-    done[0] = 0u;   // ticket counter
-    done[1] = 0u;   // work counter (64 bits)
-    done[2] = 0u;
-  }
+  if (i < count) table[offset + i] = chunk.p[i];
 }
 
 // Indexed screening: candidate slot j holds table[index[j]] for j < *count.  Builds the
@@ -1003,8 +1032,8 @@ __global__ void screen_prep_kernel(const PtrChunk chunk, const void** table, Acc
 __global__ void screen_prep_indexed_kernel(const void* const* __restrict__ all, unsigned int K_all,
                                            const int* __restrict__ index,
                                            const unsigned int* __restrict__ count, unsigned int Kmax,
-                                           const void** table, Acc* acc, unsigned int* words,
-                                           unsigned int* status) {
+                                           const void** table, Acc* acc, unsigned int* counters,
+                                           unsigned int* eff_count, unsigned int* status) {
   // single block: Kmax <= 1024 slots
   __shared__ unsigned int s_bad;
   if (threadIdx.x == 0) s_bad = 0u;
@@ -1030,10 +1059,10 @@ __global__ void screen_prep_indexed_kernel(const void* const* __restrict__ all, 
   }
   __syncthreads();
   if (threadIdx.x == 0) {
-    words[1] = 0u;   // ticket counter
-    words[2] = 0u;   // work counter (64 bits)
-    words[3] = 0u;
-    words[4] = s_bad ? 0u : n;   // effective number of candidates
+    counters[0] = 0u;   // ticket counter
+    counters[1] = 0u;   // work counter (64 bits)
+    counters[2] = 0u;
+    *eff_count = s_bad ? 0u : n;   // effective number of candidates
     if (s_bad) set_status(status, (unsigned int)((s_bad & 2u) ? KB_ERR_ALIGNMENT : KB_ERR_INVALID_ARG));
   }
 }

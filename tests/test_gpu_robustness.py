@@ -266,8 +266,8 @@ def test_guard_bands_around_adjudication_and_selection_outputs(ctx, kb, K, S):
 
 
 def test_static_scratch_is_untouched_beyond_the_part_a_call_uses(kb):
-    """kb_screen_static with K candidates uses the status words, K accumulators and K table
-    entries of its fixed array; every byte beyond them keeps its value."""
+    """kb_screen_static with K candidates uses the status words, K accumulators of either set and
+    K table entries of its fixed array; every byte beyond them keeps its value."""
     dev = torch.device("cuda", 0)
     rng = np.random.default_rng(9)
     N = 3 * 4096 + 11
@@ -280,8 +280,59 @@ def test_static_scratch_is_untouched_beyond_the_part_a_call_uses(kb):
     before = kb.static_scratch_read()
     kb.screen_static(ref, cands, 1e-5, 1e-3, out=out)
     after = kb.static_scratch_read()
-    acc_end = 256 + ((K * 48 + 255) // 256) * 256
-    tab_end = acc_end + K * 8
-    assert (after[tab_end:] == before[tab_end:]).all()
-    assert (after[256 + K * 48:acc_end] == before[256 + K * 48:acc_end]).all()
+    # [status words and counters 256 B | accumulators, set 0 | accumulators, set 1 | pointer table]
+    set_bytes = 1024 * 48
+    tab0 = 256 + 2 * set_bytes
+    assert (after[tab0 + K * 8:] == before[tab0 + K * 8:]).all()
+    for s0 in (256, 256 + set_bytes):
+        assert (after[s0 + K * 48:s0 + set_bytes] == 0).all()
     same_records(kb.records(out), oracle_records(synth.F32, ref, cands, 1e-5, 1e-3))
+
+
+def test_general_path_takes_two_launches_and_leaves_its_scratch_clean(ctx, kb):
+    """Up to 480 candidates the streaming gate is two launches (lead: scouted tiles, ragged tail,
+    pointer table, zeroing of the accumulator set the next call uses; streaming kernel, whose
+    last CTA writes the records).  Calls of different sizes, dtypes and precisions follow one
+    another on one context, larger after smaller, so that stale accumulators would show."""
+    dev = torch.device("cuda", 0)
+    ctx.set_small_path(False)
+    rng = np.random.default_rng(21)
+
+    def make(N, K, dtype):
+        tdt = synth.TORCH_DTYPE[dtype]
+        ref = torch.from_numpy(rng.standard_normal(N).astype(np.float32)).to(tdt).to(dev)
+        cands = []
+        for k in range(K):
+            c = ref.clone()
+            if k % 2:
+                idx = torch.from_numpy(rng.integers(0, N, 3)).to(dev)
+                c[idx] = 1.75
+            cands.append(c)
+        return ref, cands
+
+    def run(N, K, dtype, expect_launches):
+        ref, cands = make(N, K, dtype)
+        n0 = ctx.launch_count
+        got = kb.records(ctx.screen(ref, cands, 1e-3, 1e-2))
+        assert ctx.launch_count - n0 == expect_launches, (N, K, ctx.launch_count - n0)
+        same_records(got, oracle_records(dtype, ref, cands, 1e-3, 1e-2))
+
+    run(40 * 4096 + 5, 30, synth.BF16, 2)          # scout + tail | stream
+    run(40 * 4096, 7, synth.F16, 2)                # scout | stream
+    run(4096, 3, synth.F32, 2)                     # one tile, nothing to scout, no tail: housekeeping | stream
+    run(4096 + 1, 100, synth.F32, 2)               # tail | stream
+    run(12 * 4096 + 100, 481, synth.BF16, 4)       # pointer table: 2 x prep | lead | stream
+    run(300, 5, synth.F32, 2)                      # no full tile: lead (tail) | finalize
+    run(40 * 4096 + 5, 30, synth.BF16, 2)
+    # the double-precision gate uses the same workspace with another layout
+    ref64 = torch.from_numpy(rng.standard_normal(9000)).to(dev)
+    c64 = [ref64.clone(), ref64 + 1e-3]
+    got = kb.records_f64(ctx.screen_f64(ref64, c64, 1e-12, 1e-9))
+    same_records(got, oracle.screen_f64(ref64.cpu().numpy(), [c.cpu().numpy() for c in c64], 1e-12, 1e-9))
+    run(40 * 4096 + 5, 30, synth.BF16, 2)
+    run(40 * 4096 + 5, 200, synth.BF16, 2)         # more candidates than either set has seen cleaned
+    run(40 * 4096 + 5, 9, synth.F16, 2)
+    run(40 * 4096 + 5, 200, synth.BF16, 2)
+    run(9 * 4096, 190, synth.F32, 2)
+    assert ctx.poll() == 0
+    assert ctx.check_guards()[1] == 0
