@@ -277,6 +277,79 @@ def run_screen(args):
     ctx.close()
 
 
+# Largest output of each of the paper's six benchmarks (Appendix "Benchmark Descriptions and
+# Shapes"): MatVec M=2048; GroupConv 217800 x 20; LinearReLUDiv 1024 x 8192; SDPAttn
+# 32 x 32 x 512 x 1024; RMSNorm 16 x 64 x 768 x 768; Softmax 4096 x 393216.
+PAPER_SHAPES = [("MatVec", 2048), ("GroupConv", 217800 * 20), ("LinearReLUDiv", 1024 * 8192),
+                ("SDPAttn", 32 * 32 * 512 * 1024), ("RMSNorm", 16 * 64 * 768 * 768),
+                ("Softmax", 4096 * 393216)]
+
+
+def run_paper_scale(args):
+    """kb_screen at the paper's own scale: the six benchmark output sizes x the candidate counts of
+    its funnel (21 -> 7 -> 3), bf16 and fp32, default dispatch.  One JSON line per entry: time per
+    call (CUDA events around back-to-back calls, no kernel timers), bytes/s of (K+1)*N*sizeof
+    against the measured HBM peak, launches per call.  Secondary measurement."""
+    import torch
+    from paper_2608_02611_b200 import binding
+    dev = torch.device("cuda", 0)
+    ctx = binding.Context(0)
+    peak, src = peaks()
+    calls = max(3, min(args.steps, 20))
+    for name, N in PAPER_SHAPES:
+        for dname, tdt, idt in (("bf16", torch.bfloat16, torch.int16), ("f32", torch.float32, torch.int32)):
+            esz = 2 if dname == "bf16" else 4
+            g = torch.Generator(device=dev)
+            g.manual_seed(20260802)
+            ref = None
+            for K in (21, 7, 3):
+                if (K + 1) * N * esz > 100e9:
+                    print(json.dumps({"benchmark": name, "N": N, "dtype": dname, "K": K,
+                                      "skipped": "more than 100 GB of tensors"}), flush=True)
+                    continue
+                if ref is None:
+                    ref = torch.empty(N, dtype=tdt, device=dev)
+                    for s0 in range(0, N, 1 << 27):           # in slices: no full-size fp32 temporary
+                        ref[s0:s0 + (1 << 27)] = torch.randn(min(1 << 27, N - s0), dtype=torch.float32,
+                                                             device=dev, generator=g).to(tdt)
+                    cands = []
+                while len(cands) < K:                         # one-ulp differences on 1% of the elements
+                    c = ref.clone()
+                    c.view(idt)[len(cands)::101] += 1
+                    cands.append(c)
+                cs = cands[:K]
+                out = torch.empty((K, binding.RESULT_BYTES), dtype=torch.uint8, device=dev)
+                for _ in range(3):
+                    ctx.screen(ref, cs, 1e-2, 1.6e-2, out=out)
+                torch.cuda.synchronize()
+                # the C entry point itself with its arguments marshalled once: the Python
+                # binding's own 10-15 us per call would otherwise hide the small cases
+                import ctypes
+                L = binding.load()
+                ptrs = (ctypes.c_void_p * K)(*[c.data_ptr() for c in cs])
+                a = (ctx._h, ref.data_ptr(), ptrs, K, N, binding.DTYPE_CODE[tdt], 1e-2, 1.6e-2, None,
+                     out.data_ptr(), int(torch.cuda.current_stream(dev).cuda_stream))
+                n0 = ctx.launch_count
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(calls):
+                    L.kb_screen(*a)
+                e1.record()
+                torch.cuda.synchronize()
+                us = e0.elapsed_time(e1) / calls * 1e3
+                assert ctx.poll() == 0
+                rec = binding.records(out)
+                gbs = (K + 1) * N * esz / (us * 1e-6) / 1e9
+                print(json.dumps({"benchmark": name, "N": N, "dtype": dname, "K": K, "us_per_call": us,
+                                  "gbs": gbs, "frac_of_measured_hbm": gbs / peak,
+                                  "launches_per_call": (ctx.launch_count - n0) / calls,
+                                  "all_pass": bool((rec["pass"] == 1).all()), "calls": calls}), flush=True)
+            del ref
+            cands = []
+            torch.cuda.empty_cache()
+    ctx.close()
+
+
 def relaunch_ranks(n: int):
     """`python bench.py --gpus N` without a launcher: start N ranks (one process per GPU) under
     torch.distributed.run on this node, with the same arguments, and pass their output on."""
@@ -301,7 +374,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--workload", default="step", choices=["step", "adjudicate", "screen"],
+    ap.add_argument("--workload", default="step", choices=["step", "adjudicate", "screen", "paper-scale"],
                     help="'adjudicate' times kb_adjudicate alone on timings[K][S] (config 5 tier 1 by "
                          "default) and reports pairwise comparisons/s against the ALU roofline; it is a "
                          "secondary measurement, not the benchmark line")
@@ -324,6 +397,8 @@ def main():
         return run_adjudicate(args)
     if args.workload == "screen":
         return run_screen(args)
+    if args.workload == "paper-scale":
+        return run_paper_scale(args)
 
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         return relaunch_ranks(args.gpus)
