@@ -26,6 +26,16 @@ kb_status kb_ctx_set_grid(kb_ctx* ctx, uint32_t blocks);
  * (streaming) path instead.  Results do not depend on it. */
 kb_status kb_ctx_set_small_path(kb_ctx* ctx, int on);
 
+/* Test/tuning hook: which instantiation of the streaming screen kernel runs.  0 = automatic
+ * (the plain one, until a call reports that a quarter of its steps took a second look that
+ * found nothing -- many elements whose quotient was rounded down to the largest relative
+ * error, e.g. dense one-ulp differences -- then the one that applies the sharper test to
+ * every element, with a plain call every 32 calls to see whether that still holds),
+ * 1 = always plain, 2 = always sharp.  Results do not depend on it. */
+kb_status kb_ctx_set_filter(kb_ctx* ctx, int mode);
+/* Whether the last streaming launch of this context used the sharp instantiation (HOST out: 1 or 0). */
+kb_status kb_ctx_last_filter(const kb_ctx* ctx, int* sharp);
+
 /* ---- instrumentation (used by the benchmark) ------------------------------ */
 
 typedef enum {

@@ -47,7 +47,7 @@ EXPORTS = [
     "kb_mask_create_strided", "kb_mask_create_bitmap", "kb_mask_count", "kb_mask_destroy",
     "kb_screen", "kb_screen_f64", "kb_screen_host", "kb_screen_static", "kb_screen_indexed", "kb_screen_multi", "kb_adjudicate", "kb_adjudicate_ragged", "kb_select",
     "kb_select_by_score", "kb_tail_ratios", "kb_copeland", "kb_confirm",
-    "kb_ctx_fail_next_allocs", "kb_ctx_selftest_wait", "kb_ctx_check_guards", "kb_static_scratch_read",
+    "kb_ctx_fail_next_allocs", "kb_ctx_selftest_wait", "kb_ctx_check_guards", "kb_static_scratch_read", "kb_ctx_set_filter", "kb_ctx_last_filter",
 ]
 
 
@@ -85,6 +85,8 @@ def load() -> ctypes.CDLL:
     L.kb_ctx_launch_count.argtypes = [vp, ctypes.POINTER(u64)]
     L.kb_ctx_set_wins_algo.argtypes = [vp, i32]
     L.kb_ctx_set_small_path.argtypes = [vp, i32]
+    L.kb_ctx_set_filter.argtypes = [vp, i32]
+    L.kb_ctx_last_filter.argtypes = [vp, ctypes.POINTER(i32)]
     L.kb_ctx_fail_next_allocs.argtypes = [vp, u32, u32]
     L.kb_ctx_check_guards.argtypes = [vp, vp, ctypes.POINTER(u32), ctypes.POINTER(u32)]
     L.kb_static_scratch_read.argtypes = [vp, u32]
@@ -188,6 +190,16 @@ class Context:
     def set_small_path(self, on: bool):
         """Enable/disable the single-launch kernel for small problems (a test hook)."""
         self._check(load().kb_ctx_set_small_path(self._h, 1 if on else 0), "kb_ctx_set_small_path")
+
+    def set_filter(self, mode: int):
+        """0 automatic, 1 always the plain streaming kernel, 2 always the sharp one (a tuning hook)."""
+        self._check(load().kb_ctx_set_filter(self._h, int(mode)), "kb_ctx_set_filter")
+
+    @property
+    def last_filter_sharp(self) -> bool:
+        v = ctypes.c_int(0)
+        self._check(load().kb_ctx_last_filter(self._h, ctypes.byref(v)), "kb_ctx_last_filter")
+        return bool(v.value)
 
     def set_wins_algo(self, algo: int):
         """0 automatic, 1 direct comparison of all sample pairs, 2 binary search on sorted rows,

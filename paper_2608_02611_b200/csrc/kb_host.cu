@@ -34,8 +34,21 @@ struct kb_ctx {
   int ws_parity = 0;
   uint32_t used_K[2] = {0, 0};
   bool ws_dirty = true;
+  // Choice between the two instantiations of the streaming kernel.  The plain one reports, in a
+  // host-visible word, the share of its warp steps that took a fruitless second look; when the
+  // last report says a quarter or more, the next calls use the sharp instantiation, and every
+  // so often one of them probes the plain one again.  filter_mode: 0 automatic, 1 plain, 2 sharp.
+  unsigned int* h_hint = nullptr;   // pinned, mapped
+  unsigned int* d_hint = nullptr;   // its device address
+  int filter_mode = 0;
+  int sharp_left = 0;
+  bool sharp_probe_next = false, sharp_probed = false;
+  bool last_sharp = false;          // the last streaming launch used the sharp instantiation
+  float call_steps = 0.0f;          // warp steps of the current call's plain streaming launch (0: none)
+  float steps_hist[2] = {0.0f, 0.0f};   // the same for the last call on each accumulator set
   // [0] status, [1..3] counters of the binary64 gate, [4] effective K of an indexed call,
-  // [8..10] and [16..18] the two counter sets of the binary32 gate, [60] probe sink
+  // [8..10] and [16..18] the two counter sets of the binary32 gate, [20..23] two 64-bit sums of
+  // fruitless second looks on their way to the host, [60] probe sink
   unsigned int* d_status = nullptr;
   uint32_t forced_grid = 0;
   unsigned char* small_ws = nullptr; // single-launch path: [tickets 4 KB | partial records 384 KB]
@@ -216,6 +229,7 @@ kb_status ensure_ws(kb_ctx* ctx, uint32_t K) {
 // ring depth by stage size: 3 CTAs/SM must fit ~75 KB each
 inline uint32_t stream_stages(uint32_t tile_bytes) { return tile_bytes >= 16384 ? 3 : tile_bytes >= 8192 ? 7 : 10; }
 
+constexpr int kSharpCalls = 32, kSharpGrace = 4;
 template <int DT>
 kb_status launch_stream(kb_ctx* ctx, StreamParams& sp, cudaStream_t st) {
   const uint32_t tile_bytes = kTile * Elem<DT>::kBytes;
@@ -224,9 +238,41 @@ kb_status launch_stream(kb_ctx* ctx, StreamParams& sp, cudaStream_t st) {
   const unsigned long long nitems = (unsigned long long)sp.nchunks * sp.ntiles;
   unsigned long long grid = ctx->forced_grid ? ctx->forced_grid : 3ull * ctx->sm_count;
   if (grid > nitems) grid = nitems;
+  // which instantiation: what the last finished plain call on this context reported
+  // Plain until a plain launch reports that a quarter of its warp steps took a fruitless
+  // second look; then sharp for kSharpCalls launches, one plain launch as a probe, sharp again
+  // for the kSharpGrace launches its report needs to arrive, and the report decides.
+  bool sharp = ctx->filter_mode == 2;
+  if (ctx->filter_mode == 0 && ctx->h_hint) {
+    volatile unsigned int* hint = reinterpret_cast<volatile unsigned int*>(ctx->h_hint);
+    if (ctx->sharp_left > 0) {
+      sharp = true;
+      if (--ctx->sharp_left == 0 && !ctx->sharp_probed) {
+        ctx->sharp_probe_next = true;          // the next launch is the probe
+      } else if (ctx->sharp_left == 0) {
+        ctx->sharp_probed = false;             // the grace period is over: the report decides below
+      }
+    } else if (ctx->sharp_probe_next) {
+      ctx->sharp_probe_next = false;
+      ctx->sharp_probed = true;
+      ctx->sharp_left = kSharpGrace;
+      *hint = 0u;
+    } else if (*hint >= 16u) {                 // a quarter of the steps
+      sharp = true;
+      ctx->sharp_left = kSharpCalls - 1;
+      ctx->sharp_probed = false;
+      *hint = 0u;                              // the next plain launch reports afresh
+    }
+  }
+  ctx->last_sharp = sharp;
+  // warp steps of this launch if it counts its fruitless second looks (see LeadParams)
+  ctx->call_steps = sharp ? 0.0f : (float)sp.ntiles * (float)sp.K * (float)kWarps;
   {
     ScopedTimer tm(ctx, KB_TIMER_SCREEN_STREAM, st);
-    screen_stream_kernel<DT><<<(unsigned int)grid, kStreamThreads, smem, st>>>(sp);
+    if (sharp)
+      screen_stream_kernel<DT, true><<<(unsigned int)grid, kStreamThreads, smem, st>>>(sp);
+    else
+      screen_stream_kernel<DT, false><<<(unsigned int)grid, kStreamThreads, smem, st>>>(sp);
   }
   ++ctx->launches;
   KB_CUDA(ctx, cudaGetLastError());
@@ -253,9 +299,14 @@ template <int DT>
 kb_status set_stream_attr(kb_ctx* ctx) {
   const uint32_t tile_bytes = kTile * Elem<DT>::kBytes;
   const size_t smem = stream_smem_bytes(stream_stages(tile_bytes), tile_bytes);
-  KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT>,
+  KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT, false>,
                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT>,
+  KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT, false>,
+                                    cudaFuncAttributePreferredSharedMemoryCarveout,
+                                    (int)cudaSharedmemCarveoutMaxShared));
+  KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT, true>,
+                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT, true>,
                                     cudaFuncAttributePreferredSharedMemoryCarveout,
                                     (int)cudaSharedmemCarveoutMaxShared));
   return KB_OK;
@@ -323,6 +374,18 @@ extern "C" kb_status kb_ctx_create(int device, kb_ctx** out) {
     fail(ctx, KB_ERR_WORKSPACE, "cannot allocate the small-problem workspace");
     return bail(KB_ERR_WORKSPACE);
   }
+  // the hint word is optional: without it the plain instantiation always runs
+  if (cudaHostAlloc(reinterpret_cast<void**>(&ctx->h_hint), 64, cudaHostAllocMapped) == cudaSuccess) {
+    memset(ctx->h_hint, 0, 64);
+    if (cudaHostGetDevicePointer(reinterpret_cast<void**>(&ctx->d_hint), ctx->h_hint, 0) != cudaSuccess) {
+      cudaFreeHost(ctx->h_hint);
+      ctx->h_hint = nullptr;
+      ctx->d_hint = nullptr;
+    }
+  } else {
+    ctx->h_hint = nullptr;
+  }
+  cudaGetLastError();
   if ((st = set_stream_attr<KB_F32>(ctx)) != KB_OK) return bail(st);
   if ((st = set_stream_attr<KB_F16>(ctx)) != KB_OK) return bail(st);
   if ((st = set_stream_attr<KB_BF16>(ctx)) != KB_OK) return bail(st);
@@ -373,6 +436,7 @@ extern "C" kb_status kb_ctx_destroy(kb_ctx* ctx) {
     if (ctx->ev_done[i]) cudaEventDestroy(ctx->ev_done[i]);
   }
   ctx_free(ctx, ctx->st_out);
+  if (ctx->h_hint) cudaFreeHost(ctx->h_hint);
   if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
   for (int t = 0; t < kb_ctx::kTimers; ++t)
     for (int i = 0; i < kb_ctx::kPool; ++i) {
@@ -402,6 +466,21 @@ extern "C" kb_status kb_ctx_poll(kb_ctx* ctx, void* stream, kb_status* device_st
 extern "C" kb_status kb_ctx_set_grid(kb_ctx* ctx, uint32_t blocks) {
   if (!ctx) return KB_ERR_INVALID_ARG;
   ctx->forced_grid = blocks;
+  return KB_OK;
+}
+
+extern "C" kb_status kb_ctx_set_filter(kb_ctx* ctx, int mode) {
+  if (!ctx || mode < 0 || mode > 2) return KB_ERR_INVALID_ARG;
+  ctx->filter_mode = mode;
+  ctx->sharp_left = 0;
+  ctx->sharp_probe_next = ctx->sharp_probed = false;
+  if (ctx->h_hint) *reinterpret_cast<volatile unsigned int*>(ctx->h_hint) = 0u;
+  return KB_OK;
+}
+
+extern "C" kb_status kb_ctx_last_filter(const kb_ctx* ctx, int* sharp) {
+  if (!ctx || !sharp) return KB_ERR_INVALID_ARG;
+  *sharp = ctx->last_sharp ? 1 : 0;
   return KB_OK;
 }
 
@@ -726,8 +805,9 @@ kb_status screen_impl(kb_ctx* ctx, const void* d_ref, const void* const* h_cands
   const bool capturing = cap != cudaStreamCaptureStatusNone;
   if (capturing || ctx->ws_dirty) {
     KB_CUDA(ctx, cudaMemsetAsync(ctx->ws, 0, 2 * ws_region(ctx->ws_cap_K), st));
-    KB_CUDA(ctx, cudaMemsetAsync(counter_set(ctx, 0), 0, 16 * sizeof(unsigned int), st));   // both sets
+    KB_CUDA(ctx, cudaMemsetAsync(counter_set(ctx, 0), 0, 16 * sizeof(unsigned int), st));   // both sets, the sums
     ctx->used_K[0] = ctx->used_K[1] = 0;
+    ctx->steps_hist[0] = ctx->steps_hist[1] = 0.0f;
   }
   const int set = ctx->ws_parity;
   Acc* acc = reinterpret_cast<Acc*>(ctx->ws + (size_t)set * ws_region(ctx->ws_cap_K));
@@ -735,7 +815,9 @@ kb_status screen_impl(kb_ctx* ctx, const void* d_ref, const void* const* h_cands
   unsigned int* counters = counter_set(ctx, set);
   ctx->ws_dirty = true;      // until every launch of this call has been enqueued
   bool lead_ran = false;
+  ctx->call_steps = 0.0f;
   auto finished = [&]() {
+    ctx->steps_hist[set] = ctx->call_steps;
     // the lead kernel has cleaned the other set; without one (or under capture) the next call memsets
     if (lead_ran && !capturing) {
       ctx->used_K[set] = K;
@@ -831,6 +913,14 @@ kb_status screen_impl(kb_ctx* ctx, const void* d_ref, const void* const* h_cands
       lp.rtol = rtol;
       lp.mask = md;
       lp.count = count;
+      // This call (set `set`) clears the previous call's accumulators (set ^ 1) and adds their
+      // looks to sum[set]; sum[set ^ 1] holds the looks of the call before that (the last one on
+      // `set`), added up by the previous lead kernel, and goes out with that call's steps.
+      unsigned long long* sums = reinterpret_cast<unsigned long long*>(ctx->d_status + 20);
+      lp.looks_sum = ctx->d_hint ? sums + set : nullptr;
+      lp.looks_pub = sums + (set ^ 1);
+      lp.hint = ctx->d_hint;
+      lp.pub_steps = ctx->steps_hist[set];
       screen_lead_kernel<DT><<<dim3(lead_blocks ? lead_blocks : 1u, K), 256, 0, st>>>(lp, chunk);
       ++ctx->launches;
       KB_CUDA(ctx, cudaGetLastError());

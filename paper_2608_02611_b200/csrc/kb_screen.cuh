@@ -143,7 +143,7 @@ struct StreamSmem {
   uint64_t* sync_bar;        // consumer-wide barrier with a bounded wait (flush)
   unsigned long long* item_id;   // [stages] (chunk << 32 | position) of the work item whose reference
                                  // tile a stage holds; all ones: no more work
-  unsigned long long* cnt;   // [3][kMaxKC] mism, nan, inf
+  unsigned long long* cnt;   // [4][kMaxKC] mism, nan, inf; fruitless second looks (plain instantiation)
   unsigned long long* key;   // [kMaxKC]
   const void** ptrs;         // [kMaxKC] candidate pointers of the current chunk (producer only)
   unsigned int* rel;         // [kMaxKC] bits of the running max relative error (CTA-wide)
@@ -156,7 +156,7 @@ __host__ __device__ inline size_t stream_smem_bytes(uint32_t stages, uint32_t ti
   size_t b = (size_t)stages * tile_bytes;
   b += (size_t)kMaxKC * 16;
   b += 3 * (size_t)stages * 8 + 8;
-  b += 3 * (size_t)kMaxKC * 8 + (size_t)kMaxKC * 8 + (size_t)kMaxKC * 8 + (size_t)kMaxKC * 4;
+  b += 4 * (size_t)kMaxKC * 8 + (size_t)kMaxKC * 8 + (size_t)kMaxKC * 8 + (size_t)kMaxKC * 4;
   b += (size_t)kMaxKC * kWarps * 8;
   b += 16;
   return b + 128;  // alignment slack
@@ -175,7 +175,17 @@ __host__ __device__ inline size_t stream_smem_bytes(uint32_t stages, uint32_t ti
 // Inf - Inf) to the decision.  While rel <= rtol*(1-2^-20), (c) implies (a):
 // ad <= rel*|r| <= RN(rtol*|r|) <= tol ("lean").  Beyond that the same loop runs with rel
 // clamped to that bound, and only threads for which it fails compare element by element.
-template <int DT>
+//
+// Two instantiations.  SHARP = false is the filter above with a second look for threads whose
+// (c) fails.  SHARP = true applies the second look's sharper test to every element in the main
+// loop (two dependent fused multiply-adds instead of one): a quarter more instructions per
+// step, but no second looks.  It pays when many elements have a quotient that was rounded DOWN
+// to the running maximum (one-ulp differences everywhere whose largest quotient is inexact):
+// the plain kernel then takes a second look on nearly every step.  The plain kernel counts its
+// fruitless second looks per candidate (they travel in the accumulator's spare word); the lead
+// kernels of the following calls add them up and publish their share of all warp steps to the
+// host, which picks the instantiation from it.  The records do not depend on the choice.
+template <int DT, bool SHARP>
 __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
   using E = Elem<DT>;
   constexpr int VEC = E::kVec;
@@ -202,7 +212,7 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
     s.item_id = reinterpret_cast<unsigned long long*>(q);
     q += (size_t)p.stages * 8;
     s.cnt = reinterpret_cast<unsigned long long*>(q);
-    q += 3 * (size_t)kMaxKC * 8;
+    q += 4 * (size_t)kMaxKC * 8;
     s.key = reinterpret_cast<unsigned long long*>(q);
     q += (size_t)kMaxKC * 8;
     s.ptrs = reinterpret_cast<const void**>(q);
@@ -232,6 +242,7 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
     s.cnt[i] = 0ull;
     s.cnt[kMaxKC + i] = 0ull;
     s.cnt[2 * kMaxKC + i] = 0ull;
+    s.cnt[3 * kMaxKC + i] = 0ull;
     s.key[i] = 0ull;
     s.rel[i] = 0u;
     s.xg[i] = make_uint4(0u, 0u, 0u, 0u);
@@ -349,6 +360,8 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
         if ((v = s.key[i]) != 0ull) atomicMax(&a->key, v);
         unsigned int r = s.rel[i];
         if (r != 0u) atomicMax(&a->rel, r);
+        if (!SHARP && (v = s.cnt[3 * kMaxKC + i]) != 0ull) atomicAdd(&a->spare, v);
+        s.cnt[3 * kMaxKC + i] = 0ull;
         s.cnt[i] = 0ull;
         s.cnt[kMaxKC + i] = 0ull;
         s.cnt[2 * kMaxKC + i] = 0ull;
@@ -505,14 +518,39 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
         const bool lean = rel <= p.rtol_lean;
         const float rel_f = (has_lean && !lean) ? p.rtol_lean : rel;
         float mabs = 0.0f, mrel = 0.0f;
+        // g = (ulp(rel)/2)*(1 - 2^-20), or 0 where that would be subnormal
+        auto half_ulp_of_rel = [&]() -> float {
+          const unsigned int rb = __float_as_uint(rel);
+          return rb >= (30u << 23)
+                     ? __uint_as_float((rb & 0x7F800000u) - (24u << 23)) * 0.99999904632568359375f
+                     : 0.0f;
+        };
+        const bool sharp = SHARP && lean;
+        if (!SHARP || !sharp) {
 #pragma unroll
-        for (int e = 0; e < kEPT; e += 2) {
-          float d0, d1;
-          E::pair_diff(words, e, r[e], r[e + 1], d0, d1);
-          const float t0 = fmaf(-rel_f, fabsf(r[e]), fabsf(d0));
-          const float t1 = fmaf(-rel_f, fabsf(r[e + 1]), fabsf(d1));
-          mabs = max3(mabs, fabsf(d0), fabsf(d1));
-          mrel = max3_nan(mrel, t0, t1);
+          for (int e = 0; e < kEPT; e += 2) {
+            float d0, d1;
+            E::pair_diff(words, e, r[e], r[e + 1], d0, d1);
+            const float t0 = fmaf(-rel_f, fabsf(r[e]), fabsf(d0));
+            const float t1 = fmaf(-rel_f, fabsf(r[e + 1]), fabsf(d1));
+            mabs = max3(mabs, fabsf(d0), fabsf(d1));
+            mrel = max3_nan(mrel, t0, t1);
+          }
+        } else {
+          const float g = half_ulp_of_rel();
+#pragma unroll
+          for (int e = 0; e < kEPT; e += 2) {
+            float d0, d1;
+            E::pair_diff(words, e, r[e], r[e + 1], d0, d1);
+            const float ar0 = fabsf(r[e]), ar1 = fabsf(r[e + 1]);
+            const float t0 = fmaf(-rel, ar0, fabsf(d0)), t1 = fmaf(-rel, ar1, fabsf(d1));
+            // t <= 0: fine as before.  A normal t > 0 with t - g*|r| <= 0: the quotient still rounds
+            // to at most rel.  A tiny positive t, NaN or Inf stay positive or NaN: the exact path.
+            const float v0 = t0 >= 7.888609052e-31f ? fmaf(-g, ar0, t0) : t0;
+            const float v1 = t1 >= 7.888609052e-31f ? fmaf(-g, ar1, t1) : t1;
+            mabs = max3(mabs, fabsf(d0), fabsf(d1));
+            mrel = max3_nan(mrel, v0, v1);
+          }
         }
         // A thread whose (c) fails, or (no lean bound) whose largest error exceeds atol, looks
         // again element by element below before its warp is sent down the exact path.
@@ -537,13 +575,11 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
           // significand class, if the maximum comes from one-ulp differences) stop here instead
           // of taking the exact path each time.  Such an element is within tolerance as well:
           // ad < (rel + ulp(rel)/2)*|r| < rtol*(1 - 2^-21)*|r| <= RN(rtol*|r|) <= tol.
-          const unsigned int rb = __float_as_uint(rel);
-          const float g = rb >= (30u << 23)
-                              ? __uint_as_float((rb & 0x7F800000u) - (24u << 23)) * 0.99999904632568359375f
-                              : 0.0f;
+          const float g = half_ulp_of_rel();
           // (A failure that is large against the thread's errors is a real new maximum: no
-          // need to look.  An element of the kind above fails by 2^-24 of its error at most.)
-          bool again = !(mrel <= mabs * 9.5367431640625e-07f);
+          // need to look.  An element of the kind above fails by 2^-24 of its error at most.
+          // In the sharp instantiation the look has been taken already.)
+          bool again = sharp || !(mrel <= mabs * 9.5367431640625e-07f);
           if (!again) {
 #pragma unroll
           for (int e = 0; e < kEPT; e += 2) {
@@ -581,6 +617,10 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
         if (!__any_sync(0xFFFFFFFFu, trig)) {
           const unsigned int tot = warp_add_u32(mis_fast);
           if (lane == 0 && tot) atomicAdd(&s.cnt[kk], (unsigned long long)tot);
+          // (some lane was `bad`, or the step would have ended above: while lean that lane took
+          // a second look, and it found nothing)
+          // (32-bit add on the low word of the 64-bit slot; flush() moves it to the accumulator)
+          if (!SHARP && lane == 0 && lean) atomicAdd(reinterpret_cast<unsigned int*>(&s.cnt[3 * kMaxKC + kk]), 1u);
           continue;
         }
 
@@ -770,6 +810,15 @@ struct LeadParams {
   float atol, rtol;
   MaskDev mask;
   const unsigned int* count;
+  // Fruitless second looks of earlier plain streaming launches, on their way to the host: the
+  // spare words of the accumulators cleared here (the previous call's) are added to looks_sum;
+  // looks_pub, which the previous lead kernel filled the same way (the call before that), is
+  // published as 64 * looks / pub_steps (capped at 64) in host-visible memory (if that call had a
+  // plain streaming launch: pub_steps > 0) and reset.
+  unsigned long long* looks_sum;
+  unsigned long long* looks_pub;
+  unsigned int* hint;
+  float pub_steps;
 };
 template <int DT>
 __global__ void __launch_bounds__(256) screen_lead_kernel(const LeadParams p, const __grid_constant__ PtrChunk chunk_ptrs) {
@@ -778,8 +827,20 @@ __global__ void __launch_bounds__(256) screen_lead_kernel(const LeadParams p, co
   const unsigned int k = blockIdx.y;
   if (blockIdx.x == 0) {
     if (threadIdx.x == 0 && p.from_args) p.table[k] = chunk_ptrs.p[k];
-    for (unsigned int j = k + gridDim.y * threadIdx.x; j < p.n_clear; j += gridDim.y * 256u) clear_acc(&p.acc_next[j]);
+    unsigned long long looks = 0ull;
+    for (unsigned int j = k + gridDim.y * threadIdx.x; j < p.n_clear; j += gridDim.y * 256u) {
+      looks += p.acc_next[j].spare;
+      clear_acc(&p.acc_next[j]);
+    }
+    if (looks && p.looks_sum) atomicAdd(p.looks_sum, looks);
     if (k == 0 && threadIdx.x < 3) p.counters_next[threadIdx.x] = 0u;
+    if (k == 0 && threadIdx.x == 32 && p.hint) {
+      // (only plain launches report: the word keeps the last report until the host takes it)
+      if (p.pub_steps > 0.0f)
+        *reinterpret_cast<volatile unsigned int*>(p.hint) =
+            (unsigned int)fminf(64.0f * (float)*p.looks_pub / p.pub_steps, 64.0f);
+      *p.looks_pub = 0ull;
+    }
   }
   if (p.count && k >= *p.count) return;
   __shared__ unsigned int s_cnt[3];

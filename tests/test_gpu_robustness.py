@@ -336,3 +336,47 @@ def test_general_path_takes_two_launches_and_leaves_its_scratch_clean(ctx, kb):
     run(9 * 4096, 190, synth.F32, 2)
     assert ctx.poll() == 0
     assert ctx.check_guards()[1] == 0
+
+
+def test_sharp_filter_is_chosen_for_dense_rounded_down_quotients_and_changes_nothing(ctx, kb):
+    """One-ulp differences on many elements, none of them a power of two: the largest quotient
+    (1/129 in bf16) is inexact and rounded down, and every element of its significand class
+    fails the plain filter without being a new maximum.  After a few calls the context switches
+    to the streaming kernel's sharp instantiation; the records are the oracle's either way, and
+    sparse differences never make it switch."""
+    dev = torch.device("cuda", 0)
+    ctx.set_small_path(False)
+    g = torch.Generator(device=dev)
+    g.manual_seed(3)
+    N = 200 * 4096 + 77
+    ref = (torch.randn(N, device=dev, generator=g) * 4).to(torch.bfloat16)
+    bits = ref.view(torch.int16)
+
+    def flipped(frac, K):
+        out = []
+        for _ in range(K):
+            f = (torch.rand(N, device=dev, generator=g) < frac) & ((bits & 0x7F) != 0)
+            out.append(torch.where(f, (bits + 1).view(torch.bfloat16), ref))
+        return out
+
+    dense = flipped(0.5, 10)
+    sparse = flipped(0.001, 10)
+    want_dense = oracle_records(synth.BF16, ref, dense, 1e-2, 1.6e-2)
+    want_sparse = oracle_records(synth.BF16, ref, sparse, 1e-2, 1.6e-2)
+    assert (want_dense["pass"] == 1).all() and (fbits(want_dense["max_rel_err"]) == fbits(np.float32(1.0) / np.float32(129.0))).all()
+    for mode in (1, 2):                               # forced plain, forced sharp
+        ctx.set_filter(mode)
+        same_records(kb.records(ctx.screen(ref, dense, 1e-2, 1.6e-2)), want_dense)
+        assert ctx.last_filter_sharp == (mode == 2)
+        same_records(kb.records(ctx.screen(ref, sparse, 1e-2, 1.6e-2)), want_sparse)
+    ctx.set_filter(0)                                 # automatic
+    seen = []
+    for _ in range(8):
+        same_records(kb.records(ctx.screen(ref, dense, 1e-2, 1.6e-2)), want_dense)    # (synchronises)
+        seen.append(ctx.last_filter_sharp)
+    assert not seen[0] and seen[-1], seen             # plain first, sharp once the reports are in
+    ctx.set_filter(0)                                 # forget
+    for _ in range(8):
+        same_records(kb.records(ctx.screen(ref, sparse, 1e-2, 1.6e-2)), want_sparse)
+        assert not ctx.last_filter_sharp
+    assert ctx.poll() == 0
