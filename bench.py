@@ -234,16 +234,18 @@ def run_screen(args):
     if not args.default_dispatch:
         ctx.set_small_path(False)      # time the streaming path whatever the size
     K, N = args.K, 1 << args.log2n
-    tdt = {"f64": torch.float64, "f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16}[args.dtype]
-    idt = {8: torch.int64, 4: torch.int32, 2: torch.int16}[torch.empty(0, dtype=tdt).element_size()]
+    tdt = {"f64": torch.float64, "f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16,
+           "e4m3": torch.float8_e4m3fn, "e5m2": torch.float8_e5m2}[args.dtype]
+    idt = {8: torch.int64, 4: torch.int32, 2: torch.int16, 1: torch.int8}[torch.empty(0, dtype=tdt).element_size()]
     g = torch.Generator(device=dev)
     g.manual_seed(20260802)
     ref = torch.randn(N, dtype=torch.float32, device=dev, generator=g).to(tdt)
+    esz1 = ref.element_size() == 1           # 8-bit floats: one unit in the last place is up to 1/8
     cands = []
     for _ in range(K):
         flip = torch.rand(N, device=dev, generator=g) < args.flip_frac
-        cands.append(torch.where(flip, (ref.view(idt) + 1).view(tdt), ref))
-    atol, rtol = (1e-12, 1e-12) if args.dtype == "f64" else (1e-2, 1.6e-2)
+        cands.append(torch.where(flip, ref.view(idt) + 1, ref.view(idt)).view(tdt))
+    atol, rtol = (1e-12, 1e-12) if args.dtype == "f64" else (1e-2, 0.13) if esz1 else (1e-2, 1.6e-2)
     call = (lambda: ctx.screen_f64(ref, cands, atol, rtol)) if args.dtype == "f64" else \
         (lambda: ctx.screen(ref, cands, atol, rtol))
     steps, warmup = max(1, min(args.steps, 50)), max(3, args.warmup)
@@ -378,7 +380,7 @@ def main():
                     help="'adjudicate' times kb_adjudicate alone on timings[K][S] (config 5 tier 1 by "
                          "default) and reports pairwise comparisons/s against the ALU roofline; it is a "
                          "secondary measurement, not the benchmark line")
-    ap.add_argument("--dtype", default="bf16", choices=["bf16", "f16", "f32", "f64"],
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "f16", "f32", "f64", "e4m3", "e5m2"],
                     help="storage type of the 'screen' workload")
     ap.add_argument("--log2n", type=int, default=24, help="elements per tensor of the 'screen' workload")
     ap.add_argument("--flip-frac", type=float, default=0.25)
