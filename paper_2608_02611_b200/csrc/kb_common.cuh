@@ -117,6 +117,17 @@ template <bool E5M2> struct ElemF8 {
       asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"(pr));
     return h2;
   }
+  // four bytes -> two f16x2 words (bytes 0,1 and bytes 2,3), without shifting the halves out first
+  __device__ __forceinline__ static void widen4(unsigned int w, unsigned int& lo2, unsigned int& hi2) {
+    if (E5M2)
+      asm("{\n.reg .b16 lo, hi;\nmov.b32 {lo, hi}, %2;\ncvt.rn.f16x2.e5m2x2 %0, lo;\ncvt.rn.f16x2.e5m2x2 %1, hi;\n}"
+          : "=r"(lo2), "=r"(hi2)
+          : "r"(w));
+    else
+      asm("{\n.reg .b16 lo, hi;\nmov.b32 {lo, hi}, %2;\ncvt.rn.f16x2.e4m3x2 %0, lo;\ncvt.rn.f16x2.e4m3x2 %1, hi;\n}"
+          : "=r"(lo2), "=r"(hi2)
+          : "r"(w));
+  }
   __device__ __forceinline__ static void decode(const uint4& w, float* out) {
     const unsigned int* u = reinterpret_cast<const unsigned int*>(&w);
 #pragma unroll

@@ -12,6 +12,7 @@
 #include "kb_adjudicate.cuh"
 #include "kb_common.cuh"
 #include "kb_screen.cuh"
+#include "kb_screen8.cuh"
 #include "kb_screen64.cuh"
 #include "kb_select.cuh"
 
@@ -230,20 +231,26 @@ kb_status ensure_ws(kb_ctx* ctx, uint32_t K) {
 inline uint32_t stream_stages(uint32_t tile_bytes) { return tile_bytes >= 16384 ? 3 : tile_bytes >= 8192 ? 7 : 10; }
 
 constexpr int kSharpCalls = 32, kSharpGrace = 4;
+#ifndef KB8_STAGES
+#define KB8_STAGES 7
+#endif
+// e4m3 kernel: stages of 4 KB, CTAs of 160 threads, four resident per SM at 96 registers
+constexpr uint32_t kStages8 = KB8_STAGES, kCtas8 = 4;
 template <int DT>
 kb_status launch_stream(kb_ctx* ctx, StreamParams& sp, cudaStream_t st) {
   const uint32_t tile_bytes = kTile * Elem<DT>::kBytes;
-  sp.stages = stream_stages(tile_bytes);
-  const size_t smem = stream_smem_bytes(sp.stages, tile_bytes);
+  constexpr bool k8 = DT == KB_F8E4M3;           // e4m3 has a kernel of its own (kb_screen8.cuh)
+  sp.stages = k8 ? kStages8 : stream_stages(tile_bytes);
+  const size_t smem = k8 ? stream8_smem_bytes(sp.stages) : stream_smem_bytes(sp.stages, tile_bytes);
   const unsigned long long nitems = (unsigned long long)sp.nchunks * sp.ntiles;
-  unsigned long long grid = ctx->forced_grid ? ctx->forced_grid : 3ull * ctx->sm_count;
+  unsigned long long grid = ctx->forced_grid ? ctx->forced_grid : (k8 ? (unsigned long long)kCtas8 : 3ull) * ctx->sm_count;
   if (grid > nitems) grid = nitems;
   // which instantiation: what the last finished plain call on this context reported
   // Plain until a plain launch reports that a quarter of its warp steps took a fruitless
   // second look; then sharp for kSharpCalls launches, one plain launch as a probe, sharp again
   // for the kSharpGrace launches its report needs to arrive, and the report decides.
-  bool sharp = ctx->filter_mode == 2;
-  if (ctx->filter_mode == 0 && ctx->h_hint) {
+  bool sharp = ctx->filter_mode == 2 && !k8;
+  if (ctx->filter_mode == 0 && ctx->h_hint && !k8) {
     volatile unsigned int* hint = reinterpret_cast<volatile unsigned int*>(ctx->h_hint);
     if (ctx->sharp_left > 0) {
       sharp = true;
@@ -266,13 +273,17 @@ kb_status launch_stream(kb_ctx* ctx, StreamParams& sp, cudaStream_t st) {
   }
   ctx->last_sharp = sharp;
   // warp steps of this launch if it counts its fruitless second looks (see LeadParams)
-  ctx->call_steps = sharp ? 0.0f : (float)sp.ntiles * (float)sp.K * (float)kWarps;
+  ctx->call_steps = (sharp || k8) ? 0.0f : (float)sp.ntiles * (float)sp.K * (float)kWarps;
   {
     ScopedTimer tm(ctx, KB_TIMER_SCREEN_STREAM, st);
-    if (sharp)
-      screen_stream_kernel<DT, true><<<(unsigned int)grid, kStreamThreads, smem, st>>>(sp);
-    else
-      screen_stream_kernel<DT, false><<<(unsigned int)grid, kStreamThreads, smem, st>>>(sp);
+    if constexpr (k8) {
+      screen_stream8_kernel<DT><<<(unsigned int)grid, kThreads8, smem, st>>>(sp);
+    } else {
+      if (sharp)
+        screen_stream_kernel<DT, true><<<(unsigned int)grid, kStreamThreads, smem, st>>>(sp);
+      else
+        screen_stream_kernel<DT, false><<<(unsigned int)grid, kStreamThreads, smem, st>>>(sp);
+    }
   }
   ++ctx->launches;
   KB_CUDA(ctx, cudaGetLastError());
@@ -297,18 +308,25 @@ kb_status launch_generic(kb_ctx* ctx, const void* ref, const void* const* tab, A
 
 template <int DT>
 kb_status set_stream_attr(kb_ctx* ctx) {
-  const uint32_t tile_bytes = kTile * Elem<DT>::kBytes;
-  const size_t smem = stream_smem_bytes(stream_stages(tile_bytes), tile_bytes);
-  KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT, false>,
-                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT, false>,
-                                    cudaFuncAttributePreferredSharedMemoryCarveout,
-                                    (int)cudaSharedmemCarveoutMaxShared));
-  KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT, true>,
-                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT, true>,
-                                    cudaFuncAttributePreferredSharedMemoryCarveout,
-                                    (int)cudaSharedmemCarveoutMaxShared));
+  if constexpr (DT == KB_F8E4M3) {
+    KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream8_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)stream8_smem_bytes(kStages8)));
+    KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream8_kernel<DT>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                      (int)cudaSharedmemCarveoutMaxShared));
+  } else {
+    const uint32_t tile_bytes = kTile * Elem<DT>::kBytes;
+    const size_t smem = stream_smem_bytes(stream_stages(tile_bytes), tile_bytes);
+    KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT, false>,
+                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT, false>,
+                                      cudaFuncAttributePreferredSharedMemoryCarveout,
+                                      (int)cudaSharedmemCarveoutMaxShared));
+    KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT, true>,
+                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT, true>,
+                                      cudaFuncAttributePreferredSharedMemoryCarveout,
+                                      (int)cudaSharedmemCarveoutMaxShared));
+  }
   return KB_OK;
 }
 
@@ -932,7 +950,8 @@ kb_status screen_impl(kb_ctx* ctx, const void* d_ref, const void* const* h_cands
       // chunk the candidates: shared-memory accumulators hold kMaxKC of them, and
       // small tensors need more, smaller items to fill the machine
       uint32_t nchunks = (K + kMaxKC - 1) / kMaxKC;
-      const uint64_t grid = ctx->forced_grid ? ctx->forced_grid : 3ull * ctx->sm_count;
+      const uint64_t grid =
+          ctx->forced_grid ? ctx->forced_grid : (DT == KB_F8E4M3 ? (unsigned long long)kCtas8 : 3ull) * ctx->sm_count;
       const uint64_t want_items = 8 * grid;
       if ((uint64_t)nchunks * sp.ntiles < want_items) {
         uint64_t nc = (want_items + sp.ntiles - 1) / sp.ntiles;

@@ -789,3 +789,62 @@ def test_alu_probe_reports_a_rate(ctx, kb):
     rate = ctx.alu_probe(2000)
     assert 1e11 < rate < 1e14          # sample pairs per second; 148 SMs x 64 lanes x 2 GHz / 2 = 9.3e12
     assert ctx.poll() == 0
+
+
+@pytest.mark.parametrize("dtype_code", [synth.F8E4M3, synth.F8E5M2])
+def test_fp8_every_byte_pair_behind_established_maxima(ctx, kb, dtype_code):
+    """Every (reference byte, candidate byte) combination of an 8-bit format, each ALONE in the
+    512 bytes a warp of the e4m3 kernel looks at in one step (everything around it identical in
+    reference and candidate), scanned after a leading block has established a large absolute
+    error and a chosen relative error.  The e4m3 kernel declares a warp clean from its packed
+    half-precision pre-filter alone, so here that decision rests on one pair at a time: a pair
+    wrongly declared clean (a subtraction that rounds in binary16, a product that rounds to zero,
+    a tie with a running maximum, NaN patterns, zeros) loses a count or a maximum.  Candidates
+    keep different subsets of the pairs, so that they stay lean or not and establish different
+    maxima; tolerances lie on both sides of the pre-filter's bound of 1/2."""
+    dev = torch.device("cuda", 0)
+    tdt = synth.TORCH_DTYPE[dtype_code]
+    val = torch.arange(256, dtype=torch.uint8).view(tdt).float()               # value of every byte
+    rb = torch.arange(256, dtype=torch.int64).repeat_interleave(256)          # reference byte
+    cb = torch.arange(256, dtype=torch.int64).repeat(256)                     # candidate byte
+    one = {synth.F8E4M3: 0x38, synth.F8E5M2: 0x3C}[dtype_code]                # the byte of 1.0
+    lead = 8 * 4096                                                           # the scouted tiles
+    rng = np.random.default_rng(8 + dtype_code)
+    perm = torch.from_numpy(rng.permutation(65536))
+    rb, cb = rb[perm], cb[perm]
+    # pair p sits in tile p // 4, in the first 512-byte region of warp p % 4, at a varying offset
+    pos = lead + (torch.arange(65536) // 4) * 4096 + (torch.arange(65536) % 4) * 512 + \
+        (torch.arange(65536) * 37) % 512
+    N = lead + 16384 * 4096
+    fill = torch.from_numpy(rng.integers(0, 0x78, N)).to(torch.int64)          # finite positive fillers
+    fill[:lead] = one
+    ref_bytes = fill.clone()
+    ref_bytes[pos] = rb
+    d = (val[cb] - val[rb]).abs()
+    ratio = d / val[rb].abs()
+    keep_sets = [torch.ones(65536, dtype=torch.bool), ratio <= 0.3, ratio <= 0.14, d <= 1.0,
+                 (rb - cb).abs() <= 1, (ratio <= 0.126) & (d <= 0.5), (d <= 2.0) & (ratio <= 0.5)]
+    two = one + 8 if dtype_code == synth.F8E4M3 else one + 4                   # the byte of 2.0
+    leads = [(0x7E, one + 1), (0x50, one + 2), (one + 1, one + 1), (0x7E, one), (0x60, one + 4), (0x30, one + 1),
+             (two, one + 1)]                                                   # (established error 1.0: pairs above it follow)
+    to_t = lambda b: b.to(torch.uint8).to(dev).view(tdt)
+    ref = to_t(ref_bytes)
+    cts = []
+    for keep, (big, small) in zip(keep_sets, leads):
+        c = ref_bytes.clone()
+        c[pos[keep]] = cb[keep]
+        c[5] = big            # a large absolute error at a low index
+        c[9000] = small       # a relative error of a few units in the last place
+        cts.append(to_t(c))
+    for atol, rtol in ((1e-2, 0.13), (0.0, 0.26), (1e-3, 0.5), (1e-2, 0.75), (0.0, 0.0), (1.0, 0.04)):
+        want = oracle_screen(dtype_code, ref, cts, atol, rtol)
+        for grid in (0, 5):
+            ctx.set_grid(grid)
+            try:
+                ctx.set_small_path(False)
+                got = kb.records(ctx.screen(ref, cts, atol, rtol))
+            finally:
+                ctx.set_small_path(True)
+                ctx.set_grid(0)
+            assert ctx.poll() == 0
+            assert_records_equal(got, want, f"fp8 {dtype_code} atol={atol} rtol={rtol} grid={grid}")
