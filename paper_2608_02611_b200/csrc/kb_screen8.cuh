@@ -1,4 +1,4 @@
-// The correctness gate's streaming kernel for the two 8-bit float formats (Sec. 3.1 K(p);
+// The correctness gate's streaming kernel for 8-bit floats, used for e4m3 (Sec. 3.1 K(p);
 // Sec. 3.4 Verifier).  Same plan as screen_stream_kernel -- work items drawn from a global
 // counter, one producer lane feeding a ring of shared-memory stages with 1-D bulk copies,
 // thresholds exchanged between CTAs, integer merges, the last CTA unpacks -- with what a
@@ -15,11 +15,12 @@
 //    rounded DOWN to binary16.  A thread is certainly clean if a <= th16 and t <= 0 for all
 //    its elements and nothing is NaN:
 //      - where the subtraction is exact in binary16 (always, unless the two exponents differ
-//        by 8 or more), a = |c - r| exactly, the fused multiply-add rounds once and keeps its
+//        by 7 or more: the difference of two 4-bit significands g binades apart has at most
+//        g + 5 bits), a = |c - r| exactly, the fused multiply-add rounds once and keeps its
 //        sign, and rel16 <= rel, th16 <= th give |c - r| <= th and |c - r| - rel*|r| <= 0: the
 //        binary32 filter's conditions (b) and (c);
-//      - where it is not exact, one magnitude is at least 256 times the other, so
-//        |c - r| >= (255/256) * max(|c|, |r|) and t >= |r| * (255/256 - 1/2048 - rel16) > 0
+//      - where it is not exact, one magnitude is more than 64 times the other, so
+//        |c - r| >= (63/64) * max(|c|, |r|) and t >= |r| * (63/64 - 1/1024 - rel16) > 0
 //        (or, for |c| >> |r|, far above rel16*|r|) as long as rel16 <= 1/2: condition (c)
 //        fails and the thread is not declared clean.  The pre-filter is therefore used only
 //        with a lean bound of at most 1/2 (rtol <= 1/2); beyond the bound rel is clamped to it,
@@ -32,10 +33,12 @@
 //        pre-filter is skipped for 0 < rel < 2^-5 (8-bit formats cannot produce so small a
 //        largest relative error from a real difference).  e5m2 goes down to 2^-16 with two
 //        fraction bits: products with its tiny values would need a guard that flags most warps
-//        on data that has any, so e5m2 runs without the pre-filter (it keeps the 32 elements
-//        per thread).
+//        on data that has any, so e5m2 stays with screen_stream_kernel.
 //    A warp none of whose threads is flagged has finished the step; otherwise the whole warp
 //    runs the binary32 step of screen_stream_kernel on its two 16-element groups.
+//  * The thresholds a warp reads decide which vote it takes next (pre-filter or binary32
+//    step), so lane 0's copy is broadcast to the warp, and a wait that gives up does so for the
+//    whole warp.
 //  * No sharp instantiation and no count of fruitless second looks.
 #pragma once
 
