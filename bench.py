@@ -378,6 +378,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="skip the secondary CUDA-graph replay of the step")
     ap.add_argument("--workload", default="step", choices=["step", "adjudicate", "screen", "paper-scale"],
                     help="'adjudicate' times kb_adjudicate alone on timings[K][S] (config 5 tier 1 by "
                          "default) and reports pairwise comparisons/s against the ALU roofline; it is a "
@@ -505,6 +506,50 @@ def main():
     ms_per_step = elapsed_ms / steps
     value = world * K_CANDS * N / (ms_per_step * 1e-3)
 
+    # ---- secondary: the same step captured once into a CUDA graph and replayed (what a caller who
+    # captures the three calls gets: no per-kernel event pairs, launch gaps of a graph).  Not the
+    # benchmark value. ----
+    graph_replay = None
+    if not args.no_graph:
+        try:
+            cap = torch.cuda.Stream(dev)
+            cap2 = torch.cuda.Stream(dev)
+            g_out = torch.empty_like(out)
+
+            def graph_step():
+                cur = torch.cuda.current_stream(dev)
+                cap2.wait_stream(cur)
+                with torch.cuda.stream(cap2):
+                    med, iqr, wins = ctx_adj.adjudicate(d_timings)
+                ctx.screen(case.ref, cands, case.atol, case.rtol, out=g_out)
+                cur.wait_stream(cap2)
+                return ctx.select(g_out, med, binding.KB_SELECT_ERR_THEN_TIME, BUDGET)
+
+            cap.wait_stream(main)
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(cap):
+                with torch.cuda.graph(graph, stream=cap):
+                    g_surv, g_n = graph_step()
+            torch.cuda.synchronize()
+            for _ in range(3):
+                graph.replay()
+            torch.cuda.synchronize()
+            g_steps = min(steps, 200)
+            e0g, e1g = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0g.record()
+            for _ in range(g_steps):
+                graph.replay()
+            e1g.record()
+            torch.cuda.synchronize()
+            g_ms = e0g.elapsed_time(e1g) / g_steps
+            same = bool((g_out == out).all()) and g_surv.tolist() == surv.tolist() and int(g_n) == int(n)
+            graph_replay = {"ms_per_step": g_ms, "value": world * K_CANDS * N / (g_ms * 1e-3), "steps": g_steps,
+                            "same_results_as_direct_calls": same}
+            del graph
+        except Exception as exc:   # a secondary figure must not take the benchmark line down
+            graph_replay = {"error": str(exc)[:200]}
+        torch.cuda.synchronize()
+
     # ---- end to end through the C ABI with HOST buffers (pinned), copies inside the timing ----
     e2e_steps = max(1, min(steps, 5))
     if args.no_e2e:
@@ -598,6 +643,7 @@ def main():
         "pairwise_comparisons_per_s": K_CANDS * K_CANDS * S2 / (avg_wins_ms * 1e-3),
         "wins_kernel_ms_avg": avg_wins_ms,
         "n_survivors": int(n.item()),
+        "graph_replay": graph_replay,
     }
     print(json.dumps(line), flush=True)
     if world > 1:
