@@ -146,6 +146,48 @@ class Mask:
             pass
 
 
+class Candidates:
+    """K candidate tensors checked once, with their device pointers already laid out as the
+    ``const void* const*`` array the screening calls take.  Building the array costs about
+    0.4 us per tensor in Python, which at K = 1024 is longer than the kernels run; a caller
+    that screens the same tensors again (another tolerance, another tier's mask) passes this
+    object instead of the list.  Holds references to the tensors so the pointers stay valid."""
+
+    def __init__(self, tensors: Sequence[torch.Tensor]):
+        self.tensors = list(tensors)
+        K = len(self.tensors)
+        first = self.tensors[0] if K else None
+        self.dtype = first.dtype if K else None
+        self.numel = first.numel() if K else 0
+        self.device = first.device if K else None
+        for c in self.tensors:
+            if (c.dtype != self.dtype or c.numel() != self.numel or not c.is_cuda
+                    or not c.is_contiguous() or c.device != self.device):
+                raise KbError(1, "Candidates", "candidates must be contiguous CUDA tensors of one "
+                                               "dtype, element count and device")
+        self.ptrs = (ctypes.c_void_p * max(K, 1))(*[c.data_ptr() for c in self.tensors])
+
+    def __len__(self) -> int:
+        return len(self.tensors)
+
+
+def _marshal_cands(cands, ref: torch.Tensor, where: str):
+    """(K, pointer array) of a list of tensors or of a Candidates object, checked against ref."""
+    if isinstance(cands, Candidates):
+        if len(cands) and (cands.dtype != ref.dtype or cands.numel != ref.numel()
+                           or cands.device != ref.device):
+            raise KbError(1, where, "candidates must have the reference's dtype, element count "
+                                    "and device")
+        return len(cands), cands.ptrs
+    N = ref.numel()
+    for c in cands:
+        if c.dtype != ref.dtype or c.numel() != N or not c.is_cuda or not c.is_contiguous():
+            raise KbError(1, where, "candidates must be contiguous CUDA tensors with the "
+                                    "reference's dtype and element count")
+    K = len(cands)
+    return K, (ctypes.c_void_p * max(K, 1))(*[c.data_ptr() for c in cands])
+
+
 class Context:
     """kb_ctx bound to one CUDA device."""
 
@@ -264,20 +306,16 @@ class Context:
     # -- the three calls ----------------------------------------------------
     def screen(self, ref: torch.Tensor, cands: Sequence[torch.Tensor], atol: float, rtol: float,
                mask: Optional[Mask] = None, out: Optional[torch.Tensor] = None) -> torch.Tensor:
-        """kb_screen.  Returns a uint8 CUDA tensor [K, 48] of kb_screen_result records
-        (see ``records``); asynchronous on the current stream."""
-        K = len(cands)
+        """kb_screen.  ``cands`` is a sequence of tensors or a ``Candidates`` object.  Returns a
+        uint8 CUDA tensor [K, 48] of kb_screen_result records (see ``records``); asynchronous on
+        the current stream."""
         N = ref.numel()
         code = DTYPE_CODE.get(ref.dtype, -1)
-        for c in cands:
-            if c.dtype != ref.dtype or c.numel() != N or not c.is_cuda or not c.is_contiguous():
-                raise KbError(1, "kb_screen", "candidates must be contiguous CUDA tensors with the "
-                                              "reference's dtype and element count")
         if not ref.is_cuda or not ref.is_contiguous():
             raise KbError(1, "kb_screen", "reference must be a contiguous CUDA tensor")
+        K, ptrs = _marshal_cands(cands, ref, "kb_screen")
         if out is None:
             out = torch.empty((K, RESULT_BYTES), dtype=torch.uint8, device=ref.device)
-        ptrs = (ctypes.c_void_p * max(K, 1))(*[c.data_ptr() for c in cands])
         rc = load().kb_screen(self._h, ref.data_ptr(), ptrs, K, N, code, float(atol), float(rtol),
                               mask._h if mask is not None else None, out.data_ptr(),
                               _stream_ptr(ref.device))

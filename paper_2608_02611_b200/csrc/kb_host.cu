@@ -912,8 +912,12 @@ kb_status screen_impl(kb_ctx* ctx, const void* d_ref, const void* const* h_cands
       if (nscout > 8) nscout = 8;
     }
     const uint64_t tail0 = nfull * kTile;
-    const unsigned int tail_blocks = (unsigned int)((N - tail0 + kScoutPerBlock - 1) / kScoutPerBlock);
-    const unsigned int lead_blocks = nscout * (kTile / kScoutPerBlock) + tail_blocks;
+    // small blocks spread a few candidates over the machine; with many candidates they would
+    // only queue up, so each block then takes a whole kernel tile
+    unsigned int per_block = kScoutPerBlock;
+    if ((uint64_t)K * (nscout * (kTile / kScoutPerBlock) + 1u) > 32ull * ctx->sm_count) per_block = kTile;
+    const unsigned int tail_blocks = (unsigned int)((N - tail0 + per_block - 1) / per_block);
+    const unsigned int lead_blocks = nscout * (kTile / per_block) + tail_blocks;
     {
       LeadParams lp;
       lp.ref = d_ref;
@@ -939,6 +943,7 @@ kb_status screen_impl(kb_ctx* ctx, const void* d_ref, const void* const* h_cands
       lp.looks_pub = sums + (set ^ 1);
       lp.hint = ctx->d_hint;
       lp.pub_steps = ctx->steps_hist[set];
+      lp.per_block = per_block;
       screen_lead_kernel<DT><<<dim3(lead_blocks ? lead_blocks : 1u, K), 256, 0, st>>>(lp, chunk);
       ++ctx->launches;
       KB_CUDA(ctx, cudaGetLastError());

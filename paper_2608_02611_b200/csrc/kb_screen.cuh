@@ -795,9 +795,30 @@ __global__ void __launch_bounds__(256) screen_generic_kernel(const void* __restr
 // the blocks with blockIdx.x == 0: candidate k's pointer goes from the kernel's arguments to
 // the device table the streaming kernel reads (when `from_args`), and the accumulators and
 // counters of the OTHER set -- the one the next call will work on -- are zeroed (nobody else
-// touches them during this call).  A block takes 1024 elements of one candidate and issues
-// one set of atomics.  grid = (max(1, nscout * 4 + ceil((N - tail0) / 1024)), K).
+// touches them during this call).  A block takes per_block elements of one candidate (1024,
+// or a whole kernel tile when there are many candidates) and issues one set of atomics.
+// grid = (max(1, nscout * (4096 / per_block) + ceil((N - tail0) / per_block)), K).
 constexpr unsigned int kScoutPerBlock = 1024;
+// four consecutive elements starting at element i (i a multiple of 4, p 16-byte aligned)
+template <int DT>
+__device__ __forceinline__ void load4(const void* p, unsigned long long i, float* out) {
+  using E = Elem<DT>;
+  uint4 w = make_uint4(0u, 0u, 0u, 0u);
+  const char* at = reinterpret_cast<const char*>(p) + i * E::kBytes;
+  if (E::kBytes == 4) {
+    w = *reinterpret_cast<const uint4*>(at);
+  } else if (E::kBytes == 2) {
+    const uint2 v = *reinterpret_cast<const uint2*>(at);
+    w.x = v.x;
+    w.y = v.y;
+  } else {
+    w.x = *reinterpret_cast<const unsigned int*>(at);
+  }
+  float o[E::kVec];
+  E::decode(w, o);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) out[j] = o[j];
+}
 struct LeadParams {
   const void* ref;
   const void** table;           // device pointer table [K]
@@ -819,11 +840,15 @@ struct LeadParams {
   unsigned long long* looks_pub;
   unsigned int* hint;
   float pub_steps;
+  unsigned int per_block;       // elements one block classifies: kScoutPerBlock or kTile
 };
 template <int DT>
 __global__ void __launch_bounds__(256) screen_lead_kernel(const LeadParams p, const __grid_constant__ PtrChunk chunk_ptrs) {
   using E = Elem<DT>;
-  constexpr unsigned int kBlocksPerTile = kTile / kScoutPerBlock;
+  // elements per block: kScoutPerBlock, or a whole kernel tile when the call has so many
+  // candidates that the smaller blocks would queue up in many waves
+  const unsigned int per_block = p.per_block;
+  const unsigned int kBlocksPerTile = kTile / per_block;
   const unsigned int k = blockIdx.y;
   if (blockIdx.x == 0) {
     if (threadIdx.x == 0 && p.from_args) p.table[k] = chunk_ptrs.p[k];
@@ -857,17 +882,43 @@ __global__ void __launch_bounds__(256) screen_lead_kernel(const LeadParams p, co
   if (blockIdx.x < p.nscout * kBlocksPerTile) {
     const unsigned int slot = blockIdx.x / kBlocksPerTile;
     const unsigned long long tile = p.tile_list ? p.tile_list[slot] : slot;
-    const unsigned long long base = tile * kTile + (blockIdx.x % kBlocksPerTile) * kScoutPerBlock;
+    const unsigned long long base = tile * kTile + (blockIdx.x % kBlocksPerTile) * per_block;
+    // four consecutive elements per thread and step (one vector load each from the reference
+    // and the candidate); the running maxima stay plain floats, and the quotient is only
+    // formed where it can exceed the thread's largest so far
+    float bad = -1.0f, qf = 0.0f;
+    unsigned int bi = 0u;
+    for (unsigned int j0 = 0; j0 < per_block / 1024; ++j0) {
+      const unsigned long long i0 = base + ((unsigned long long)j0 * 256 + threadIdx.x) * 4;
+      float rv[4], cv[4];
+      load4<DT>(p.ref, i0, rv);
+      load4<DT>(cand, i0, cv);
 #pragma unroll
-    for (unsigned int j = 0; j < kScoutPerBlock / 256; ++j) {
-      const unsigned long long i = base + j * 256 + threadIdx.x;
-      x.add(E::load(p.ref, i), E::load(cand, i), i, p.atol, p.rtol);
+      for (unsigned int j = 0; j < 4; ++j) {
+        const float r = rv[j], c = cv[j];
+        const float ad = fabsf(__fsub_rn(c, r));
+        const bool match = (c == r) || (ad <= tol_clamped(r, p.atol, p.rtol));
+        x.n_mis += match ? 0u : 1u;
+        x.n_nan += (c != c) ? 1u : 0u;
+        x.n_inf += (fabsf(c) == __uint_as_float(0x7F800000u)) ? 1u : 0u;
+        if (is_finite_nonneg(ad)) {
+          if (ad > bad) {          // indices rise within a thread: the first of equal maxima stays
+            bad = ad;
+            bi = (unsigned int)(i0 + j);
+          }
+          const float ar = fabsf(r);
+          // RD(qf * ar) >= ad  =>  ad / ar <= qf  =>  RN(ad / ar) <= qf: nothing to gain
+          if (ar > 0.0f && is_finite_nonneg(ar) && !(__fmul_rd(qf, ar) >= ad))
+            qf = fmaxf(qf, __fdiv_rn(ad, ar));
+        }
+      }
     }
+    if (bad >= 0.0f) x.best = pack_key(bad, bi);
+    x.qb = __float_as_uint(qf);
   } else {
     const unsigned long long base =
-        p.tail0 + (unsigned long long)(blockIdx.x - p.nscout * kBlocksPerTile) * kScoutPerBlock;
-#pragma unroll
-    for (unsigned int j = 0; j < kScoutPerBlock / 256; ++j) {
+        p.tail0 + (unsigned long long)(blockIdx.x - p.nscout * kBlocksPerTile) * per_block;
+    for (unsigned int j = 0; j < per_block / 256; ++j) {
       const unsigned long long i = base + j * 256 + threadIdx.x;
       if (i < p.N && mask_selected(p.mask, i)) x.add(E::load(p.ref, i), E::load(cand, i), i, p.atol, p.rtol);
     }

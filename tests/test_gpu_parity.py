@@ -290,6 +290,27 @@ def test_candidate_counts_around_chunk_size(ctx, kb, K):
     assert_records_equal(got, want, f"K={K}")
 
 
+def test_prepared_candidate_set_is_the_same_call(ctx, kb):
+    rng = np.random.default_rng(4242)
+    dev = torch.device("cuda", 0)
+    N = 5 * 4096 + 3
+    ref = awkward(N, synth.BF16, rng, dev)
+    cands = [perturbed(ref, synth.BF16, rng, dev) for _ in range(9)]
+    held = kb.Candidates(cands)
+    assert len(held) == 9
+    want = oracle_screen(synth.BF16, ref, cands, 1e-2, 1.6e-2)
+    for _ in range(3):                                          # the same object serves every call
+        got = kb.records(ctx.screen(ref, held, 1e-2, 1.6e-2))
+        assert_records_equal(got, want, "prepared candidate set")
+    m = ctx.mask_strided(N, 12, 2, 1)
+    assert torch.equal(ctx.screen(ref, held, 1e-2, 1.6e-2, m), ctx.screen(ref, cands, 1e-2, 1.6e-2, m))
+    m.close()
+    with pytest.raises(kb.KbError):                             # made for another element count
+        ctx.screen(ref[:4096].contiguous(), held, 1e-2, 1.6e-2)
+    with pytest.raises(kb.KbError):
+        kb.Candidates([cands[0], cands[1].float()])
+
+
 @pytest.mark.parametrize("grid", [1, 2, 5, 37, 0])
 def test_result_does_not_depend_on_grid(ctx, kb, grid):
     rng = np.random.default_rng(99)
