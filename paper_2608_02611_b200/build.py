@@ -18,7 +18,7 @@ DEPS = ["kb_host.cu", "kb_common.cuh", "kb_screen.cuh", "kb_screen8.cuh", "kb_sc
 
 NVCC_FLAGS = [
     "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
-    "-Xcompiler", "-fPIC", "-Xcompiler", "-Wno-format-truncation", "-shared",
+    "-Xcompiler", "-fPIC", "-Xcompiler", "-Wno-format-truncation", "-shared", "-ldl",
 ]
 
 

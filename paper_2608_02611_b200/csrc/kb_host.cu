@@ -9,6 +9,8 @@
 #include <new>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "kb_adjudicate.cuh"
 #include "kb_common.cuh"
 #include "kb_screen.cuh"
@@ -136,6 +138,15 @@ inline bool known_dtype(int dt) { return dt >= KB_F32 && dt <= KB_F8E5M2; }
 constexpr size_t kSmallTicketBytes = 4096;
 constexpr size_t kSmallMaxPartials = 8192;
 constexpr size_t kSmallWsBytes = kSmallTicketBytes + kSmallMaxPartials * sizeof(Acc);
+
+// A named range around an entry point's host work, for a timeline tool that is attached
+// (the header-only NVTX v3 calls do nothing otherwise).
+struct TraceRange {
+  explicit TraceRange(const char* name) { nvtxRangePushA(name); }
+  ~TraceRange() { nvtxRangePop(); }
+  TraceRange(const TraceRange&) = delete;
+  TraceRange& operator=(const TraceRange&) = delete;
+};
 
 // Event pair around one launch of an instrumented kernel (no-op unless timing is on).
 struct ScopedTimer {
@@ -996,6 +1007,7 @@ kb_status screen_dispatch(kb_ctx* ctx, const void* d_ref, const void* const* h_c
 extern "C" kb_status kb_screen(kb_ctx* ctx, const void* d_ref, const void* const* h_cands, uint32_t K,
                                uint64_t N, kb_dtype dtype, float atol, float rtol,
                                const kb_mask* mask, kb_screen_result* d_out, void* stream) {
+  TraceRange trace("kb_screen");
   kb_status rc = validate_screen(ctx, d_ref, h_cands, K, N, dtype, atol, rtol, mask, d_out, true);
   if (rc != KB_OK) return rc;
   DeviceGuard g(ctx->device);
@@ -1009,6 +1021,7 @@ extern "C" kb_status kb_screen(kb_ctx* ctx, const void* d_ref, const void* const
 extern "C" kb_status kb_screen_f64(kb_ctx* ctx, const double* d_ref, const double* const* h_cands,
                                    uint32_t K, uint64_t N, double atol, double rtol,
                                    const kb_mask* mask, kb_screen_result_f64* d_out, void* stream) {
+  TraceRange trace("kb_screen_f64");
   if (!ctx) return KB_ERR_INVALID_ARG;
   if (!d_ref || !h_cands || !d_out) return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen_f64: null pointer");
   if (K == 0 || K > KB_MAX_K) return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen_f64: K=%u outside [1, %u]", K, KB_MAX_K);
@@ -1126,6 +1139,7 @@ extern "C" kb_status kb_screen_indexed(kb_ctx* ctx, const void* d_ref, const voi
                                        const uint32_t* d_count, uint32_t Kmax, uint64_t N,
                                        kb_dtype dtype, float atol, float rtol, const kb_mask* mask,
                                        kb_screen_result* d_out, void* stream) {
+  TraceRange trace("kb_screen_indexed");
   if (!ctx) return KB_ERR_INVALID_ARG;
   if (!d_ref || !d_table || !d_index || !d_count || !d_out)
     return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen_indexed: null pointer");
@@ -1151,6 +1165,7 @@ extern "C" kb_status kb_screen_multi(kb_ctx* ctx, uint32_t G, const void* const*
                                      const void* const* h_cands, const uint32_t* h_K,
                                      const uint64_t* h_N, kb_dtype dtype, float atol, float rtol,
                                      kb_screen_result* d_out, void* stream) {
+  TraceRange trace("kb_screen_multi");
   if (!ctx) return KB_ERR_INVALID_ARG;
   if (!h_refs || !h_cands || !h_K || !h_N || !d_out)
     return fail(ctx, KB_ERR_INVALID_ARG, "kb_screen_multi: null pointer");
@@ -1265,6 +1280,7 @@ kb_status static_setup(int device, kb_ctx** out) {
 extern "C" kb_status kb_screen_static(const void* d_ref, const void* const* h_cands, uint32_t K,
                                       uint64_t N, kb_dtype dtype, float atol, float rtol,
                                       kb_screen_result* d_out, void* stream) {
+  TraceRange trace("kb_screen_static");
   int device = -1;
   if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= kStaticMaxDevices) {
     cudaGetLastError();
@@ -1308,6 +1324,7 @@ extern "C" kb_status kb_static_scratch_read(void* h_dst, uint32_t bytes) {
 extern "C" kb_status kb_screen_host(kb_ctx* ctx, const void* h_ref, const void* const* h_cands_host,
                                     uint32_t K, uint64_t N, kb_dtype dtype, float atol, float rtol,
                                     const kb_mask* mask, kb_screen_result* h_out, void* stream) {
+  TraceRange trace("kb_screen_host");
   kb_status rc = validate_screen(ctx, h_ref, h_cands_host, K, N, dtype, atol, rtol, mask, h_out, false);
   if (rc != KB_OK) return rc;
   DeviceGuard g(ctx->device);
@@ -1364,6 +1381,7 @@ extern "C" kb_status kb_screen_host(kb_ctx* ctx, const void* h_ref, const void* 
 
 extern "C" kb_status kb_adjudicate(kb_ctx* ctx, const float* d_timings, uint32_t K, uint32_t S,
                                    float* d_median, float* d_iqr, uint32_t* d_wins, void* stream) {
+  TraceRange trace("kb_adjudicate");
   if (!ctx) return KB_ERR_INVALID_ARG;
   if (!d_timings) return fail(ctx, KB_ERR_INVALID_ARG, "kb_adjudicate: timings is NULL");
   if (K == 0 || K > KB_MAX_K) return fail(ctx, KB_ERR_INVALID_ARG, "kb_adjudicate: K=%u outside [1, %u]", K, KB_MAX_K);
@@ -1492,6 +1510,7 @@ extern "C" kb_status kb_adjudicate(kb_ctx* ctx, const float* d_timings, uint32_t
 extern "C" kb_status kb_select(kb_ctx* ctx, const kb_screen_result* d_screen, const float* d_median,
                                uint32_t K, kb_select_policy policy, uint32_t budget,
                                int32_t* d_survivors, uint32_t* d_n_survivors, void* stream) {
+  TraceRange trace("kb_select");
   if (!ctx) return KB_ERR_INVALID_ARG;
   if (!d_screen || !d_median || !d_survivors || !d_n_survivors)
     return fail(ctx, KB_ERR_INVALID_ARG, "kb_select: null pointer");
@@ -1517,6 +1536,7 @@ extern "C" kb_status kb_select_by_score(kb_ctx* ctx, const kb_screen_result* d_s
                                         uint32_t rung_budget, float alpha, float beta,
                                         uint32_t budget, float* d_score, int32_t* d_survivors,
                                         uint32_t* d_n_survivors, void* stream) {
+  TraceRange trace("kb_select_by_score");
   if (!ctx) return KB_ERR_INVALID_ARG;
   if (!d_screen || !d_median || !d_survivors || !d_n_survivors)
     return fail(ctx, KB_ERR_INVALID_ARG, "kb_select_by_score: null pointer");
@@ -1539,6 +1559,7 @@ extern "C" kb_status kb_select_by_score(kb_ctx* ctx, const kb_screen_result* d_s
 
 extern "C" kb_status kb_tail_ratios(kb_ctx* ctx, const float* d_timings, uint32_t K, uint32_t S,
                                     float* d_ratios, void* stream) {
+  TraceRange trace("kb_tail_ratios");
   if (!ctx) return KB_ERR_INVALID_ARG;
   if (!d_timings || !d_ratios) return fail(ctx, KB_ERR_INVALID_ARG, "kb_tail_ratios: null pointer");
   if (K == 0 || K > KB_MAX_K) return fail(ctx, KB_ERR_INVALID_ARG, "kb_tail_ratios: K=%u outside [1, %u]", K, KB_MAX_K);
@@ -1555,6 +1576,7 @@ extern "C" kb_status kb_tail_ratios(kb_ctx* ctx, const float* d_timings, uint32_
 
 extern "C" kb_status kb_copeland(kb_ctx* ctx, const uint32_t* d_wins, uint32_t K, uint32_t S,
                                  uint32_t* d_beats, uint32_t* d_ties, void* stream) {
+  TraceRange trace("kb_copeland");
   if (!ctx) return KB_ERR_INVALID_ARG;
   if (!d_wins || !d_beats) return fail(ctx, KB_ERR_INVALID_ARG, "kb_copeland: null pointer");
   if (K == 0 || K > KB_MAX_K) return fail(ctx, KB_ERR_INVALID_ARG, "kb_copeland: K=%u outside [1, %u]", K, KB_MAX_K);
@@ -1570,6 +1592,7 @@ extern "C" kb_status kb_copeland(kb_ctx* ctx, const uint32_t* d_wins, uint32_t K
 extern "C" kb_status kb_confirm(kb_ctx* ctx, const float* d_first, const float* d_second,
                                 const float* d_prev, uint32_t K, float threshold,
                                 uint32_t* d_status, float* d_score, void* stream) {
+  TraceRange trace("kb_confirm");
   if (!ctx) return KB_ERR_INVALID_ARG;
   if (!d_first || !d_second || !d_prev || !d_status || !d_score)
     return fail(ctx, KB_ERR_INVALID_ARG, "kb_confirm: null pointer");
@@ -1587,6 +1610,7 @@ extern "C" kb_status kb_adjudicate_ragged(kb_ctx* ctx, const float* d_timings,
                                           const uint32_t* d_offsets, uint32_t K, uint32_t S_max,
                                           uint64_t total, float* d_median, float* d_iqr,
                                           uint32_t* d_wins, void* stream) {
+  TraceRange trace("kb_adjudicate_ragged");
   if (!ctx) return KB_ERR_INVALID_ARG;
   if (!d_timings || !d_offsets) return fail(ctx, KB_ERR_INVALID_ARG, "kb_adjudicate_ragged: null pointer");
   if (K == 0 || K > KB_MAX_K) return fail(ctx, KB_ERR_INVALID_ARG, "kb_adjudicate_ragged: K=%u outside [1, %u]", K, KB_MAX_K);
