@@ -13,7 +13,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libkb.so")
 SOURCES = ["kb_host.cu"]
-DEPS = ["kb_host.cu", "kb_common.cuh", "kb_screen.cuh", "kb_screen8.cuh", "kb_screen64.cuh", "kb_adjudicate.cuh", "kb_select.cuh",
+DEPS = ["kb_host.cu", "kb_common.cuh", "kb_screen.cuh", "kb_screen8.cuh", "kb_ring.cuh", "kb_screen64.cuh", "kb_adjudicate.cuh", "kb_select.cuh",
         os.path.join("..", "..", "include", "kb.h"), os.path.join("..", "..", "include", "kb_hooks.h")]
 
 NVCC_FLAGS = [

@@ -30,6 +30,7 @@
 #pragma once
 
 #include "kb_common.cuh"
+#include "kb_ring.cuh"
 
 namespace kb {
 
@@ -260,6 +261,8 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
 
   if (warp == kWarps) {
     // ------------------------------ producer ------------------------------
+    // (ring_producer of kb_ring.cuh with TileItemMap written in: this kernel's consumer loop is
+    // compiled measurably slower when the producer branch is the shared routine)
     const uint64_t pol_first = l2_policy_evict_first();
     const uint64_t pol_last = l2_policy_evict_last();
     uint32_t stage = 0, phase = 0;   // phase of the ring pass being filled

@@ -199,6 +199,23 @@ struct Stream64Params {
   kb_screen_result_f64* out;
 };
 
+// Items of the binary64 kernel: chunk-major over half tiles (a stage holds 2048 doubles, half a
+// kernel tile); the consumers read the item number itself.
+struct HalfTileItemMap {
+  uint32_t nhalf, half0, KC, K;
+  const uint32_t* tile_list;          // NULL: tile = slot / 2
+  __device__ __forceinline__ void locate(unsigned long long item, uint32_t& chunk, uint32_t& k0, int& kc,
+                                         size_t& off, unsigned long long& id) const {
+    chunk = (uint32_t)(item / nhalf);
+    const uint32_t slot = half0 + (uint32_t)(item % nhalf);
+    k0 = chunk * KC;
+    kc = (int)min(KC, K - k0);
+    const uint32_t tile = tile_list ? tile_list[slot >> 1] : (slot >> 1);
+    off = ((size_t)tile * kTile + (size_t)(slot & 1u) * kTile64) * 8;
+    id = item;
+  }
+};
+
 struct Stream64Smem {
   unsigned char* buf;
   uint64_t* full;
@@ -273,76 +290,12 @@ __global__ void __maxnreg__(160) screen_stream64_kernel(const Stream64Params p) 
   __syncthreads();
 
   const unsigned long long nitems = (unsigned long long)p.nchunks * p.nhalf;
-  constexpr unsigned long long kNoItem = ~0ull;
 
   if (warp == kWarps) {
     // ------------------------------ producer ------------------------------
-    const uint64_t pol_first = l2_policy_evict_first();
-    const uint64_t pol_last = l2_policy_evict_last();
-    uint32_t stage = 0, phase = 0;
-    unsigned long long issued = 0;
-    bool ok = true;
-    int cur_chunk = -1;
-    unsigned long long next_item = 0ull;
-    if (lane == 0) next_item = atomicAdd(p.sched, 1ull);
-    for (;;) {
-      const unsigned long long item = __shfl_sync(0xFFFFFFFFu, next_item, 0);
-      if (item >= nitems) break;
-      if (lane == 0) next_item = atomicAdd(p.sched, 1ull);
-      const uint32_t chunk = (uint32_t)(item / p.nhalf);
-      const uint32_t slot = p.half0 + (uint32_t)(item % p.nhalf);
-      const uint32_t k0 = chunk * p.KC;
-      const int kc = (int)min(p.KC, p.K - k0);
-      if ((int)chunk != cur_chunk) {
-        cur_chunk = (int)chunk;
-        __syncwarp();
-        for (int i = lane; i < kc; i += 32) s.ptrs[i] = p.cands[k0 + i];
-        __syncwarp();
-      }
-      if (lane == 0) {
-        const uint32_t tile = p.tile_list ? p.tile_list[slot >> 1] : (slot >> 1);
-        const size_t off = ((size_t)tile * kTile + (size_t)(slot & 1u) * kTile64) * 8;
-        for (int kk = -1; kk < kc; ++kk) {
-          if (!mbar_wait_bounded(&s.empty[stage], phase ^ 1u, s.abort_flag, p.status)) {
-            ok = false;
-            break;
-          }
-          if (kk < 0) s.item_id[stage] = item;
-          const unsigned char* src =
-              reinterpret_cast<const unsigned char*>(kk < 0 ? (const void*)p.ref : s.ptrs[kk]) + off;
-          mbar_arrive_expect_tx(&s.full[stage], kTileBytes64);
-          bulk_g2s(s.buf + (size_t)stage * kTileBytes64, src, kTileBytes64, &s.full[stage],
-                   (kk < 0 && p.nchunks > 1) ? pol_last : pol_first);
-          ++issued;
-          if (++stage == stages) {
-            stage = 0;
-            phase ^= 1u;
-          }
-        }
-      }
-      ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
-      if (!ok) break;
-    }
-    if (lane == 0 && ok) {
-      if (mbar_wait_bounded(&s.empty[stage], phase ^ 1u, s.abort_flag, p.status)) {
-        s.item_id[stage] = kNoItem;
-        mbar_arrive(&s.full[stage]);
-      } else {
-        ok = false;
-      }
-    }
-    if (lane == 0 && !ok) {
-      // Gave up: let every copy already issued land before the CTA may exit.
-      const unsigned long long back = issued < stages ? issued : stages;
-      for (unsigned long long m = issued - back; m < issued; ++m) {
-        uint64_t* bar = &s.full[m % stages];
-        const uint32_t par = (uint32_t)((m / stages) & 1ull);
-        const unsigned long long t0 = global_ns();
-        while (!mbar_try_wait(bar, par)) {
-          if (global_ns() - t0 > 1000000000ull) break;
-        }
-      }
-    }
+    const RingProducerView ring{s.buf, s.full, s.empty, s.item_id, s.ptrs, s.abort_flag};
+    const HalfTileItemMap map{p.nhalf, p.half0, p.KC, p.K, p.tile_list};
+    ring_producer(ring, map, lane, stages, kTileBytes64, nitems, p.sched, p.ref, p.cands, p.nchunks > 1, p.status);
   } else {
     // ------------------------------ consumers -----------------------------
     uint32_t stage = 0, phase = 0;

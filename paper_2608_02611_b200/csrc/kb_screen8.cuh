@@ -136,79 +136,12 @@ __global__ void __maxnreg__(96) screen_stream8_kernel(const StreamParams p) {
   const uint32_t K_eff = p.K_dev ? min(*p.K_dev, p.K) : p.K;
   const uint32_t nchunks_eff = (K_eff + p.KC - 1) / p.KC;
   const unsigned long long nitems = (unsigned long long)nchunks_eff * p.ntiles;
-  constexpr unsigned long long kNoItem = ~0ull;
 
   if (warp == kWarps) {
     // ------------------------------ producer ------------------------------
-    const uint64_t pol_first = l2_policy_evict_first();
-    const uint64_t pol_last = l2_policy_evict_last();
-    uint32_t stage = 0, phase = 0;   // phase of the ring pass being filled
-    unsigned long long issued = 0;
-    bool ok = true;
-    int cur_chunk = -1;
-    unsigned long long next_item = 0ull;
-    if (lane == 0) next_item = atomicAdd(p.sched, 1ull);
-    for (;;) {
-      const unsigned long long item = __shfl_sync(0xFFFFFFFFu, next_item, 0);
-      if (item >= nitems) break;
-      if (lane == 0) next_item = atomicAdd(p.sched, 1ull);   // drawn one item ahead: latency hidden
-      const uint32_t chunk = (uint32_t)(item / p.ntiles);
-      const uint32_t slot = p.slot0 + (uint32_t)(item % p.ntiles);
-      const uint32_t k0 = chunk * p.KC;
-      const int kc = (int)min(p.KC, K_eff - k0);
-      if ((int)chunk != cur_chunk) {
-        // the chunk's candidate pointers go to shared memory once (whole warp)
-        cur_chunk = (int)chunk;
-        __syncwarp();
-        for (int i = lane; i < kc; i += 32) s.ptrs[i] = p.cands[k0 + i];
-        __syncwarp();
-      }
-      if (lane == 0) {
-        const uint32_t tile = p.tile_list ? p.tile_list[slot] : slot;
-        const size_t off = (size_t)tile * TILE_BYTES;
-        for (int kk = -1; kk < kc; ++kk) {
-          if (!mbar_wait_bounded(&s.empty[stage], phase ^ 1u, s.abort_flag, p.status)) {
-            ok = false;
-            break;
-          }
-          // (chunk, position in the visit order), visible to the consumers with the phase
-          if (kk < 0) s.item_id[stage] = ((unsigned long long)chunk << 32) | (unsigned long long)(slot - p.slot0);
-          const unsigned char* src =
-              reinterpret_cast<const unsigned char*>(kk < 0 ? p.ref : s.ptrs[kk]) + off;
-          mbar_arrive_expect_tx(&s.full[stage], TILE_BYTES);
-          bulk_g2s(s.buf + (size_t)stage * TILE_BYTES, src, TILE_BYTES, &s.full[stage],
-                   (kk < 0 && p.nchunks > 1) ? pol_last : pol_first);
-          ++issued;
-          if (++stage == stages) {
-            stage = 0;
-            phase ^= 1u;
-          }
-        }
-      }
-      ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
-      if (!ok) break;
-    }
-    if (lane == 0 && ok) {
-      // no more work: an empty stage that carries the end marker
-      if (mbar_wait_bounded(&s.empty[stage], phase ^ 1u, s.abort_flag, p.status)) {
-        s.item_id[stage] = kNoItem;
-        mbar_arrive(&s.full[stage]);
-      } else {
-        ok = false;
-      }
-    }
-    if (lane == 0 && !ok) {
-      // Gave up: let every copy already issued land before the CTA may exit.
-      const unsigned long long back = issued < stages ? issued : stages;
-      for (unsigned long long m = issued - back; m < issued; ++m) {
-        uint64_t* bar = &s.full[m % stages];
-        const uint32_t par = (uint32_t)((m / stages) & 1ull);
-        const unsigned long long t0 = global_ns();
-        while (!mbar_try_wait(bar, par)) {
-          if (global_ns() - t0 > 1000000000ull) break;
-        }
-      }
-    }
+    const RingProducerView ring{s.buf, s.full, s.empty, s.item_id, s.ptrs, s.abort_flag};
+    const TileItemMap map{p.ntiles, p.slot0, p.KC, K_eff, p.tile_list, TILE_BYTES};
+    ring_producer(ring, map, lane, stages, TILE_BYTES, nitems, p.sched, p.ref, p.cands, p.nchunks > 1, p.status);
   } else {
     // ------------------------------ consumers -----------------------------
     uint32_t stage = 0, phase = 0;
