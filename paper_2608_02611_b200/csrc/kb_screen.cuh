@@ -482,9 +482,12 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
         }
 #pragma unroll
         for (int j = 0; j < NV; ++j) E::decode(w[j], &r[j * VEC]);
+        // (binary16 and e5m2 have no value in (0, 2^-100): their smallest are 2^-24 and 2^-16)
+        if constexpr (DT != KB_F16 && DT != KB_F8E5M2) {
 #pragma unroll
-        for (int e = 0; e < kEPT; ++e)   // 0 < |r| < 2^-100 on the bit pattern (zero wraps to the top)
-          extreme |= ((__float_as_uint(r[e]) & 0x7FFFFFFFu) - 1u) < (0x0D800000u - 1u);
+          for (int e = 0; e < kEPT; ++e)   // 0 < |r| < 2^-100 on the bit pattern (zero wraps to the top)
+            extreme |= ((__float_as_uint(r[e]) & 0x7FFFFFFFu) - 1u) < (0x0D800000u - 1u);
+        }
       }
       if (first_of_chunk) exchange_apply(tile_base);
 
