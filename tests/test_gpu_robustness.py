@@ -7,7 +7,9 @@
   leaves the context with its old, valid buffers;
 * guard bands: every caller-owned output sits between two bands of a canary pattern that must
   be intact after the call, and the library's own device buffers carry the same bands
-  (kb_ctx_check_guards) -- the stand-in for a memory checker.
+  (kb_ctx_check_guards) -- the stand-in for a memory checker;
+* reads: every input sits between halos of NaN patterns, so that an element read from outside
+  a tensor changes the records (NaN count, mismatch count, non-finite timing).
 """
 import os
 
@@ -380,3 +382,89 @@ def test_sharp_filter_is_chosen_for_dense_rounded_down_quotients_and_changes_not
         same_records(kb.records(ctx.screen(ref, sparse, 1e-2, 1.6e-2)), want_sparse)
         assert not ctx.last_filter_sharp
     assert ctx.poll() == 0
+
+
+# ---------------------------------------------------------------------------------------------
+# out-of-range READS: every input tensor sits between two halos of NaN patterns (all-ones bytes
+# are NaN in all six storage types).  An element read from outside [0, N) as a candidate would
+# be counted as NaN, as a reference it would count a mismatch: either differs from the oracle,
+# which only ever sees the tensor itself.
+# ---------------------------------------------------------------------------------------------
+
+HALO = 8192        # bytes on either side (a multiple of 256: the tensor stays 16-byte aligned)
+
+
+def between_nan_halos(values: torch.Tensor) -> torch.Tensor:
+    n = values.numel() * values.element_size()
+    raw = torch.full((n + 2 * HALO,), 0xFF, dtype=torch.uint8, device=values.device)
+    raw[HALO:HALO + n] = values.contiguous().view(torch.uint8).reshape(-1)
+    return raw[HALO:HALO + n].view(values.dtype)
+
+
+@pytest.mark.parametrize("dtype", [synth.F32, synth.F16, synth.BF16, synth.F8E4M3, synth.F8E5M2])
+def test_inputs_between_nan_halos_are_read_inside_their_bounds_only(ctx, kb, dtype):
+    dev = torch.device("cuda", 0)
+    rng = np.random.default_rng(900 + dtype)
+    tdt = synth.TORCH_DTYPE[dtype]
+    rtol = 0.3 if dtype in (synth.F8E4M3, synth.F8E5M2) else 1.6e-2
+    for N in (1, 7, 16, 4095, 4096, 4097, 3 * 4096 + 1000, 70000):
+        base = torch.from_numpy(rng.standard_normal(N).astype(np.float32)).to(dev)
+        ref = between_nan_halos(base.to(tdt))
+        cands = []
+        for k in range(3):
+            c = base.clone()
+            if k:                                   # a few real differences, first and last element among them
+                c[[0, N - 1]] += 0.5 * k
+                c[rng.integers(0, N, 3)] *= 1.01
+            cands.append(between_nan_halos(c.to(tdt)))
+        want = oracle_records(dtype, ref, cands, 1e-2, rtol)
+        assert (want["nan_count"] == 0).all()
+        masks = [(None, want)]
+        if N >= 4096:
+            spec = ("strided", 12, 2, 0)
+            masks.append((ctx.mask_strided(N, 12, 2, 0), oracle_records(dtype, ref, cands, 1e-2, rtol, spec)))
+        for small in (True, False):
+            ctx.set_small_path(small)
+            for mask, w in masks:
+                same_records(kb.records(ctx.screen(ref, cands, 1e-2, rtol, mask)), w)
+        ctx.set_small_path(True)
+        for m, _ in masks[1:]:
+            m.close()
+    assert ctx.poll() == 0
+
+
+def test_double_precision_inputs_between_nan_halos(ctx, kb):
+    dev = torch.device("cuda", 0)
+    rng = np.random.default_rng(977)
+    for N in (1, 9, 2047, 2048, 2049, 4097, 3 * 4096 + 1000):
+        base = torch.from_numpy(rng.standard_normal(N)).to(dev)
+        ref = between_nan_halos(base)
+        cands = [between_nan_halos(base * (1.0 + 1e-9 * k)) for k in range(3)]
+        want = oracle.screen_f64(ref.cpu().numpy(), [c.cpu().numpy() for c in cands], 1e-12, 1e-8)
+        got = kb.records_f64(ctx.screen_f64(ref, cands, 1e-12, 1e-8))
+        same_records(got, want)
+        assert (got["nan_count"] == 0).all()
+    assert ctx.poll() == 0
+
+
+@pytest.mark.parametrize("K,S", [(1, 1), (3, 5), (13, 33), (37, 100), (230, 17), (5, 2100)])
+def test_timings_between_nan_halos(ctx, kb, K, S):
+    """A timing read from outside [0, K*S) would be NaN: the call would report a non-finite
+    timing, or the medians and win counts would differ from the oracle's."""
+    dev = torch.device("cuda", 0)
+    rng = np.random.default_rng(K * 1000 + S)
+    t = (1.0 + rng.random((K, S))).astype(np.float32)
+    d_t = between_nan_halos(torch.from_numpy(t).to(dev).reshape(-1)).view(K, S)
+    want_med, want_iqr, want_wins = oracle.adjudicate(t)
+    for algo in (0, 1, 2, 3):
+        if algo == 3 and S > 1024:                  # the merge win count's row limit
+            continue
+        ctx.set_wins_algo(algo)
+        med, iqr, wins = ctx.adjudicate(d_t)
+        assert ctx.poll() == 0, algo
+        assert (fbits(med.cpu().numpy()) == fbits(want_med)).all(), algo
+        assert (fbits(iqr.cpu().numpy()) == fbits(want_iqr)).all(), algo
+        assert (wins.cpu().numpy() == want_wins).all(), algo
+    ctx.set_wins_algo(0)
+    ratios = ctx.tail_ratios(d_t)
+    assert torch.isfinite(ratios).all() and ctx.poll() == 0
