@@ -391,7 +391,7 @@ def test_sharp_filter_is_chosen_for_dense_rounded_down_quotients_and_changes_not
 # which only ever sees the tensor itself.
 # ---------------------------------------------------------------------------------------------
 
-HALO = 8192        # bytes on either side (a multiple of 256: the tensor stays 16-byte aligned)
+HALO = 32768       # bytes on either side: a whole kernel tile of any type (and a multiple of 256)
 
 
 def between_nan_halos(values: torch.Tensor) -> torch.Tensor:
