@@ -476,13 +476,22 @@ def main():
     assert ctx.poll() == 0 and ctx_adj.poll() == 0
 
     # ---- timed region: exactly `steps` steps, CUDA events, clocks sampled meanwhile ----
-    ctx.enable_timing(True)           # event pair around the dominant kernel only
+    # An event pair around the dominant kernel costs the step 6-9 us (the launches around it no
+    # longer run back to back, and the streaming kernel can no longer be set up while the lead
+    # kernel runs), so it is put on every fourth step of the timed region only.
+    TIMED_EVERY = 4
+    ctx.enable_timing(True)           # (creates the context's event pool, outside the timed region)
+    ctx.enable_timing(False)
     launches0 = ctx.launch_count + ctx_adj.launch_count
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     t_begin = time.perf_counter()
     e0.record()
-    for _ in range(steps):
+    for i in range(steps):
+        if i % TIMED_EVERY == 0:
+            ctx.enable_timing(True, keep=i > 0)
+        elif i % TIMED_EVERY == 1:
+            ctx.enable_timing(False)
         surv, n = step()
     e1.record()
     barrier()
@@ -616,6 +625,7 @@ def main():
                 "kernel": "screen_stream_kernel<bf16>", "launch_ms_avg": avg_stream_ms,
                 "launch_ms_min": float(np.min(stream_ms)) if len(stream_ms) else None,
                 "algorithmic_bytes_per_launch": stream_bytes, "launches_timed": int(len(stream_ms)),
+                "timed": f"every {TIMED_EVERY}th launch of the timed region",
                 "share_of_step": avg_stream_ms / ms_per_step}
 
     # ---- CPU baseline: the oracle as it stands on a bounded sample (rank 0, N=1 only) ----

@@ -26,6 +26,12 @@ kb_status kb_ctx_set_grid(kb_ctx* ctx, uint32_t blocks);
  * (streaming) path instead.  Results do not depend on it. */
 kb_status kb_ctx_set_small_path(kb_ctx* ctx, int on);
 
+/* Test/tuning hook: the streaming screen kernel is launched as a programmatic dependent of the
+ * lead kernel in front of it (its CTAs are set up while the lead kernel still runs and wait
+ * for it before they read anything); on = 0 launches it in plain stream order.  Never used
+ * while the stream is being captured into a graph.  Results do not depend on it. */
+kb_status kb_ctx_set_dependent_launch(kb_ctx* ctx, int on);
+
 /* Test/tuning hook: which instantiation of the streaming screen kernel runs.  0 = automatic
  * (the plain one, until a call reports that a quarter of its steps took a second look that
  * found nothing -- many elements whose quotient was rounded down to the largest relative
@@ -45,7 +51,9 @@ typedef enum {
 
 /* With timing on, every launch of the two kernels above is bracketed by a pair
  * of CUDA events recorded on the launching stream (taken from a ctx-owned
- * pool of 256 pairs per timer; older launches are overwritten). */
+ * pool of 256 pairs per timer, created at the first call with on != 0; older launches are
+ * overwritten).  on = 1 starts a new record, on = 0 stops recording and keeps the record,
+ * on = 2 goes on recording into the kept record (to time a subset of a sequence of calls). */
 kb_status kb_ctx_enable_timing(kb_ctx* ctx, int on);
 /* Wait for the recorded launches of `which` since the last read, write their
  * durations in milliseconds (oldest first, at most `cap`) to h_ms (HOST) and

@@ -43,7 +43,7 @@ RESULT_F64_BYTES = 56
 
 EXPORTS = [
     "kb_ctx_create", "kb_ctx_destroy", "kb_last_error", "kb_ctx_poll", "kb_ctx_set_grid",
-    "kb_ctx_enable_timing", "kb_ctx_read_timer", "kb_alu_probe", "kb_ctx_launch_count", "kb_ctx_set_wins_algo", "kb_ctx_set_small_path",
+    "kb_ctx_enable_timing", "kb_ctx_read_timer", "kb_alu_probe", "kb_ctx_launch_count", "kb_ctx_set_wins_algo", "kb_ctx_set_small_path", "kb_ctx_set_dependent_launch",
     "kb_mask_create_strided", "kb_mask_create_bitmap", "kb_mask_count", "kb_mask_destroy",
     "kb_screen", "kb_screen_f64", "kb_screen_host", "kb_screen_static", "kb_screen_indexed", "kb_screen_multi", "kb_adjudicate", "kb_adjudicate_ragged", "kb_select",
     "kb_select_by_score", "kb_tail_ratios", "kb_copeland", "kb_confirm",
@@ -85,6 +85,7 @@ def load() -> ctypes.CDLL:
     L.kb_ctx_launch_count.argtypes = [vp, ctypes.POINTER(u64)]
     L.kb_ctx_set_wins_algo.argtypes = [vp, i32]
     L.kb_ctx_set_small_path.argtypes = [vp, i32]
+    L.kb_ctx_set_dependent_launch.argtypes = [vp, i32]
     L.kb_ctx_set_filter.argtypes = [vp, i32]
     L.kb_ctx_last_filter.argtypes = [vp, ctypes.POINTER(i32)]
     L.kb_ctx_fail_next_allocs.argtypes = [vp, u32, u32]
@@ -233,6 +234,11 @@ class Context:
         """Enable/disable the single-launch kernel for small problems (a test hook)."""
         self._check(load().kb_ctx_set_small_path(self._h, 1 if on else 0), "kb_ctx_set_small_path")
 
+    def set_dependent_launch(self, on: bool):
+        """Launch the streaming kernel as a programmatic dependent of the lead kernel (default)
+        or in plain stream order (a test hook)."""
+        self._check(load().kb_ctx_set_dependent_launch(self._h, 1 if on else 0), "kb_ctx_set_dependent_launch")
+
     def set_filter(self, mode: int):
         """0 automatic, 1 always the plain streaming kernel, 2 always the sharp one (a tuning hook)."""
         self._check(load().kb_ctx_set_filter(self._h, int(mode)), "kb_ctx_set_filter")
@@ -265,8 +271,10 @@ class Context:
         self._check(load().kb_ctx_selftest_wait(self._h, int(limit_ns), _stream_ptr(self.device)),
                     "kb_ctx_selftest_wait")
 
-    def enable_timing(self, on: bool = True):
-        self._check(load().kb_ctx_enable_timing(self._h, 1 if on else 0), "kb_ctx_enable_timing")
+    def enable_timing(self, on: bool = True, keep: bool = False):
+        """Event pairs around the instrumented kernels: on starts a new record (or, with
+        ``keep``, goes on with the one there is); off stops recording and keeps the record."""
+        self._check(load().kb_ctx_enable_timing(self._h, (2 if keep else 1) if on else 0), "kb_ctx_enable_timing")
 
     def read_timer(self, which: int, cap: int = 256) -> np.ndarray:
         """Durations (ms) of the instrumented kernel's launches since the last read."""

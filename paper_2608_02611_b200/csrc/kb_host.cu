@@ -80,6 +80,7 @@ struct kb_ctx {
   // instrumentation
   uint64_t launches = 0;
   bool timing = false;
+  bool dependent_launch = true;     // streaming kernel as a programmatic dependent of the lead kernel
   static constexpr int kTimers = 2, kPool = 256;
   cudaEvent_t tm_beg[kTimers][kPool] = {};
   cudaEvent_t tm_end[kTimers][kPool] = {};
@@ -248,7 +249,7 @@ constexpr int kSharpCalls = 32, kSharpGrace = 4;
 // e4m3 kernel: stages of 4 KB, CTAs of 160 threads, four resident per SM at 96 registers
 constexpr uint32_t kStages8 = KB8_STAGES, kCtas8 = 4;
 template <int DT>
-kb_status launch_stream(kb_ctx* ctx, StreamParams& sp, cudaStream_t st) {
+kb_status launch_stream(kb_ctx* ctx, StreamParams& sp, cudaStream_t st, bool behind_lead = false) {
   const uint32_t tile_bytes = kTile * Elem<DT>::kBytes;
   constexpr bool k8 = DT == KB_F8E4M3;           // e4m3 has a kernel of its own (kb_screen8.cuh)
   sp.stages = k8 ? kStages8 : stream_stages(tile_bytes);
@@ -290,10 +291,24 @@ kb_status launch_stream(kb_ctx* ctx, StreamParams& sp, cudaStream_t st) {
     if constexpr (k8) {
       screen_stream8_kernel<DT><<<(unsigned int)grid, kThreads8, smem, st>>>(sp);
     } else {
-      if (sharp)
-        screen_stream_kernel<DT, true><<<(unsigned int)grid, kStreamThreads, smem, st>>>(sp);
-      else
-        screen_stream_kernel<DT, false><<<(unsigned int)grid, kStreamThreads, smem, st>>>(sp);
+      if (sharp) {
+        screen_stream_kernel<DT, 1><<<(unsigned int)grid, kStreamThreads, smem, st>>>(sp);
+      } else if (behind_lead && ctx->dependent_launch) {
+        // launch and set-up overlap the lead kernel (about 3 us per call)
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned int)grid);
+        cfg.blockDim = dim3(kStreamThreads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        KB_CUDA(ctx, cudaLaunchKernelEx(&cfg, screen_stream_kernel<DT, 2>, sp));
+      } else {
+        screen_stream_kernel<DT, 0><<<(unsigned int)grid, kStreamThreads, smem, st>>>(sp);
+      }
     }
   }
   ++ctx->launches;
@@ -327,14 +342,19 @@ kb_status set_stream_attr(kb_ctx* ctx) {
   } else {
     const uint32_t tile_bytes = kTile * Elem<DT>::kBytes;
     const size_t smem = stream_smem_bytes(stream_stages(tile_bytes), tile_bytes);
-    KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT, false>,
+    KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT, 0>,
                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT, false>,
+    KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT, 0>,
                                       cudaFuncAttributePreferredSharedMemoryCarveout,
                                       (int)cudaSharedmemCarveoutMaxShared));
-    KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT, true>,
+    KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT, 1>,
                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT, true>,
+    KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT, 1>,
+                                      cudaFuncAttributePreferredSharedMemoryCarveout,
+                                      (int)cudaSharedmemCarveoutMaxShared));
+    KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT, 2>,
+                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT, 2>,
                                       cudaFuncAttributePreferredSharedMemoryCarveout,
                                       (int)cudaSharedmemCarveoutMaxShared));
   }
@@ -513,6 +533,12 @@ extern "C" kb_status kb_ctx_last_filter(const kb_ctx* ctx, int* sharp) {
   return KB_OK;
 }
 
+extern "C" kb_status kb_ctx_set_dependent_launch(kb_ctx* ctx, int on) {
+  if (!ctx) return KB_ERR_INVALID_ARG;
+  ctx->dependent_launch = on != 0;
+  return KB_OK;
+}
+
 extern "C" kb_status kb_ctx_set_small_path(kb_ctx* ctx, int on) {
   if (!ctx) return KB_ERR_INVALID_ARG;
   ctx->small_on = on != 0;
@@ -570,7 +596,7 @@ extern "C" kb_status kb_ctx_enable_timing(kb_ctx* ctx, int on) {
       }
   }
   ctx->timing = on != 0;
-  ctx->tm_used[0] = ctx->tm_used[1] = 0;
+  if (on == 1) ctx->tm_used[0] = ctx->tm_used[1] = 0;
   return KB_OK;
 }
 
@@ -980,7 +1006,7 @@ kb_status screen_impl(kb_ctx* ctx, const void* d_ref, const void* const* h_cands
       sp.done = counters;
       sp.sched = reinterpret_cast<unsigned long long*>(counters + 2);
       sp.out = d_out;
-      rc = launch_stream<DT>(ctx, sp, st);
+      rc = launch_stream<DT>(ctx, sp, st, lead_ran && !capturing);
       return rc == KB_OK ? finished() : rc;
     }
   }

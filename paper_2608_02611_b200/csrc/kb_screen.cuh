@@ -186,8 +186,12 @@ __host__ __device__ inline size_t stream_smem_bytes(uint32_t stages, uint32_t ti
 // fruitless second looks per candidate (they travel in the accumulator's spare word); the lead
 // kernels of the following calls add them up and publish their share of all warp steps to the
 // host, which picks the instantiation from it.  The records do not depend on the choice.
-template <int DT, bool SHARP>
+//
+// MODE 0: plain, 1: sharp, 2: plain, launched as a programmatic dependent of the lead kernel
+// (short calls: its CTAs are set up while the lead kernel still runs, and wait for it below).
+template <int DT, int MODE>
 __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
+  constexpr bool SHARP = MODE == 1;
   using E = Elem<DT>;
   constexpr int VEC = E::kVec;
   constexpr int NV = kEPT / VEC;
@@ -250,6 +254,8 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
   }
   for (int i = tid; i < kMaxKC * kWarps; i += kStreamThreads) s.thr2[i] = make_float2(-1.0f, 0.0f);
   __syncthreads();
+  // everything the lead kernel wrote (pointer table, seeds, zeroed counters) is read below
+  if constexpr (MODE == 2) asm volatile("griddepcontrol.wait;" ::: "memory");
 
   // Work items (chunk, tile), chunk-major, are drawn from a global counter: a CTA gets
   // ascending items (so ascending tiles inside a chunk, which the index tie-break needs),
@@ -856,6 +862,9 @@ __global__ void __launch_bounds__(256) screen_lead_kernel(const LeadParams p, co
   const unsigned int per_block = p.per_block;
   const unsigned int kBlocksPerTile = kTile / per_block;
   const unsigned int k = blockIdx.y;
+  // a streaming kernel launched as a programmatic dependent may be set up from here on (it
+  // waits for this grid to finish before it reads anything); no effect otherwise
+  asm volatile("griddepcontrol.launch_dependents;");
   if (blockIdx.x == 0) {
     if (threadIdx.x == 0 && p.from_args) p.table[k] = chunk_ptrs.p[k];
     unsigned long long looks = 0ull;

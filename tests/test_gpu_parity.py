@@ -100,14 +100,20 @@ def run_screen(ctx, kb, ref, cands, atol, rtol, mask_spec=None, N=None):
             mask = ctx.mask_bitmap(N, mask_spec[1], mask_spec[2])
     # both dispatch paths: the general (streaming) one and, where the size allows it, the
     # single-launch kernel for small problems; they must agree byte for byte
+    # (and the general path with the streaming kernel launched in plain stream order instead of
+    # as a programmatic dependent of the lead kernel)
     try:
         ctx.set_small_path(False)
         rec = kb.records(ctx.screen(ref, cands, atol, rtol, mask))
+        ctx.set_dependent_launch(False)
+        rec_plain = kb.records(ctx.screen(ref, cands, atol, rtol, mask))
     finally:
         ctx.set_small_path(True)
+        ctx.set_dependent_launch(True)
     rec_small = kb.records(ctx.screen(ref, cands, atol, rtol, mask))
     assert ctx.poll() == 0
     assert rec.tobytes() == rec_small.tobytes()
+    assert rec.tobytes() == rec_plain.tobytes()
     if mask is not None:
         mask.close()
     return rec

@@ -468,3 +468,25 @@ def test_timings_between_nan_halos(ctx, kb, K, S):
     ctx.set_wins_algo(0)
     ratios = ctx.tail_ratios(d_t)
     assert torch.isfinite(ratios).all() and ctx.poll() == 0
+
+
+def test_kernel_timers_record_a_subset_of_a_sequence_of_calls(ctx, kb):
+    dev = torch.device("cuda", 0)
+    ref = torch.zeros(64 * 4096, dtype=torch.bfloat16, device=dev)
+    cands = kb.Candidates([ref.clone() for _ in range(4)])
+    ctx.set_small_path(False)
+    for i in range(9):                              # timers on for calls 0, 4 and 8
+        if i % 4 == 0:
+            ctx.enable_timing(True, keep=i > 0)
+        elif i % 4 == 1:
+            ctx.enable_timing(False)
+        ctx.screen(ref, cands, 0.0, 0.0)
+    ms = ctx.read_timer(kb.KB_TIMER_SCREEN_STREAM)
+    assert len(ms) == 3 and (ms > 0).all()
+    assert len(ctx.read_timer(kb.KB_TIMER_SCREEN_STREAM)) == 0      # a read clears the record
+    ctx.enable_timing(True)                                          # a plain "on" starts afresh
+    ctx.screen(ref, cands, 0.0, 0.0)
+    assert len(ctx.read_timer(kb.KB_TIMER_SCREEN_STREAM)) == 1
+    ctx.enable_timing(False)
+    ctx.set_small_path(True)
+    assert ctx.poll() == 0
