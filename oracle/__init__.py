@@ -105,6 +105,8 @@ def lib() -> ctypes.CDLL:
         L.kbo_confirm.restype = i32
         L.kbo_adjudicate_ragged.argtypes = [vp, vp, u32, vp, vp, vp]
         L.kbo_adjudicate_ragged.restype = i32
+        L.kbo_merge_ranges.argtypes = [vp, u32, u32, vp, vp]
+        L.kbo_merge_ranges.restype = i32
         L.kbo_decode_f16.argtypes = [ctypes.c_uint16]
         L.kbo_decode_f16.restype = f32
         L.kbo_decode_bf16.argtypes = [ctypes.c_uint16]
@@ -374,3 +376,20 @@ def adjudicate_ragged(rows):
     if rc != 0:
         raise ValueError(f"kbo_adjudicate_ragged rejected its arguments (rc={rc})")
     return med, iqr, wins
+
+
+def merge_ranges(parts, first) -> np.ndarray:
+    """Records of a whole element range from the records of R consecutive parts of it:
+    ``parts`` is a sequence of R record arrays (K each), ``first`` the global index of each
+    part's first element."""
+    R = len(parts)
+    K = len(parts[0])
+    flat = np.ascontiguousarray(np.concatenate([np.asarray(p, dtype=RESULT_DTYPE).reshape(-1) for p in parts]))
+    if flat.size != R * K:
+        raise ValueError("every part must hold K records")
+    first = np.ascontiguousarray(first, dtype=np.uint64)
+    out = np.zeros(K, dtype=RESULT_DTYPE)
+    rc = lib().kbo_merge_ranges(flat.ctypes.data, R, K, first.ctypes.data, out.ctypes.data)
+    if rc != 0:
+        raise ValueError(f"kbo_merge_ranges rejected its arguments (rc={rc})")
+    return out

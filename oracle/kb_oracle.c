@@ -647,3 +647,43 @@ int kbo_adjudicate_ragged(const float* timings, const uint32_t* offsets, uint32_
   }
   return 0;
 }
+
+/*
+ * The gate over an element range split into R consecutive parts (Sec. 3.1 K(p); the paper
+ * runs on one GPU, this is the definition carried over a partition of the index set): the
+ * record of the whole range from the records of the parts.  parts[r*K + k] is candidate k's
+ * record over part r, whose first element has global index first[r] (ascending in r).
+ *   counts add; the largest error wins, the earlier part on ties (its indices are lower),
+ *   with its index moved to global numbering; the largest relative error is the maximum;
+ *   pass = no mismatch anywhere.  A part without a finite difference (argmax_idx = -1)
+ *   contributes no error.
+ * Returns 0, or -1 on a bad argument.
+ */
+int kbo_merge_ranges(const kbo_screen_result* parts, uint32_t R, uint32_t K, const uint64_t* first,
+                     kbo_screen_result* out) {
+  uint32_t r, k;
+  if (!parts || !first || !out || R == 0 || K == 0) return -1;
+  for (r = 1; r < R; ++r)
+    if (first[r] <= first[r - 1]) return -1;
+  for (k = 0; k < K; ++k) {
+    kbo_screen_result m;
+    int have = 0;
+    memset(&m, 0, sizeof m);
+    m.argmax_idx = -1;
+    for (r = 0; r < R; ++r) {
+      const kbo_screen_result* p = &parts[(size_t)r * K + k];
+      m.mismatch_count += p->mismatch_count;
+      m.nan_count += p->nan_count;
+      m.inf_count += p->inf_count;
+      if (p->argmax_idx >= 0 && (!have || p->max_abs_err > m.max_abs_err)) {
+        have = 1;
+        m.max_abs_err = p->max_abs_err;
+        m.argmax_idx = p->argmax_idx + (int64_t)first[r];
+      }
+      if (p->max_rel_err > m.max_rel_err) m.max_rel_err = p->max_rel_err;
+    }
+    m.pass = (m.mismatch_count == 0) ? 1u : 0u;
+    out[k] = m;
+  }
+  return 0;
+}

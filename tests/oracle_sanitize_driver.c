@@ -187,6 +187,34 @@ static int run_ragged_and_select(void) {
   if (!(kbo_score(1.0f, 1, 8, 0.02f, 0.01f) > kbo_score(2.0f, 1, 8, 0.02f, 0.01f)))
     return fail("score not decreasing in time", 0, 0);
   free(t);
+  /* a range in three parts: the merged records are those of the whole range */
+  {
+    const uint64_t N = 3000, cuts[4] = {0, 1, 1500, 3000};
+    const uint64_t first[3] = {0, 1, 1500};
+    float* r = (float*)malloc((size_t)N * 4);
+    float* c = (float*)malloc((size_t)N * 4);
+    kbo_screen_result* parts = (kbo_screen_result*)malloc(3 * sizeof(kbo_screen_result));
+    kbo_screen_result whole, merged;
+    uint64_t j;
+    if (!r || !c || !parts) return fail("malloc", (long)N, 0);
+    for (j = 0; j < N; ++j) {
+      r[j] = timing();
+      c[j] = (rnd() & 7u) ? r[j] : r[j] + 0.125f;
+    }
+    for (j = 0; j < 3; ++j)
+      if (kbo_screen(r + cuts[j], c + cuts[j], cuts[j + 1] - cuts[j], KBO_F32, 1e-2f, 1e-2f, KBO_MASK_NONE, 0, 0,
+                     0, NULL, &parts[j]))
+        return fail("screen part", (long)j, 0);
+    if (kbo_screen(r, c, N, KBO_F32, 1e-2f, 1e-2f, KBO_MASK_NONE, 0, 0, 0, NULL, &whole)) return fail("screen whole", 0, 0);
+    if (kbo_merge_ranges(parts, 3, 1, first, &merged)) return fail("merge_ranges", 0, 0);
+    if (merged.mismatch_count != whole.mismatch_count || merged.argmax_idx != whole.argmax_idx ||
+        merged.max_abs_err != whole.max_abs_err || merged.max_rel_err != whole.max_rel_err ||
+        merged.pass != whole.pass)
+      return fail("merged parts differ from the whole", (long)merged.argmax_idx, (long)whole.argmax_idx);
+    free(r);
+    free(c);
+    free(parts);
+  }
   return 0;
 }
 
