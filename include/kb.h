@@ -194,6 +194,21 @@ kb_status kb_screen_multi(kb_ctx* ctx, uint32_t G, const void* const* h_refs,
                           kb_dtype dtype, float atol, float rtol, kb_screen_result* d_out,
                           void* stream);
 
+/* The gate over an element range cut into R consecutive parts (the definition of Sec. 3.1
+ * K(p) carried over a partition of the index set; used when the ELEMENTS of a few large
+ * tensors, not the candidates, are spread over several GPUs): the records of the whole range
+ * from the records of its parts.  Counts add; the largest error wins and the earlier part
+ * keeps it on a tie (its indices are lower), with argmax_idx moved to global numbering; the
+ * largest relative error is the maximum; pass = no mismatch anywhere.  A part that saw no
+ * finite difference (argmax_idx = -1) contributes no error.
+ *   d_parts  DEVICE [R][K] records, part after part; part r covers the elements from global
+ *            index h_first[r] on (the parts' own records number their elements from 0).
+ *   h_first  HOST array of R strictly ascending indices.
+ *   d_out    DEVICE [K] records (8-byte aligned); may not overlap d_parts.
+ * 1 <= R <= 64, 1 <= K <= KB_MAX_K.  Asynchronous on `stream`; no allocation. */
+kb_status kb_merge_ranges(kb_ctx* ctx, const kb_screen_result* d_parts, uint32_t R, uint32_t K,
+                          const uint64_t* h_first, kb_screen_result* d_out, void* stream);
+
 /* ---- the gate for double-precision tensors (Sec. 3.1 K(p); Sec. 3.4 Verifier) ----
  * The same gate with the reference and the candidates stored in binary64 and
  * EVERY operation of the record (d, tol, the comparison, d/|r|) in binary64,

@@ -45,7 +45,7 @@ EXPORTS = [
     "kb_ctx_create", "kb_ctx_destroy", "kb_last_error", "kb_ctx_poll", "kb_ctx_set_grid",
     "kb_ctx_enable_timing", "kb_ctx_read_timer", "kb_alu_probe", "kb_ctx_launch_count", "kb_ctx_set_wins_algo", "kb_ctx_set_small_path", "kb_ctx_set_dependent_launch",
     "kb_mask_create_strided", "kb_mask_create_bitmap", "kb_mask_count", "kb_mask_destroy",
-    "kb_screen", "kb_screen_f64", "kb_screen_host", "kb_screen_static", "kb_screen_indexed", "kb_screen_multi", "kb_adjudicate", "kb_adjudicate_ragged", "kb_select",
+    "kb_screen", "kb_screen_f64", "kb_screen_host", "kb_screen_static", "kb_screen_indexed", "kb_screen_multi", "kb_merge_ranges", "kb_adjudicate", "kb_adjudicate_ragged", "kb_select",
     "kb_select_by_score", "kb_tail_ratios", "kb_copeland", "kb_confirm",
     "kb_ctx_fail_next_allocs", "kb_ctx_selftest_wait", "kb_ctx_check_guards", "kb_static_scratch_read", "kb_ctx_set_filter", "kb_ctx_last_filter",
 ]
@@ -101,6 +101,7 @@ def load() -> ctypes.CDLL:
     L.kb_screen_host.argtypes = [vp, vp, vp, u32, u64, i32, f32, f32, vp, vp, vp]
     L.kb_screen_indexed.argtypes = [vp, vp, vp, u32, vp, vp, u32, u64, i32, f32, f32, vp, vp, vp]
     L.kb_screen_multi.argtypes = [vp, u32, vp, vp, vp, vp, i32, f32, f32, vp, vp]
+    L.kb_merge_ranges.argtypes = [vp, vp, u32, u32, vp, vp, vp]
     L.kb_screen_static.argtypes = [vp, vp, u32, u64, i32, f32, f32, vp, vp]
     L.kb_adjudicate.argtypes = [vp, vp, u32, u32, vp, vp, vp, vp]
     L.kb_adjudicate_ragged.argtypes = [vp, vp, vp, u32, u32, u64, vp, vp, vp, vp]
@@ -544,6 +545,24 @@ def screen_multi(self, groups, atol: float, rtol: float, out: Optional[torch.Ten
     rc = load().kb_screen_multi(self._h, G, refs, ptrs, Ks, Ns, DTYPE_CODE.get(groups[0][0].dtype, -1),
                                 float(atol), float(rtol), out.data_ptr(), _stream_ptr(dev))
     self._check(rc, "kb_screen_multi")
+    return out
+
+
+@_ctx_method
+def merge_ranges(self, parts: torch.Tensor, first, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """kb_merge_ranges: ``parts`` is a uint8 CUDA tensor [R, K, 48] of the records of R
+    consecutive parts of an element range, ``first`` the global index of each part's first
+    element.  Returns the [K, 48] records of the whole range."""
+    R, K = int(parts.shape[0]), int(parts.shape[1])
+    if parts.dtype != torch.uint8 or parts.dim() != 3 or parts.shape[2] != RESULT_BYTES or not parts.is_contiguous():
+        raise KbError(1, "kb_merge_ranges", "parts must be a contiguous uint8 tensor [R, K, 48]")
+    firsts = (ctypes.c_uint64 * max(R, 1))(*[int(x) for x in first])
+    if len(first) != R:
+        raise KbError(1, "kb_merge_ranges", "one first index per part")
+    if out is None:
+        out = torch.empty((K, RESULT_BYTES), dtype=torch.uint8, device=parts.device)
+    rc = load().kb_merge_ranges(self._h, parts.data_ptr(), R, K, firsts, out.data_ptr(), _stream_ptr(parts.device))
+    self._check(rc, "kb_merge_ranges")
     return out
 
 

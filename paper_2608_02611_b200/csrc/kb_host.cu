@@ -1044,6 +1044,33 @@ extern "C" kb_status kb_screen(kb_ctx* ctx, const void* d_ref, const void* const
 // ---------------------------------------------------------------------------
 // kb_screen_f64: the gate in binary64
 // ---------------------------------------------------------------------------
+extern "C" kb_status kb_merge_ranges(kb_ctx* ctx, const kb_screen_result* d_parts, uint32_t R, uint32_t K,
+                                     const uint64_t* h_first, kb_screen_result* d_out, void* stream) {
+  TraceRange trace("kb_merge_ranges");
+  if (!ctx) return KB_ERR_INVALID_ARG;
+  if (!d_parts || !h_first || !d_out) return fail(ctx, KB_ERR_INVALID_ARG, "kb_merge_ranges: null pointer");
+  if (R == 0 || R > (uint32_t)kMergeMaxParts)
+    return fail(ctx, KB_ERR_INVALID_ARG, "kb_merge_ranges: R=%u outside [1, %d]", R, kMergeMaxParts);
+  if (K == 0 || K > KB_MAX_K) return fail(ctx, KB_ERR_INVALID_ARG, "kb_merge_ranges: K=%u outside [1, %u]", K, KB_MAX_K);
+  if ((reinterpret_cast<uintptr_t>(d_parts) & 7u) || (reinterpret_cast<uintptr_t>(d_out) & 7u))
+    return fail(ctx, KB_ERR_ALIGNMENT, "kb_merge_ranges: records not 8-byte aligned");
+  RangeFirsts f;
+  for (uint32_t r = 0; r < (uint32_t)kMergeMaxParts; ++r) f.first[r] = 0ull;
+  for (uint32_t r = 0; r < R; ++r) {
+    if (r && h_first[r] <= h_first[r - 1])
+      return fail(ctx, KB_ERR_INVALID_ARG, "kb_merge_ranges: the parts' first indices must ascend (part %u)", r);
+    if (h_first[r] >= KB_MAX_N)
+      return fail(ctx, KB_ERR_INVALID_ARG, "kb_merge_ranges: first index of part %u beyond the element limit", r);
+    f.first[r] = h_first[r];
+  }
+  DeviceGuard g(ctx->device);
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  merge_ranges_kernel<<<(K + 127) / 128, 128, 0, st>>>(d_parts, R, K, f, d_out);
+  ++ctx->launches;
+  KB_CUDA(ctx, cudaGetLastError());
+  return KB_OK;
+}
+
 extern "C" kb_status kb_screen_f64(kb_ctx* ctx, const double* d_ref, const double* const* h_cands,
                                    uint32_t K, uint64_t N, double atol, double rtol,
                                    const kb_mask* mask, kb_screen_result_f64* d_out, void* stream) {

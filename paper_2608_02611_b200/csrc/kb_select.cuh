@@ -169,4 +169,42 @@ __global__ void confirm_kernel(const float* __restrict__ s1, const float* __rest
   score[k] = sc;
 }
 
+// ---------------------------------------------------------------------------
+// Records of a whole element range from the records of its R consecutive parts
+// (kb_merge_ranges): one thread per candidate walks the parts in order.
+// ---------------------------------------------------------------------------
+constexpr int kMergeMaxParts = 64;
+struct RangeFirsts {
+  unsigned long long first[kMergeMaxParts];
+};
+
+__global__ void merge_ranges_kernel(const kb_screen_result* __restrict__ parts, unsigned int R,
+                                    unsigned int K, const RangeFirsts f,
+                                    kb_screen_result* __restrict__ out) {
+  const unsigned int k = blockIdx.x * blockDim.x + threadIdx.x;
+  if (k >= K) return;
+  kb_screen_result m;
+  m.mismatch_count = m.nan_count = m.inf_count = 0ull;
+  m.argmax_idx = -1;
+  m.max_abs_err = 0.0f;
+  m.max_rel_err = 0.0f;
+  m.reserved = 0u;
+  bool have = false;
+  for (unsigned int r = 0; r < R; ++r) {
+    const kb_screen_result p = parts[(size_t)r * K + k];
+    m.mismatch_count += p.mismatch_count;
+    m.nan_count += p.nan_count;
+    m.inf_count += p.inf_count;
+    // errors are non-negative and finite: their order is the order of their bit patterns
+    if (p.argmax_idx >= 0 && (!have || __float_as_uint(p.max_abs_err) > __float_as_uint(m.max_abs_err))) {
+      have = true;
+      m.max_abs_err = p.max_abs_err;
+      m.argmax_idx = p.argmax_idx + (long long)f.first[r];
+    }
+    if (__float_as_uint(p.max_rel_err) > __float_as_uint(m.max_rel_err)) m.max_rel_err = p.max_rel_err;
+  }
+  m.pass = m.mismatch_count == 0ull ? 1u : 0u;
+  out[k] = m;
+}
+
 }  // namespace kb

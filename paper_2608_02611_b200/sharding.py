@@ -71,3 +71,60 @@ def screen_sharded(ctx, ref: torch.Tensor, make_cand, K: int, atol: float, rtol:
     out = gather_records(local, K, device=ref.device)
     return out.reshape(-1).view(binding.RESULT_DTYPE)
 
+
+
+# ---------------------------------------------------------------------------------------------
+# Element-range sharding: few, large tensors (the last rungs of a funnel: 3 candidates of 1.6e9
+# elements).  Every rank holds one contiguous part of the reference and of every candidate,
+# screens it, and the K records of the parts are merged into the records of the whole range
+# (kb_merge_ranges).  The only exchange is an all-gather of R x K 48-byte records.
+# ---------------------------------------------------------------------------------------------
+
+RANGE_ALIGN = 4096          # elements: parts start on kernel-tile boundaries (and so 16-byte aligned)
+
+
+def element_range(N: int, rank: int, world: int, align: int = RANGE_ALIGN):
+    """[lo, hi) of rank's part of N elements: consecutive, covering, every part but the last a
+    whole number of `align`-element tiles; trailing ranks get an empty part when there are
+    fewer tiles than ranks."""
+    tiles = (N + align - 1) // align
+    per, extra = divmod(tiles, world)
+    t_lo = rank * per + min(rank, extra)
+    t_hi = t_lo + per + (1 if rank < extra else 0)
+    return min(t_lo * align, N), min(t_hi * align, N)
+
+
+def gather_parts(local: torch.Tensor, lo: int, hi: int):
+    """All-gather every rank's [K, 48] records and range start.  Returns (parts, firsts): the
+    records of the non-empty parts as one uint8 tensor [R, K, 48] on `local`'s device, in
+    ascending range order, and their first global indices."""
+    world = dist.get_world_size()
+    local = local.contiguous().view(torch.uint8).reshape(-1, RECORD_BYTES)
+    got = [torch.empty_like(local) for _ in range(world)]
+    dist.all_gather(got, local)
+    bounds = torch.tensor([lo, hi], dtype=torch.int64, device=local.device)
+    all_bounds = [torch.empty_like(bounds) for _ in range(world)]
+    dist.all_gather(all_bounds, bounds)
+    keep = [(int(b[0]), r) for r, b in enumerate(all_bounds) if int(b[1]) > int(b[0])]
+    keep.sort()
+    parts = torch.stack([got[r] for _, r in keep])
+    return parts, [f for f, _ in keep]
+
+
+def screen_range_sharded(ctx, ref_part: torch.Tensor, cand_parts, lo: int, hi: int,
+                         atol: float, rtol: float) -> np.ndarray:
+    """The gate over tensors whose ELEMENTS are spread over the ranks of the default process
+    group: this rank holds elements [lo, hi) of the reference (`ref_part`) and of each of the
+    K candidates (`cand_parts`), with `lo` a multiple of RANGE_ALIGN (see `element_range`).
+    Each rank screens its part through `ctx`; the records are all-gathered and merged on the
+    device by kb_merge_ranges, so every rank returns the K records of the whole range.  A rank
+    with an empty part (hi == lo) passes any tensors of K candidates' shape [0]."""
+    from . import binding
+    K = len(cand_parts)
+    if hi > lo:
+        local = ctx.screen(ref_part, cand_parts, atol, rtol)
+    else:
+        local = torch.zeros((K, RECORD_BYTES), dtype=torch.uint8, device=ref_part.device)
+    parts, firsts = gather_parts(local, lo, hi)
+    merged = ctx.merge_ranges(parts, firsts)
+    return binding.records(merged)

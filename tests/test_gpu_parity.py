@@ -875,3 +875,52 @@ def test_fp8_every_byte_pair_behind_established_maxima(ctx, kb, dtype_code):
                 ctx.set_grid(0)
             assert ctx.poll() == 0
             assert_records_equal(got, want, f"fp8 {dtype_code} atol={atol} rtol={rtol} grid={grid}")
+
+
+# --------------------------------------------------------------------------
+# records of a range from the records of its parts (element-range sharding)
+# --------------------------------------------------------------------------
+
+@pytest.mark.parametrize("dtype_code", [synth.F32, synth.BF16, synth.F16])
+@pytest.mark.parametrize("cuts", [[], [4096], [4096, 8192, 12288], [8192, 36864]])
+def test_merge_ranges_gives_the_whole_range(ctx, kb, dtype_code, cuts):
+    rng = np.random.default_rng(31 + dtype_code + len(cuts))
+    dev = torch.device("cuda", 0)
+    N = 10 * 4096 + 333
+    ref = awkward(N, dtype_code, rng, dev)
+    cands = [perturbed(ref, dtype_code, rng, dev) for _ in range(5)]
+    same_err = ref.clone()                          # the same largest error on both sides of every cut
+    ref[0] = 1.0
+    same_err[0] = 1.0
+    for cut in cuts:
+        for i in (cut - 1, cut):
+            ref[i] = 1.0
+            same_err[i] = 3.0
+    for c in cands:
+        for i in [0] + [j for cut in cuts for j in (cut - 1, cut)]:
+            c[i] = ref[i]
+    all_nan_first_part = ref.clone()                # a part without any finite difference
+    all_nan_first_part[: (cuts[0] if cuts else N)] = float("nan")
+    cands += [same_err, all_nan_first_part]
+    want = oracle_screen(dtype_code, ref, cands, 1e-2, 1.6e-2)
+    first = [0] + cuts
+    last = cuts + [N]
+    parts = torch.stack([ctx.screen(ref[a:b], [c[a:b] for c in cands], 1e-2, 1.6e-2) for a, b in zip(first, last)])
+    got = kb.records(ctx.merge_ranges(parts, first))
+    assert_records_equal(got, want, f"dtype={dtype_code} cuts={cuts}")
+    # ... and the oracle's own merge of the oracle's own part records says the same
+    oparts = [oracle_screen(dtype_code, ref[a:b], [c[a:b] for c in cands], 1e-2, 1.6e-2) for a, b in zip(first, last)]
+    assert_records_equal(got, oracle.merge_ranges(oparts, first), "oracle merge")
+    assert ctx.poll() == 0
+
+
+def test_merge_ranges_argument_errors(ctx, kb):
+    dev = torch.device("cuda", 0)
+    parts = torch.zeros((2, 3, 48), dtype=torch.uint8, device=dev)
+    with pytest.raises(kb.KbError):
+        ctx.merge_ranges(parts, [4096, 4096])                     # must ascend
+    with pytest.raises(kb.KbError):
+        ctx.merge_ranges(parts, [0])                              # one index per part
+    with pytest.raises(kb.KbError):
+        ctx.merge_ranges(torch.zeros((65, 1, 48), dtype=torch.uint8, device=dev), list(range(0, 65 * 4096, 4096)))
+    assert ctx.poll() == 0
