@@ -5,6 +5,7 @@
 #include <cuda_runtime_api.h>
 #include <math.h>
 #include <stdio.h>
+#include <string.h>
 #include <stdlib.h>
 
 #include "kb.h"
@@ -65,6 +66,33 @@ int main(void) {
   if (!(out[2].pass == 0 && out[2].mismatch_count == 1 && out[2].nan_count == 1 && out[2].argmax_idx == 0)) {
     fprintf(stderr, "candidate 2: unexpected record\n");
     return 4;
+  }
+  /* the same tensors in two parts cut on a tile boundary, merged: the same records */
+  {
+    const uint64_t cut = 4096u * 50u;
+    const uint64_t first[2] = {0u, cut};
+    kb_screen_result *d_parts = 0, *d_merged = 0;
+    kb_screen_result merged[3];
+    const void* lo[3];
+    const void* hi[3];
+    CHECK(cudaMalloc((void**)&d_parts, 2 * sizeof out));
+    CHECK(cudaMalloc((void**)&d_merged, sizeof out));
+    for (k = 0; k < 3; ++k) {
+      lo[k] = d_c[k];
+      hi[k] = d_c[k] + cut;
+    }
+    CHECK(kb_screen(ctx, d_ref, lo, 3, cut, KB_F32, 1e-3f, 1e-3f, 0, d_parts, 0));
+    CHECK(kb_screen(ctx, d_ref + cut, hi, 3, N - cut, KB_F32, 1e-3f, 1e-3f, 0, d_parts + 3, 0));
+    CHECK(kb_merge_ranges(ctx, d_parts, 2, 3, first, d_merged, 0));
+    CHECK(kb_ctx_poll(ctx, 0, &dev_status));
+    CHECK(dev_status);
+    CHECK(cudaMemcpy(merged, d_merged, sizeof merged, cudaMemcpyDeviceToHost));
+    if (memcmp(merged, out, sizeof out) != 0) {
+      fprintf(stderr, "merged parts differ from the whole range\n");
+      return 5;
+    }
+    cudaFree(d_parts);
+    cudaFree(d_merged);
   }
   CHECK(kb_ctx_destroy(ctx));
   printf("ok\n");
