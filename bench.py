@@ -301,6 +301,16 @@ def run_paper_scale(args):
     ctx = binding.Context(0)
     peak, src = peaks()
     calls = max(3, min(args.steps, 20))
+    # a fresh process finds the GPU at idle clocks: keep it busy for a moment first, or the first
+    # (smallest) entries are timed while the clocks still rise
+    warm = torch.randn(1 << 24, device=dev).to(torch.bfloat16)
+    warm_c = binding.Candidates([warm.clone() for _ in range(8)])
+    t_warm = time.perf_counter()
+    while time.perf_counter() - t_warm < 0.3:
+        for _ in range(20):
+            ctx.screen(warm, warm_c, 1e-2, 1.6e-2)
+        torch.cuda.synchronize()
+    del warm, warm_c
     for name, N in PAPER_SHAPES:
         for dname, tdt, idt in (("bf16", torch.bfloat16, torch.int16), ("f32", torch.float32, torch.int32)):
             esz = 2 if dname == "bf16" else 4
@@ -336,19 +346,22 @@ def run_paper_scale(args):
                      out.data_ptr(), int(torch.cuda.current_stream(dev).cuda_stream))
                 n0 = ctx.launch_count
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                # (ten times the calls for the tiny outputs: 20 calls of 5 us are over before the
+                # launch pipeline has filled)
+                n_calls = calls * 10 if (K + 1) * N * esz < (1 << 24) else calls
                 e0.record()
-                for _ in range(calls):
+                for _ in range(n_calls):
                     L.kb_screen(*a)
                 e1.record()
                 torch.cuda.synchronize()
-                us = e0.elapsed_time(e1) / calls * 1e3
+                us = e0.elapsed_time(e1) / n_calls * 1e3
                 assert ctx.poll() == 0
                 rec = binding.records(out)
                 gbs = (K + 1) * N * esz / (us * 1e-6) / 1e9
                 print(json.dumps({"benchmark": name, "N": N, "dtype": dname, "K": K, "us_per_call": us,
                                   "gbs": gbs, "frac_of_measured_hbm": gbs / peak,
-                                  "launches_per_call": (ctx.launch_count - n0) / calls,
-                                  "all_pass": bool((rec["pass"] == 1).all()), "calls": calls}), flush=True)
+                                  "launches_per_call": (ctx.launch_count - n0) / n_calls,
+                                  "all_pass": bool((rec["pass"] == 1).all()), "calls": n_calls}), flush=True)
             del ref
             cands = []
             torch.cuda.empty_cache()

@@ -839,7 +839,22 @@ kb_status screen_impl(kb_ctx* ctx, const void* d_ref, const void* const* h_cands
     PtrChunk ch;
     memcpy(ch.p, h_cands, K * sizeof(void*));
     dim3 grid((unsigned int)nb_small, K);
-    screen_small_kernel<DT><<<grid, 256, 0, st>>>(sm, ch);
+    cudaStreamCaptureStatus cap_small = cudaStreamCaptureStatusNone;
+    if (ctx->dependent_launch && cudaStreamIsCapturing(st, &cap_small) == cudaSuccess &&
+        cap_small == cudaStreamCaptureStatusNone) {
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = grid;
+      cfg.blockDim = dim3(256);
+      cfg.stream = st;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      attr[0].val.programmaticStreamSerializationAllowed = 1;
+      cfg.attrs = attr;
+      cfg.numAttrs = 1;
+      KB_CUDA(ctx, cudaLaunchKernelEx(&cfg, screen_small_kernel<DT>, sm, ch));
+    } else {
+      screen_small_kernel<DT><<<grid, 256, 0, st>>>(sm, ch);
+    }
     ++ctx->launches;
     KB_CUDA(ctx, cudaGetLastError());
     return KB_OK;

@@ -1087,6 +1087,12 @@ __device__ __forceinline__ void small_block(const void* ref, const void* cand, u
 
 template <int DT>
 __global__ void __launch_bounds__(256) screen_small_kernel(const SmallParams p, const PtrChunk cands) {
+  // Launched as a programmatic dependent of whatever precedes it in the stream (back-to-back
+  // calls: the next launch is set up while this one runs): let the next one be scheduled, then
+  // wait until the previous grid has finished and its writes are visible.  No effect when the
+  // launch carries no such attribute.
+  asm volatile("griddepcontrol.launch_dependents;");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const unsigned int k = blockIdx.y;
   small_block<DT>(p.ref, cands.p[k], p.N, (unsigned long long)blockIdx.x * kSmallPerBlock, p.mask,
                   p.atol, p.rtol, p.partials + (size_t)k * p.nb, blockIdx.x, p.nb, &p.tickets[k],
