@@ -144,7 +144,9 @@ template <bool E5M2> struct ElemF8 {
   }
   __device__ __forceinline__ static void pair_diff(const unsigned int* words, int e, float r0, float r1,
                                                    float& d0, float& d1) {
-    const unsigned int h2 = widen2((unsigned short)(words[e >> 2] >> (16 * ((e >> 1) & 1))));
+    // e5m2 is the high byte of binary16: a byte permute widens a pair (no conversion, no shift)
+    const unsigned int h2 = E5M2 ? __byte_perm(words[e >> 2], 0u, ((e >> 1) & 1) ? 0x3424u : 0x1404u)
+                                 : widen2((unsigned short)(words[e >> 2] >> (16 * ((e >> 1) & 1))));
     asm("{\n.reg .b16 lo, hi;\nmov.b32 {lo, hi}, %2;\nsub.rn.f32.f16 %0, lo, %3;\nsub.rn.f32.f16 %1, hi, %4;\n}"
         : "=f"(d0), "=f"(d1)
         : "r"(h2), "f"(r0), "f"(r1));
