@@ -32,15 +32,20 @@ kb_status kb_ctx_set_small_path(kb_ctx* ctx, int on);
  * while the stream is being captured into a graph.  Results do not depend on it. */
 kb_status kb_ctx_set_dependent_launch(kb_ctx* ctx, int on);
 
-/* Test/tuning hook: which instantiation of the streaming screen kernel runs.  0 = automatic
- * (the plain one, until a call reports that a quarter of its steps took a second look that
- * found nothing -- many elements whose quotient was rounded down to the largest relative
- * error, e.g. dense one-ulp differences -- then the one that applies the sharper test to
- * every element, with a plain call every 32 calls to see whether that still holds),
- * 1 = always plain, 2 = always sharp.  Results do not depend on it. */
+/* Test/tuning hook: which instantiation of the streaming screen kernel runs.  0 = automatic:
+ * the plain one, until a call reports that a quarter of its steps took a second look that
+ * found nothing.  If those looks came while the candidate was lean (many elements whose
+ * quotient was rounded down to the largest relative error, e.g. dense one-ulp differences)
+ * the next 32 calls use the SHARP instantiation, which applies the sharper test to every
+ * element; if they came beyond the lean bound (elements that pass by atol alone, e.g.
+ * candidates that differ by absolute noise where the reference is near zero) they use the BY
+ * DEFINITION instantiation, which there tests every element against its own tolerance.  A
+ * plain call every 32 calls checks whether the report still holds.
+ * 1 = always plain, 2 = always sharp, 3 = always by definition.  Results do not depend on it. */
 kb_status kb_ctx_set_filter(kb_ctx* ctx, int mode);
-/* Whether the last streaming launch of this context used the sharp instantiation (HOST out: 1 or 0). */
-kb_status kb_ctx_last_filter(const kb_ctx* ctx, int* sharp);
+/* The instantiation of this context's last streaming launch (HOST out): 0 plain, 1 sharp,
+ * 3 by definition. */
+kb_status kb_ctx_last_filter(const kb_ctx* ctx, int* mode);
 
 /* ---- instrumentation (used by the benchmark) ------------------------------ */
 

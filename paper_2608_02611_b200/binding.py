@@ -241,14 +241,21 @@ class Context:
         self._check(load().kb_ctx_set_dependent_launch(self._h, 1 if on else 0), "kb_ctx_set_dependent_launch")
 
     def set_filter(self, mode: int):
-        """0 automatic, 1 always the plain streaming kernel, 2 always the sharp one (a tuning hook)."""
+        """0 automatic, 1 always the plain streaming kernel, 2 always the sharp one, 3 always the
+        one that tests by the definition beyond the lean bound (a tuning hook)."""
         self._check(load().kb_ctx_set_filter(self._h, int(mode)), "kb_ctx_set_filter")
 
     @property
     def last_filter_sharp(self) -> bool:
+        """Whether the last streaming launch used another instantiation than the plain one."""
+        return self.last_filter_mode != 0
+
+    @property
+    def last_filter_mode(self) -> int:
+        """Instantiation of the last streaming launch: 0 plain, 1 sharp, 3 by definition."""
         v = ctypes.c_int(0)
         self._check(load().kb_ctx_last_filter(self._h, ctypes.byref(v)), "kb_ctx_last_filter")
-        return bool(v.value)
+        return int(v.value)
 
     def set_wins_algo(self, algo: int):
         """0 automatic, 1 direct comparison of all sample pairs, 2 binary search on sorted rows,

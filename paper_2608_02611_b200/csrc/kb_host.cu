@@ -43,10 +43,11 @@ struct kb_ctx {
   // so often one of them probes the plain one again.  filter_mode: 0 automatic, 1 plain, 2 sharp.
   unsigned int* h_hint = nullptr;   // pinned, mapped
   unsigned int* d_hint = nullptr;   // its device address
-  int filter_mode = 0;
+  int filter_mode = 0;              // 0 automatic, 1 plain, 2 sharp, 3 by definition
+  int alt_mode = 1;                 // the instantiation the automatic choice currently alternates with: 1 or 3
   int sharp_left = 0;
   bool sharp_probe_next = false, sharp_probed = false;
-  bool last_sharp = false;          // the last streaming launch used the sharp instantiation
+  int last_mode = 0;                // instantiation of the last streaming launch: 0 plain, 1 sharp, 3 by definition
   float call_steps = 0.0f;          // warp steps of the current call's plain streaming launch (0: none)
   float steps_hist[2] = {0.0f, 0.0f};   // the same for the last call on each accumulator set
   // [0] status, [1..3] counters of the binary64 gate, [4] effective K of an indexed call,
@@ -261,7 +262,9 @@ kb_status launch_stream(kb_ctx* ctx, StreamParams& sp, cudaStream_t st, bool beh
   // Plain until a plain launch reports that a quarter of its warp steps took a fruitless
   // second look; then sharp for kSharpCalls launches, one plain launch as a probe, sharp again
   // for the kSharpGrace launches its report needs to arrive, and the report decides.
-  bool sharp = ctx->filter_mode == 2 && !k8;
+  bool sharp = ctx->filter_mode >= 2 && !k8;     // "sharp": not the plain instantiation
+  if (ctx->filter_mode == 2) ctx->alt_mode = 1;
+  if (ctx->filter_mode == 3) ctx->alt_mode = 3;
   if (ctx->filter_mode == 0 && ctx->h_hint && !k8) {
     volatile unsigned int* hint = reinterpret_cast<volatile unsigned int*>(ctx->h_hint);
     if (ctx->sharp_left > 0) {
@@ -276,14 +279,22 @@ kb_status launch_stream(kb_ctx* ctx, StreamParams& sp, cudaStream_t st, bool beh
       ctx->sharp_probed = true;
       ctx->sharp_left = kSharpGrace;
       *hint = 0u;
-    } else if (*hint >= 16u) {                 // a quarter of the steps
-      sharp = true;
-      ctx->sharp_left = kSharpCalls - 1;
-      ctx->sharp_probed = false;
-      *hint = 0u;                              // the next plain launch reports afresh
+    } else {
+      // byte 0: second looks taken while lean, byte 1: fruitless looks beyond the lean bound,
+      // in 64ths of the reporting call's warp steps; a quarter of the steps decides
+      const unsigned int h = *hint;
+      const unsigned int lean_share = h & 0xFFu, atol_share = (h >> 8) & 0xFFu;
+      if (lean_share >= 16u || atol_share >= 16u) {
+        sharp = true;
+        ctx->alt_mode = atol_share > lean_share ? 3 : 1;
+        ctx->sharp_left = kSharpCalls - 1;
+        ctx->sharp_probed = false;
+        *hint = 0u;                            // the next plain launch reports afresh
+      }
     }
   }
-  ctx->last_sharp = sharp;
+  const int alt = ctx->alt_mode;
+  ctx->last_mode = sharp ? alt : 0;
   // warp steps of this launch if it counts its fruitless second looks (see LeadParams)
   ctx->call_steps = (sharp || k8) ? 0.0f : (float)sp.ntiles * (float)sp.K * (float)kWarps;
   {
@@ -291,9 +302,10 @@ kb_status launch_stream(kb_ctx* ctx, StreamParams& sp, cudaStream_t st, bool beh
     if constexpr (k8) {
       screen_stream8_kernel<DT><<<(unsigned int)grid, kThreads8, smem, st>>>(sp);
     } else {
-      if (sharp) {
+      const bool dependent = behind_lead && ctx->dependent_launch;
+      if (sharp && alt == 1) {
         screen_stream_kernel<DT, 1><<<(unsigned int)grid, kStreamThreads, smem, st>>>(sp);
-      } else if (behind_lead && ctx->dependent_launch) {
+      } else if (dependent) {
         // launch and set-up overlap the lead kernel (about 3 us per call)
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned int)grid);
@@ -305,7 +317,12 @@ kb_status launch_stream(kb_ctx* ctx, StreamParams& sp, cudaStream_t st, bool beh
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        KB_CUDA(ctx, cudaLaunchKernelEx(&cfg, screen_stream_kernel<DT, 2>, sp));
+        if (sharp)
+          KB_CUDA(ctx, cudaLaunchKernelEx(&cfg, screen_stream_kernel<DT, 3>, sp));
+        else
+          KB_CUDA(ctx, cudaLaunchKernelEx(&cfg, screen_stream_kernel<DT, 2>, sp));
+      } else if (sharp) {
+        screen_stream_kernel<DT, 3><<<(unsigned int)grid, kStreamThreads, smem, st>>>(sp);
       } else {
         screen_stream_kernel<DT, 0><<<(unsigned int)grid, kStreamThreads, smem, st>>>(sp);
       }
@@ -355,6 +372,11 @@ kb_status set_stream_attr(kb_ctx* ctx) {
     KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT, 2>,
                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT, 2>,
+                                      cudaFuncAttributePreferredSharedMemoryCarveout,
+                                      (int)cudaSharedmemCarveoutMaxShared));
+    KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT, 3>,
+                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    KB_CUDA(ctx, cudaFuncSetAttribute(screen_stream_kernel<DT, 3>,
                                       cudaFuncAttributePreferredSharedMemoryCarveout,
                                       (int)cudaSharedmemCarveoutMaxShared));
   }
@@ -519,7 +541,7 @@ extern "C" kb_status kb_ctx_set_grid(kb_ctx* ctx, uint32_t blocks) {
 }
 
 extern "C" kb_status kb_ctx_set_filter(kb_ctx* ctx, int mode) {
-  if (!ctx || mode < 0 || mode > 2) return KB_ERR_INVALID_ARG;
+  if (!ctx || mode < 0 || mode > 3) return KB_ERR_INVALID_ARG;
   ctx->filter_mode = mode;
   ctx->sharp_left = 0;
   ctx->sharp_probe_next = ctx->sharp_probed = false;
@@ -527,9 +549,9 @@ extern "C" kb_status kb_ctx_set_filter(kb_ctx* ctx, int mode) {
   return KB_OK;
 }
 
-extern "C" kb_status kb_ctx_last_filter(const kb_ctx* ctx, int* sharp) {
-  if (!ctx || !sharp) return KB_ERR_INVALID_ARG;
-  *sharp = ctx->last_sharp ? 1 : 0;
+extern "C" kb_status kb_ctx_last_filter(const kb_ctx* ctx, int* mode) {
+  if (!ctx || !mode) return KB_ERR_INVALID_ARG;
+  *mode = ctx->last_mode;
   return KB_OK;
 }
 

@@ -177,7 +177,7 @@ __host__ __device__ inline size_t stream_smem_bytes(uint32_t stages, uint32_t ti
 // ad <= rel*|r| <= RN(rtol*|r|) <= tol ("lean").  Beyond that the same loop runs with rel
 // clamped to that bound, and only threads for which it fails compare element by element.
 //
-// Two instantiations.  SHARP = false is the filter above with a second look for threads whose
+// Instantiations (MODE, below).  SHARP = false is the filter above with a second look for threads whose
 // (c) fails.  SHARP = true applies the second look's sharper test to every element in the main
 // loop (two dependent fused multiply-adds instead of one): a quarter more instructions per
 // step, but no second looks.  It pays when many elements have a quotient that was rounded DOWN
@@ -188,10 +188,18 @@ __host__ __device__ inline size_t stream_smem_bytes(uint32_t stages, uint32_t ti
 // host, which picks the instantiation from it.  The records do not depend on the choice.
 //
 // MODE 0: plain, 1: sharp, 2: plain, launched as a programmatic dependent of the lead kernel
-// (short calls: its CTAs are set up while the lead kernel still runs, and wait for it below).
+// (its CTAs are set up while the lead kernel still runs, and wait for it below), 3: "by
+// definition": the plain loop while a candidate is lean, and beyond the lean bound a loop that
+// tests every element against its own tolerance and the real running maximum, so that elements
+// that pass by atol alone (candidates that differ from the reference by absolute noise, where
+// the reference has values near zero) do not send their thread to a second look every step.
+// The plain instantiations count such fruitless looks beside the lean ones; the host picks 3
+// from that report the way it picks 1.  Mode 3 waits for the lead kernel like mode 2.
 template <int DT, int MODE>
 __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
   constexpr bool SHARP = MODE == 1;
+  constexpr bool BYDEF = MODE == 3;
+  constexpr bool PLAIN = MODE == 0 || MODE == 2;
   using E = Elem<DT>;
   constexpr int VEC = E::kVec;
   constexpr int NV = kEPT / VEC;
@@ -255,7 +263,7 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
   for (int i = tid; i < kMaxKC * kWarps; i += kStreamThreads) s.thr2[i] = make_float2(-1.0f, 0.0f);
   __syncthreads();
   // everything the lead kernel wrote (pointer table, seeds, zeroed counters) is read below
-  if constexpr (MODE == 2) asm volatile("griddepcontrol.wait;" ::: "memory");
+  if constexpr (MODE == 2 || MODE == 3) asm volatile("griddepcontrol.wait;" ::: "memory");
 
   // Work items (chunk, tile), chunk-major, are drawn from a global counter: a CTA gets
   // ascending items (so ascending tiles inside a chunk, which the index tie-break needs),
@@ -369,7 +377,7 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
         if ((v = s.key[i]) != 0ull) atomicMax(&a->key, v);
         unsigned int r = s.rel[i];
         if (r != 0u) atomicMax(&a->rel, r);
-        if (!SHARP && (v = s.cnt[3 * kMaxKC + i]) != 0ull) atomicAdd(&a->spare, v);
+        if (PLAIN && (v = s.cnt[3 * kMaxKC + i]) != 0ull) atomicAdd(&a->spare, v);
         s.cnt[3 * kMaxKC + i] = 0ull;
         s.cnt[i] = 0ull;
         s.cnt[kMaxKC + i] = 0ull;
@@ -538,7 +546,23 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
                      : 0.0f;
         };
         const bool sharp = SHARP && lean;
-        if (!SHARP || !sharp) {
+        if (BYDEF && has_lean && !lean) {
+          // every element within its own tolerance (|d| - tol <= 0, tol rounded as the definition
+          // rounds it; a NaN or Inf difference makes the difference NaN) and no quotient above
+          // the real running maximum: twice the arithmetic of the clamped test below
+#pragma unroll
+          for (int e = 0; e < kEPT; e += 2) {
+            float d0, d1;
+            E::pair_diff(words, e, r[e], r[e + 1], d0, d1);
+            const float ar0 = fabsf(r[e]), ar1 = fabsf(r[e + 1]);
+            const float w0 = __fsub_rn(fabsf(d0), __fadd_rn(p.atol, __fmul_rn(p.rtol, ar0)));
+            const float w1 = __fsub_rn(fabsf(d1), __fadd_rn(p.atol, __fmul_rn(p.rtol, ar1)));
+            const float t0 = fmaf(-rel, ar0, fabsf(d0)), t1 = fmaf(-rel, ar1, fabsf(d1));
+            mabs = max3(mabs, fabsf(d0), fabsf(d1));
+            mrel = max3_nan(mrel, w0, t0);
+            mrel = max3_nan(mrel, w1, t1);
+          }
+        } else if (!SHARP || !sharp) {
 #pragma unroll
           for (int e = 0; e < kEPT; e += 2) {
             float d0, d1;
@@ -632,7 +656,10 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
           // (some lane was `bad`, or the step would have ended above: while lean that lane took
           // a second look, and it found nothing)
           // (32-bit add on the low word of the 64-bit slot; flush() moves it to the accumulator)
-          if (!SHARP && lane == 0 && lean) atomicAdd(reinterpret_cast<unsigned int*>(&s.cnt[3 * kMaxKC + kk]), 1u);
+          // (low word: looks taken while lean; high word: looks beyond the lean bound that found
+          // no mismatch either, i.e. the thread's elements pass by atol)
+          if (PLAIN && lane == 0 && (lean || tot == 0u))
+            atomicAdd(reinterpret_cast<unsigned int*>(&s.cnt[3 * kMaxKC + kk]) + (lean ? 0 : 1), 1u);
           continue;
         }
 
@@ -876,9 +903,14 @@ __global__ void __launch_bounds__(256) screen_lead_kernel(const LeadParams p, co
     if (k == 0 && threadIdx.x < 3) p.counters_next[threadIdx.x] = 0u;
     if (k == 0 && threadIdx.x == 32 && p.hint) {
       // (only plain launches report: the word keeps the last report until the host takes it)
-      if (p.pub_steps > 0.0f)
-        *reinterpret_cast<volatile unsigned int*>(p.hint) =
-            (unsigned int)fminf(64.0f * (float)*p.looks_pub / p.pub_steps, 64.0f);
+      if (p.pub_steps > 0.0f) {
+        // byte 0: looks taken while lean, byte 1: fruitless looks beyond the lean bound, each as
+        // 64ths of the call's warp steps
+        const unsigned long long looks = *p.looks_pub;
+        const unsigned int lean_share = (unsigned int)fminf(64.0f * (float)(looks & 0xFFFFFFFFull) / p.pub_steps, 64.0f);
+        const unsigned int atol_share = (unsigned int)fminf(64.0f * (float)(looks >> 32) / p.pub_steps, 64.0f);
+        *reinterpret_cast<volatile unsigned int*>(p.hint) = lean_share | (atol_share << 8);
+      }
       *p.looks_pub = 0ull;
     }
   }

@@ -107,9 +107,15 @@ def run_screen(ctx, kb, ref, cands, atol, rtol, mask_spec=None, N=None):
         rec = kb.records(ctx.screen(ref, cands, atol, rtol, mask))
         ctx.set_dependent_launch(False)
         rec_plain = kb.records(ctx.screen(ref, cands, atol, rtol, mask))
+        ctx.set_dependent_launch(True)
+        for mode in (2, 3):                 # the sharp and the by-definition instantiation
+            ctx.set_filter(mode)
+            rec_mode = kb.records(ctx.screen(ref, cands, atol, rtol, mask))
+            assert rec.tobytes() == rec_mode.tobytes(), f"filter mode {mode}"
     finally:
         ctx.set_small_path(True)
         ctx.set_dependent_launch(True)
+        ctx.set_filter(0)
     rec_small = kb.records(ctx.screen(ref, cands, atol, rtol, mask))
     assert ctx.poll() == 0
     assert rec.tobytes() == rec_small.tobytes()

@@ -120,10 +120,12 @@ def one_case(ctx, kb, seed, log2_lo, log2_hi):
         try:
             ctx.set_grid(grid)
             ctx.set_small_path(small)
+            ctx.set_filter(int(rng.integers(0, 4)))      # automatic, plain, sharp or by definition
             got = kb.records(ctx.screen(ref.to(dev), [c.to(dev) for c in cands], atol, rtol, mk))
         finally:
             ctx.set_grid(0)
             ctx.set_small_path(True)
+            ctx.set_filter(0)
         want = oracle.screen(synth.to_oracle_array(ref, code), [synth.to_oracle_array(c, code) for c in cands],
                              code, atol, rtol, mask_spec, threads=8)
     assert ctx.poll() == 0

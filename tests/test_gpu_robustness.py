@@ -369,18 +369,60 @@ def test_sharp_filter_is_chosen_for_dense_rounded_down_quotients_and_changes_not
     for mode in (1, 2):                               # forced plain, forced sharp
         ctx.set_filter(mode)
         same_records(kb.records(ctx.screen(ref, dense, 1e-2, 1.6e-2)), want_dense)
-        assert ctx.last_filter_sharp == (mode == 2)
+        assert ctx.last_filter_mode == (1 if mode == 2 else 0)
         same_records(kb.records(ctx.screen(ref, sparse, 1e-2, 1.6e-2)), want_sparse)
     ctx.set_filter(0)                                 # automatic
     seen = []
     for _ in range(8):
         same_records(kb.records(ctx.screen(ref, dense, 1e-2, 1.6e-2)), want_dense)    # (synchronises)
-        seen.append(ctx.last_filter_sharp)
-    assert not seen[0] and seen[-1], seen             # plain first, sharp once the reports are in
+        seen.append(ctx.last_filter_mode)
+    assert seen[0] == 0 and seen[-1] == 1, seen       # plain first, sharp once the reports are in
     ctx.set_filter(0)                                 # forget
     for _ in range(8):
         same_records(kb.records(ctx.screen(ref, sparse, 1e-2, 1.6e-2)), want_sparse)
         assert not ctx.last_filter_sharp
+    assert ctx.poll() == 0
+
+
+@pytest.mark.parametrize("dtype", [synth.BF16, synth.F16, synth.F32])
+def test_by_definition_filter_is_chosen_for_absolute_noise_and_changes_nothing(ctx, kb, dtype):
+    """Candidates that differ from the reference by absolute noise: where the reference is near
+    zero the relative error is far above rtol and the element passes by atol alone.  The plain
+    filter then sends nearly every step to a fruitless second look; after a few calls the
+    context switches to the instantiation that tests such steps by the definition.  Same
+    records in every mode, for passing and for failing candidates."""
+    dev = torch.device("cuda", 0)
+    ctx.set_small_path(False)
+    g = torch.Generator(device=dev)
+    g.manual_seed(17 + dtype)
+    tdt = synth.TORCH_DTYPE[dtype]
+    N = 150 * 4096 + 901
+    base = torch.randn(N, device=dev, generator=g) * 4
+    ref = base.to(tdt)
+    sigma, atol, rtol = {synth.BF16: (1e-3, 1e-2, 1.6e-2), synth.F16: (1e-4, 1e-3, 1e-2),
+                         synth.F32: (1e-6, 1e-5, 1e-6)}[dtype]
+    noisy = [(base + torch.randn(N, device=dev, generator=g) * sigma).to(tdt) for _ in range(6)]
+    failing = [(base + torch.randn(N, device=dev, generator=g) * (30 * sigma)).to(tdt) for _ in range(3)]
+    failing[1][5] = float("nan")
+    failing[2][N - 1] = float("inf")
+    want = oracle_records(dtype, ref, noisy, atol, rtol)
+    want_fail = oracle_records(dtype, ref, failing, atol, rtol)
+    assert (want["pass"] == 1).all() and (want["max_rel_err"] > rtol).all()
+    assert (want_fail["pass"] == 0).all()
+    for mode in (1, 2, 3):                            # forced plain, sharp, by definition
+        ctx.set_filter(mode)
+        same_records(kb.records(ctx.screen(ref, noisy, atol, rtol)), want)
+        assert ctx.last_filter_mode == {1: 0, 2: 1, 3: 3}[mode]
+        same_records(kb.records(ctx.screen(ref, failing, atol, rtol)), want_fail)
+        same_records(kb.records(ctx.screen(ref, noisy + failing, atol, rtol)), np.concatenate([want, want_fail]))
+    ctx.set_filter(0)                                 # automatic
+    seen = []
+    for _ in range(8):
+        same_records(kb.records(ctx.screen(ref, noisy, atol, rtol)), want)
+        seen.append(ctx.last_filter_mode)
+    assert seen[0] == 0 and seen[-1] == 3, seen       # plain first, by definition once the reports are in
+    ctx.set_filter(0)
+    ctx.set_small_path(True)
     assert ctx.poll() == 0
 
 
