@@ -546,22 +546,29 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
                      : 0.0f;
         };
         const bool sharp = SHARP && lean;
+        float mtol = -kInf;   // (by definition only) largest |d| - rtol_lean*|r| of the thread
         if (BYDEF && has_lean && !lean) {
-          // every element within its own tolerance (|d| - tol <= 0, tol rounded as the definition
-          // rounds it; a NaN or Inf difference makes the difference NaN) and no quotient above
-          // the real running maximum: twice the arithmetic of the clamped test below
+          // Beyond the lean bound: no quotient above the REAL running maximum (t <= 0 as in the
+          // lean form) and every element within tolerance by a sufficient test,
+          //   RN(|d| - rtol_lean*|r|) <= atol*(1 - 2^-20)   =>   |d| <= RN(atol + RN(rtol*|r|)):
+          // the left side is one fused multiply-add, so |d| <= atol_d*(1 + 2^-24) + rtol_lean*|r|
+          // <= (atol + rtol*|r|)*(1 - 2^-21), below the definition's twice-rounded tolerance
+          // (rtol*|r| >= 2^-120 is normal here: rtol >= 2^-20, |r| >= 2^-100 or the thread is
+          // `extreme`; |r| = 0 leaves |d| <= atol_d).  NaN and Inf differences make it NaN or
+          // Inf.  An element within 2^-20 of its tolerance is flagged and settled by the second look.
 #pragma unroll
           for (int e = 0; e < kEPT; e += 2) {
             float d0, d1;
             E::pair_diff(words, e, r[e], r[e + 1], d0, d1);
             const float ar0 = fabsf(r[e]), ar1 = fabsf(r[e + 1]);
-            const float w0 = __fsub_rn(fabsf(d0), __fadd_rn(p.atol, __fmul_rn(p.rtol, ar0)));
-            const float w1 = __fsub_rn(fabsf(d1), __fadd_rn(p.atol, __fmul_rn(p.rtol, ar1)));
+            const float u0 = fmaf(-p.rtol_lean, ar0, fabsf(d0)), u1 = fmaf(-p.rtol_lean, ar1, fabsf(d1));
             const float t0 = fmaf(-rel, ar0, fabsf(d0)), t1 = fmaf(-rel, ar1, fabsf(d1));
             mabs = max3(mabs, fabsf(d0), fabsf(d1));
-            mrel = max3_nan(mrel, w0, t0);
-            mrel = max3_nan(mrel, w1, t1);
+            mtol = max3_nan(mtol, u0, u1);
+            mrel = max3_nan(mrel, t0, t1);
           }
+          // (folded into the relative test's flag: positive, or NaN, when some element may be out of tolerance)
+          mrel = max2_nan(mrel, __fsub_rn(mtol, p.atol * 0.99999904632568359375f));
         } else if (!SHARP || !sharp) {
 #pragma unroll
           for (int e = 0; e < kEPT; e += 2) {

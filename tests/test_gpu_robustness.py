@@ -426,6 +426,40 @@ def test_by_definition_filter_is_chosen_for_absolute_noise_and_changes_nothing(c
     assert ctx.poll() == 0
 
 
+def test_by_definition_filter_at_the_edge_of_the_tolerance(ctx, kb):
+    """Beyond the lean bound the by-definition instantiation tests |d| <= tol by a sufficient
+    condition with a margin of 2^-20: elements whose error EQUALS the tolerance, or misses it by
+    one unit in the last place either way, must come out as the definition says."""
+    dev = torch.device("cuda", 0)
+    ctx.set_small_path(False)
+    rng = np.random.default_rng(2025)
+    N = 40 * 4096 + 5
+    atol, rtol = np.float32(2.0 ** -10), np.float32(2.0 ** -6)
+    r = (rng.integers(1, 1 << 12, N).astype(np.float32) / np.float32(256.0))        # multiples of 2^-8 below 16
+    r[::7] = np.float32(2.0 ** -12)                       # tiny references ...
+    tol = (atol + (rtol * np.abs(r)).astype(np.float32)).astype(np.float32)          # exact here: dyadic values
+    cands = []
+    for shift in (0, 1, -1):                              # error = tol, one ulp above, one ulp below
+        c = (r + tol).astype(np.float32)
+        assert ((c - r).astype(np.float32) == tol).all()
+        if shift:
+            c = np.nextafter(c, np.float32(np.inf if shift > 0 else -np.inf), dtype=np.float32)
+        c[::7] = r[::7] + np.float32(2.0 ** -11)          # ... whose error passes by atol with a quotient of 2
+        cands.append(c)
+    ref_t = torch.from_numpy(r).to(dev)
+    cand_t = [torch.from_numpy(c).to(dev) for c in cands]
+    want = oracle.screen(r, cands, oracle.F32, float(atol), float(rtol), threads=THREADS)
+    assert want["pass"][0] == 1 and want["pass"][2] == 1 and want["pass"][1] == 0
+    assert want["mismatch_count"][1] == N - len(r[::7]) and (want["max_rel_err"] == 2.0).all()
+    for mode in (1, 2, 3, 0):
+        ctx.set_filter(mode)
+        for _ in range(3):
+            same_records(kb.records(ctx.screen(ref_t, cand_t, float(atol), float(rtol))), want)
+    ctx.set_filter(0)
+    ctx.set_small_path(True)
+    assert ctx.poll() == 0
+
+
 # ---------------------------------------------------------------------------------------------
 # out-of-range READS: every input tensor sits between two halos of NaN patterns (all-ones bytes
 # are NaN in all six storage types).  An element read from outside [0, N) as a candidate would
