@@ -239,12 +239,20 @@ def run_screen(args):
     idt = {8: torch.int64, 4: torch.int32, 2: torch.int16, 1: torch.int8}[torch.empty(0, dtype=tdt).element_size()]
     g = torch.Generator(device=dev)
     g.manual_seed(20260802)
-    ref = torch.randn(N, dtype=torch.float32, device=dev, generator=g).to(tdt)
+    base = torch.randn(N, dtype=torch.float32, device=dev, generator=g) * args.ref_scale
+    ref = (torch.relu(base) if args.relu else base).to(tdt)   # (noise goes in before the rectifier)
     esz1 = ref.element_size() == 1           # 8-bit floats: one unit in the last place is up to 1/8
     cands = []
     for _ in range(K):
+        if args.noise_sigma > 0.0:
+            # accumulated rounding error does not scale with the value: where the reference is near
+            # zero the relative error is large and the element passes by atol alone
+            c = base + torch.randn(N, dtype=torch.float32, device=dev, generator=g) * args.noise_sigma
+            cands.append((torch.relu(c) if args.relu else c).to(tdt))
+            continue
         flip = torch.rand(N, device=dev, generator=g) < args.flip_frac
         cands.append(torch.where(flip, ref.view(idt) + 1, ref.view(idt)).view(tdt))
+    del base
     # tolerances under which a one-ulp difference passes: 2^-3 relative in e4m3, 2^-2 in e5m2
     atol, rtol = (1e-12, 1e-12) if args.dtype == "f64" else \
         (1e-2, 0.26 if args.dtype == "e5m2" else 0.13) if esz1 else (1e-2, 1.6e-2)
@@ -252,6 +260,8 @@ def run_screen(args):
     call = (lambda: ctx.screen_f64(ref, cands, atol, rtol)) if args.dtype == "f64" else \
         (lambda: ctx.screen(ref, held, atol, rtol))
     steps, warmup = max(1, min(args.steps, 50)), max(3, args.warmup)
+    if args.noise_sigma > 0.0:
+        warmup = max(warmup, 12)       # the context's choice of instantiation follows its reports
     for _ in range(warmup):
         call()
     torch.cuda.synchronize()
@@ -271,8 +281,11 @@ def run_screen(args):
     esz = ref.element_size()
     stream_bytes = (K + 1) * (ntiles - nscout) * 4096 * esz
     peak, src = peaks()
-    line = {"workload": f"screen K={K} N=2^{args.log2n} {args.dtype}, one-ulp differences on "
-                        f"{args.flip_frac:.0%} of the elements",
+    what = (f"absolute noise sigma={args.noise_sigma:g} on a reference of scale {args.ref_scale:g}"
+            + (", rectified" if args.relu else "")) if args.noise_sigma > 0.0 else \
+        f"one-ulp differences on {args.flip_frac:.0%} of the elements"
+    line = {"workload": f"screen K={K} N=2^{args.log2n} {args.dtype}, {what}",
+            "filter": {0: "plain", 1: "sharp", 3: "by definition"}.get(ctx.last_filter_mode, "-"),
             "ms_per_call": ms, "stream_kernel_ms": k_ms, "steps": steps,
             "call_gbs": (K + 1) * N * esz / (ms * 1e-3) / 1e9,
             "roofline": {"bound": "hbm", "achieved": stream_bytes / (k_ms * 1e-3) / 1e9, "peak": peak,
@@ -401,6 +414,10 @@ def main():
                     help="storage type of the 'screen' workload")
     ap.add_argument("--log2n", type=int, default=24, help="elements per tensor of the 'screen' workload")
     ap.add_argument("--flip-frac", type=float, default=0.25)
+    ap.add_argument("--noise-sigma", type=float, default=0.0,
+                    help="'screen' workload: candidates = round(reference + N(0, sigma^2)) instead of one-ulp differences")
+    ap.add_argument("--ref-scale", type=float, default=1.0, help="'screen' workload: standard deviation of the reference")
+    ap.add_argument("--relu", action="store_true", help="'screen' workload: rectified reference and candidates")
     ap.add_argument("--default-dispatch", action="store_true",
                     help="'screen' workload: let small problems take the single-launch kernel")
     ap.add_argument("--K", type=int, default=512)

@@ -622,7 +622,7 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
           // (A failure that is large against the thread's errors is a real new maximum: no
           // need to look.  An element of the kind above fails by 2^-24 of its error at most.
           // In the sharp instantiation the look has been taken already.)
-          bool again = sharp || !(mrel <= mabs * 9.5367431640625e-07f);
+          bool again = sharp || (!BYDEF && !(mrel <= mabs * 9.5367431640625e-07f));
           if (!again) {
 #pragma unroll
           for (int e = 0; e < kEPT; e += 2) {
@@ -631,8 +631,14 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
             const float ar0 = fabsf(r[e]), ar1 = fabsf(r[e + 1]);
             const float t0 = fmaf(-rel, ar0, fabsf(d0)), t1 = fmaf(-rel, ar1, fabsf(d1));
             // (a NaN or Inf difference makes t NaN or Inf: neither clause holds)
-            const bool c0 = (t0 <= 0.0f) || (t0 >= 7.888609052e-31f && fmaf(-g, ar0, t0) <= 0.0f);
-            const bool c1 = (t1 <= 0.0f) || (t1 >= 7.888609052e-31f && fmaf(-g, ar1, t1) <= 0.0f);
+            // (by definition only: a zero reference has no quotient, its element only has to be
+            // within atol.  In the other instantiations such an element goes to the exact path;
+            // the clause is kept out of them because it changes how the compiler lays out their
+            // main loop.)
+            const bool c0 = (t0 <= 0.0f) || (t0 >= 7.888609052e-31f && fmaf(-g, ar0, t0) <= 0.0f) ||
+                            (BYDEF && ar0 == 0.0f && fabsf(d0) <= p.atol);
+            const bool c1 = (t1 <= 0.0f) || (t1 >= 7.888609052e-31f && fmaf(-g, ar1, t1) <= 0.0f) ||
+                            (BYDEF && ar1 == 0.0f && fabsf(d1) <= p.atol);
             again |= !c0 || !c1;
           }
           }
@@ -651,7 +657,9 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
             const float tol1 = __fadd_rn(p.atol, __fmul_rn(p.rtol, fabsf(r[e + 1])));
             const bool f0 = a0 <= kFltMax, f1 = a1 <= kFltMax;
             again |= !f0 || !f1;
-            again |= !(fmaf(-rel, fabsf(r[e]), a0) <= 0.0f) || !(fmaf(-rel, fabsf(r[e + 1]), a1) <= 0.0f);
+            // (by definition only: a zero reference has no quotient)
+            again |= ((!BYDEF || fabsf(r[e]) > 0.0f) && !(fmaf(-rel, fabsf(r[e]), a0) <= 0.0f)) ||
+                     ((!BYDEF || fabsf(r[e + 1]) > 0.0f) && !(fmaf(-rel, fabsf(r[e + 1]), a1) <= 0.0f));
             mis_fast += ((a0 > tol0) && f0) ? 1u : 0u;   // (c == r would give a0 = 0 <= tol0)
             mis_fast += ((a1 > tol1) && f1) ? 1u : 0u;
           }
