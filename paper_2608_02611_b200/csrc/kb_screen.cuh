@@ -745,6 +745,11 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
             atomicMax(&s.rel[kk], qb);
 #pragma unroll
             for (int w2 = 0; w2 < kWarps; ++w2) atomicMax(row + 2 * w2 + 1, (int)qb);
+          } else if (PLAIN && best == 0ull && (n_mis | n_nan | n_inf) == 0u) {
+            // an exact path that changed nothing (typically a zero reference under a non-zero
+            // candidate within atol, which has no quotient): reported with the fruitless looks
+            // beyond the lean bound, since the by-definition instantiation settles those earlier
+            atomicAdd(reinterpret_cast<unsigned int*>(&s.cnt[3 * kMaxKC + kk]) + 1, 1u);
           }
         }
         __syncwarp();
