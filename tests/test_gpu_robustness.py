@@ -426,6 +426,39 @@ def test_by_definition_filter_is_chosen_for_absolute_noise_and_changes_nothing(c
     assert ctx.poll() == 0
 
 
+def test_by_definition_filter_is_chosen_for_nonzero_candidates_under_zero_references(ctx, kb):
+    """A rectified reference (half of it exactly zero) and candidates that are tiny but not zero
+    there: such elements have no quotient, the relative test cannot pass them, and in the plain
+    instantiation every step ends in an exact path that changes nothing.  Those are reported and
+    the context moves to the by-definition instantiation; one candidate is too large under a
+    zero reference and must be counted out exactly as the oracle says, in every mode."""
+    dev = torch.device("cuda", 0)
+    ctx.set_small_path(False)
+    g = torch.Generator(device=dev)
+    g.manual_seed(99)
+    N = 120 * 4096 + 13
+    ref = torch.relu(torch.randn(N, device=dev, generator=g) * 4).to(torch.bfloat16)
+    cands = []
+    for k in range(5):
+        tiny = (torch.rand(N, device=dev, generator=g) * (3e-2 if k == 4 else 1e-4)).to(torch.bfloat16)
+        cands.append(torch.where(ref == 0, tiny, ref))
+    want = oracle_records(synth.BF16, ref, cands, 1e-2, 1.6e-2)
+    assert list(want["pass"]) == [1, 1, 1, 1, 0] and want["mismatch_count"][4] > 1000
+    assert (want["max_rel_err"] == 0).all()               # no element with a non-zero reference differs
+    for mode in (1, 2, 3):
+        ctx.set_filter(mode)
+        same_records(kb.records(ctx.screen(ref, cands, 1e-2, 1.6e-2)), want)
+    ctx.set_filter(0)
+    seen = []
+    for _ in range(8):
+        same_records(kb.records(ctx.screen(ref, cands[:4], 1e-2, 1.6e-2)), want[:4])
+        seen.append(ctx.last_filter_mode)
+    assert seen[0] == 0 and seen[-1] == 3, seen
+    ctx.set_filter(0)
+    ctx.set_small_path(True)
+    assert ctx.poll() == 0
+
+
 def test_by_definition_filter_at_the_edge_of_the_tolerance(ctx, kb):
     """Beyond the lean bound the by-definition instantiation tests |d| <= tol by a sufficient
     condition with a margin of 2^-20: elements whose error EQUALS the tolerance, or misses it by
