@@ -483,6 +483,7 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
       float r[kEPT];
       bool extreme = false;   // 0 < |r| < 2^-100: the fused multiply-add of the filter could
                               // underflow to zero and lose its sign; such threads go exact
+      float rlim = 0.0f;      // (by definition only: extreme in a step iff 0 < rel_f < rlim)
       {
         const uint4* src = reinterpret_cast<const uint4*>(s.buf + (size_t)stage * TILE_BYTES);
         uint4 w[NV];
@@ -498,9 +499,21 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
         for (int j = 0; j < NV; ++j) E::decode(w[j], &r[j * VEC]);
         // (binary16 and e5m2 have no value in (0, 2^-100): their smallest are 2^-24 and 2^-16)
         if constexpr (DT != KB_F16 && DT != KB_F8E5M2) {
+          if constexpr (BYDEF) {
+            // By definition: the same danger, judged per step.  The fused multiply-add can only
+            // mislead if rel_f*|r| < 2^-125 (see above), so with the thread's smallest non-zero
+            // magnitude m the thread is extreme in a step iff 0 < rel_f < 2^-124/m.  Outputs
+            // with long tails of tiny values (a softmax over widely spread logits) then leave
+            // the filter only while the running maximum is still tiny itself.
+            unsigned int umin = 0xFFFFFFFFu;
 #pragma unroll
-          for (int e = 0; e < kEPT; ++e)   // 0 < |r| < 2^-100 on the bit pattern (zero wraps to the top)
-            extreme |= ((__float_as_uint(r[e]) & 0x7FFFFFFFu) - 1u) < (0x0D800000u - 1u);
+            for (int e = 0; e < kEPT; ++e) umin = min(umin, (__float_as_uint(r[e]) & 0x7FFFFFFFu) - 1u);
+            if (umin < 0x0D800000u - 1u) rlim = __fdiv_ru(4.70197740328915e-38f, __uint_as_float(umin + 1u));
+          } else {
+#pragma unroll
+            for (int e = 0; e < kEPT; ++e)   // 0 < |r| < 2^-100 on the bit pattern (zero wraps to the top)
+              extreme |= ((__float_as_uint(r[e]) & 0x7FFFFFFFu) - 1u) < (0x0D800000u - 1u);
+          }
         }
       }
       if (first_of_chunk) exchange_apply(tile_base);
@@ -537,6 +550,7 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
         const bool has_lean = p.rtol_lean >= 0.0f;
         const bool lean = rel <= p.rtol_lean;
         const float rel_f = (has_lean && !lean) ? p.rtol_lean : rel;
+        const bool ext = BYDEF ? (rel_f > 0.0f && rel_f < rlim) : extreme;
         float mabs = 0.0f, mrel = 0.0f;
         // g = (ulp(rel)/2)*(1 - 2^-20), or 0 where that would be subnormal
         auto half_ulp_of_rel = [&]() -> float {
@@ -553,8 +567,8 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
           //   RN(|d| - rtol_lean*|r|) <= atol*(1 - 2^-20)   =>   |d| <= RN(atol + RN(rtol*|r|)):
           // the left side is one fused multiply-add, so |d| <= atol_d*(1 + 2^-24) + rtol_lean*|r|
           // <= (atol + rtol*|r|)*(1 - 2^-21), below the definition's twice-rounded tolerance
-          // (rtol*|r| >= 2^-120 is normal here: rtol >= 2^-20, |r| >= 2^-100 or the thread is
-          // `extreme`; |r| = 0 leaves |d| <= atol_d).  NaN and Inf differences make it NaN or
+          // (rtol_lean*|r| >= 2^-124 is normal for every non-zero |r| of a thread that is not
+          // extreme in this step; |r| = 0 leaves |d| <= atol_d).  NaN and Inf differences make it NaN or
           // Inf.  An element within 2^-20 of its tolerance is flagged and settled by the second look.
 #pragma unroll
           for (int e = 0; e < kEPT; e += 2) {
@@ -600,7 +614,7 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
         // A thread whose (c) fails, or (no lean bound) whose largest error exceeds atol, looks
         // again element by element below before its warp is sent down the exact path.
         const bool bad = !(mrel <= 0.0f) || (!has_lean && mabs > p.atol);
-        bool trig = (mabs > th) || extreme;
+        bool trig = (mabs > th) || ext;
         // Every vote below is reached by all 32 lanes: no warp-synchronous call sits under a
         // condition that could differ between lanes.
         if (!__any_sync(0xFFFFFFFFu, trig || bad)) continue;
@@ -699,7 +713,10 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
               m = ad;
               mi = e;
             }
-            bool hot = !(t <= 0.0f) || !fin || extreme;
+            // (by definition: only the elements the danger is about, rel_f*|r| < 2^-124, are
+            // evaluated unconditionally; the thread's other elements have a reliable t)
+            const bool ext_e = BYDEF ? (ext && ar * rel_f < 4.70197740328915e-38f) : ext;
+            bool hot = !(t <= 0.0f) || !fin || ext_e;
             if (!lean) hot = hot || !(ad <= __fadd_rn(p.atol, __fmul_rn(p.rtol, ar)));
             if (hot) {
               const float tol = __fadd_rn(p.atol, __fmul_rn(p.rtol, ar));
@@ -707,7 +724,7 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
               n_mis += match ? 0u : 1u;
               n_nan += (c[e] != c[e]) ? 1u : 0u;
               n_inf += (fabsf(c[e]) == kInf) ? 1u : 0u;
-              if (fin && ar > 0.0f && ar <= kFltMax && (extreme || t > 0.0f)) {
+              if (fin && ar > 0.0f && ar <= kFltMax && (ext_e || t > 0.0f)) {
                 const unsigned int q = __float_as_uint(__fdiv_rn(ad, ar));
                 qb = q > qb ? q : qb;
               }

@@ -459,6 +459,37 @@ def test_by_definition_filter_is_chosen_for_nonzero_candidates_under_zero_refere
     assert ctx.poll() == 0
 
 
+@pytest.mark.parametrize("dtype", [synth.F32, synth.BF16])
+def test_outputs_with_long_tails_of_tiny_values(ctx, kb, dtype):
+    """A softmax over widely spread logits: thousands of outputs below 2^-100, some subnormal,
+    some zero.  Threads that hold such values leave the filter in the plain instantiation; the
+    by-definition one judges the danger per step from the running maximum.  Same records in
+    every mode; tiny values are exactly where a missed maximum of the relative error would hide."""
+    dev = torch.device("cuda", 0)
+    ctx.set_small_path(False)
+    g = torch.Generator(device=dev)
+    g.manual_seed(41 + dtype)
+    tdt = synth.TORCH_DTYPE[dtype]
+    rows, cols = 48, 8192
+    atol, rtol = (1e-6, 1e-3) if dtype == synth.F32 else (1e-3, 1.6e-2)
+    cands, refs = [], None
+    for spread in (10.0, 25.0):
+        logits = torch.randn(rows, cols, device=dev, generator=g) * spread
+        ref = torch.softmax(logits, dim=1).reshape(-1).to(tdt)
+        assert int(((ref.float() > 0) & (ref.float() < 7.8e-31)).sum()) > 200
+        cs = [torch.softmax(logits + torch.randn(rows, cols, device=dev, generator=g) * 1e-4, dim=1).reshape(-1).to(tdt)
+              for _ in range(4)]
+        cs.append(torch.where(ref.float() < 1e-33, ref * 2, ref))            # tiny values doubled: quotient 1
+        cs.append(torch.where(ref.float() < 1e-36, torch.zeros_like(ref), ref))   # ... flushed to zero
+        want = oracle_records(dtype, ref, cs, atol, rtol)
+        for mode in (1, 2, 3, 0, 0, 0, 0, 0, 0):
+            ctx.set_filter(mode) if mode else None
+            same_records(kb.records(ctx.screen(ref, cs, atol, rtol)), want)
+        ctx.set_filter(0)
+    ctx.set_small_path(True)
+    assert ctx.poll() == 0
+
+
 def test_by_definition_filter_at_the_edge_of_the_tolerance(ctx, kb):
     """Beyond the lean bound the by-definition instantiation tests |d| <= tol by a sufficient
     condition with a margin of 2^-20: elements whose error EQUALS the tolerance, or misses it by
