@@ -613,8 +613,13 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
         // again element by element below before its warp is sent down the exact path.
         // A thread whose (c) fails, or (no lean bound) whose largest error exceeds atol, looks
         // again element by element below before its warp is sent down the exact path.
-        const bool bad = !(mrel <= 0.0f) || (!has_lean && mabs > p.atol);
-        bool trig = (mabs > th) || ext;
+        // (by definition: an extreme thread takes the second look, which tests its tiny elements
+        // with both operands scaled by 2^64 so that the fused multiply-add cannot underflow.  A
+        // tiny element whose quotient is fine also matches, given atol >= 2^-124: its error is
+        // at most rel_f*|r| < 2^-124.  Without such an atol the thread goes exact as elsewhere.)
+        const bool ext_look = BYDEF && ext && p.atol >= 4.70197740328915e-38f;
+        const bool bad = !(mrel <= 0.0f) || (!has_lean && mabs > p.atol) || ext_look;
+        bool trig = (mabs > th) || (ext && !ext_look);
         // Every vote below is reached by all 32 lanes: no warp-synchronous call sits under a
         // condition that could differ between lanes.
         if (!__any_sync(0xFFFFFFFFu, trig || bad)) continue;
@@ -642,17 +647,23 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
           for (int e = 0; e < kEPT; e += 2) {
             float d0, d1;
             E::pair_diff(words, e, r[e], r[e + 1], d0, d1);
-            const float ar0 = fabsf(r[e]), ar1 = fabsf(r[e + 1]);
-            const float t0 = fmaf(-rel, ar0, fabsf(d0)), t1 = fmaf(-rel, ar1, fabsf(d1));
+            float ar0 = fabsf(r[e]), ar1 = fabsf(r[e + 1]);
+            float a0 = fabsf(d0), a1 = fabsf(d1);
+            if constexpr (BYDEF) {   // magnitudes below 2^-64 and their errors times 2^64 (exact)
+              const float s0 = (ar0 > 0.0f && ar0 < 5.421010862427522e-20f) ? 18446744073709551616.0f : 1.0f;
+              const float s1 = (ar1 > 0.0f && ar1 < 5.421010862427522e-20f) ? 18446744073709551616.0f : 1.0f;
+              ar0 *= s0, a0 *= s0, ar1 *= s1, a1 *= s1;
+            }
+            const float t0 = fmaf(-rel, ar0, a0), t1 = fmaf(-rel, ar1, a1);
             // (a NaN or Inf difference makes t NaN or Inf: neither clause holds)
             // (by definition only: a zero reference has no quotient, its element only has to be
             // within atol.  In the other instantiations such an element goes to the exact path;
             // the clause is kept out of them because it changes how the compiler lays out their
             // main loop.)
             const bool c0 = (t0 <= 0.0f) || (t0 >= 7.888609052e-31f && fmaf(-g, ar0, t0) <= 0.0f) ||
-                            (BYDEF && ar0 == 0.0f && fabsf(d0) <= p.atol);
+                            (BYDEF && ar0 == 0.0f && a0 <= p.atol);
             const bool c1 = (t1 <= 0.0f) || (t1 >= 7.888609052e-31f && fmaf(-g, ar1, t1) <= 0.0f) ||
-                            (BYDEF && ar1 == 0.0f && fabsf(d1) <= p.atol);
+                            (BYDEF && ar1 == 0.0f && a1 <= p.atol);
             again |= !c0 || !c1;
           }
           }
@@ -671,9 +682,17 @@ __global__ void __maxnreg__(72) screen_stream_kernel(const StreamParams p) {
             const float tol1 = __fadd_rn(p.atol, __fmul_rn(p.rtol, fabsf(r[e + 1])));
             const bool f0 = a0 <= kFltMax, f1 = a1 <= kFltMax;
             again |= !f0 || !f1;
-            // (by definition only: a zero reference has no quotient)
-            again |= ((!BYDEF || fabsf(r[e]) > 0.0f) && !(fmaf(-rel, fabsf(r[e]), a0) <= 0.0f)) ||
-                     ((!BYDEF || fabsf(r[e + 1]) > 0.0f) && !(fmaf(-rel, fabsf(r[e + 1]), a1) <= 0.0f));
+            // (by definition only: a zero reference has no quotient; magnitudes below 2^-64 and
+            // their errors are scaled by 2^64, which is exact, so that the product cannot underflow)
+            if constexpr (BYDEF) {
+              const float q0 = fabsf(r[e]), q1 = fabsf(r[e + 1]);
+              const float s0 = q0 < 5.421010862427522e-20f ? 18446744073709551616.0f : 1.0f;
+              const float s1 = q1 < 5.421010862427522e-20f ? 18446744073709551616.0f : 1.0f;
+              again |= (q0 > 0.0f && !(fmaf(-rel, q0 * s0, a0 * s0) <= 0.0f)) ||
+                       (q1 > 0.0f && !(fmaf(-rel, q1 * s1, a1 * s1) <= 0.0f));
+            } else {
+              again |= !(fmaf(-rel, fabsf(r[e]), a0) <= 0.0f) || !(fmaf(-rel, fabsf(r[e + 1]), a1) <= 0.0f);
+            }
             mis_fast += ((a0 > tol0) && f0) ? 1u : 0u;   // (c == r would give a0 = 0 <= tol0)
             mis_fast += ((a1 > tol1) && f1) ? 1u : 0u;
           }
