@@ -89,6 +89,14 @@ def test_config2_full(ctx, kb):
         assert same_record(got[k], want[k]), (k, got[k], want[k])
         assert bool(got[k]["pass"]) == case.truth[k]["passes"]
     assert int(got["pass"].sum()) == 54
+    # the same batch through every instantiation of the streaming kernel, and in plain stream order
+    for mode, dependent in ((1, True), (2, True), (3, True), (1, False), (3, False)):
+        ctx.set_filter(mode)
+        ctx.set_dependent_launch(dependent)
+        again = kb.records(ctx.screen(case.ref, cands, case.atol, case.rtol))
+        assert again.tobytes() == got.tobytes(), (mode, dependent)
+    ctx.set_filter(0)
+    ctx.set_dependent_launch(True)
     med, omed = check_adjudicate(ctx, timings)
     surv, n = ctx.select(out, med, kb.KB_SELECT_ERR_THEN_TIME, 32)
     osurv, on = oracle.select(want, omed, 0, 32)
