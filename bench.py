@@ -240,10 +240,19 @@ def run_screen(args):
     g = torch.Generator(device=dev)
     g.manual_seed(20260802)
     base = torch.randn(N, dtype=torch.float32, device=dev, generator=g) * args.ref_scale
+    soft = None
+    if args.softmax_spread > 0.0:
+        # rows of 16384 logits of the given spread: outputs with a long tail of tiny values
+        soft = (torch.randn(N, dtype=torch.float32, device=dev, generator=g) * args.softmax_spread).view(-1, min(N, 16384))
+        base = torch.softmax(soft, dim=1).reshape(-1)
     ref = (torch.relu(base) if args.relu else base).to(tdt)   # (noise goes in before the rectifier)
     esz1 = ref.element_size() == 1           # 8-bit floats: one unit in the last place is up to 1/8
     cands = []
     for _ in range(K):
+        if soft is not None:
+            c = torch.softmax(soft + torch.randn(soft.shape, dtype=torch.float32, device=dev, generator=g) * 1e-4, dim=1)
+            cands.append(c.reshape(-1).to(tdt))
+            continue
         if args.noise_sigma > 0.0:
             # accumulated rounding error does not scale with the value: where the reference is near
             # zero the relative error is large and the element passes by atol alone
@@ -252,15 +261,17 @@ def run_screen(args):
             continue
         flip = torch.rand(N, device=dev, generator=g) < args.flip_frac
         cands.append(torch.where(flip, ref.view(idt) + 1, ref.view(idt)).view(tdt))
-    del base
+    del base, soft
     # tolerances under which a one-ulp difference passes: 2^-3 relative in e4m3, 2^-2 in e5m2
     atol, rtol = (1e-12, 1e-12) if args.dtype == "f64" else \
         (1e-2, 0.26 if args.dtype == "e5m2" else 0.13) if esz1 else (1e-2, 1.6e-2)
+    atol = args.atol if args.atol is not None else atol
+    rtol = args.rtol if args.rtol is not None else rtol
     held = cands if args.dtype == "f64" else binding.Candidates(cands)   # pointer array built once
     call = (lambda: ctx.screen_f64(ref, cands, atol, rtol)) if args.dtype == "f64" else \
         (lambda: ctx.screen(ref, held, atol, rtol))
     steps, warmup = max(1, min(args.steps, 50)), max(3, args.warmup)
-    if args.noise_sigma > 0.0:
+    if args.noise_sigma > 0.0 or args.softmax_spread > 0.0:
         warmup = max(warmup, 12)       # the context's choice of instantiation follows its reports
     for _ in range(warmup):
         call()
@@ -281,8 +292,10 @@ def run_screen(args):
     esz = ref.element_size()
     stream_bytes = (K + 1) * (ntiles - nscout) * 4096 * esz
     peak, src = peaks()
-    what = (f"absolute noise sigma={args.noise_sigma:g} on a reference of scale {args.ref_scale:g}"
-            + (", rectified" if args.relu else "")) if args.noise_sigma > 0.0 else \
+    what = f"softmax over rows of 16384 logits of spread {args.softmax_spread:g}, candidates from logits + N(0, 1e-8)" \
+        if args.softmax_spread > 0.0 else \
+        (f"absolute noise sigma={args.noise_sigma:g} on a reference of scale {args.ref_scale:g}"
+         + (", rectified" if args.relu else "")) if args.noise_sigma > 0.0 else \
         f"one-ulp differences on {args.flip_frac:.0%} of the elements"
     line = {"workload": f"screen K={K} N=2^{args.log2n} {args.dtype}, {what}",
             "filter": {0: "plain", 1: "sharp", 3: "by definition"}.get(ctx.last_filter_mode, "-"),
@@ -417,6 +430,10 @@ def main():
     ap.add_argument("--noise-sigma", type=float, default=0.0,
                     help="'screen' workload: candidates = round(reference + N(0, sigma^2)) instead of one-ulp differences")
     ap.add_argument("--ref-scale", type=float, default=1.0, help="'screen' workload: standard deviation of the reference")
+    ap.add_argument("--atol", type=float, default=None, help="'screen' workload: tolerance override")
+    ap.add_argument("--rtol", type=float, default=None, help="'screen' workload: tolerance override")
+    ap.add_argument("--softmax-spread", type=float, default=0.0,
+                    help="'screen' workload: reference = softmax over rows of 16384 logits N(0, spread^2)")
     ap.add_argument("--relu", action="store_true", help="'screen' workload: rectified reference and candidates")
     ap.add_argument("--default-dispatch", action="store_true",
                     help="'screen' workload: let small problems take the single-launch kernel")
