@@ -148,6 +148,54 @@ def test_random_large(ctx, kb, block):
         one_case(ctx, kb, 9_000_000 + block * 1000 + i, 20, 24)
 
 
+@pytest.mark.parametrize("block", range(4))
+def test_random_tiny_magnitudes(ctx, kb, block):
+    """References and candidates whose magnitudes go from ordinary down through 2^-100, the
+    smallest normals and the subnormals to zero, under tolerances from nothing to generous, through
+    the plain, the sharp and the by-definition instantiation: where products underflow and
+    quotients are undefined is where a filter would go wrong first."""
+    rng = np.random.default_rng(31_000 + block)
+    dev = torch.device("cuda", 0)
+    ctx.set_small_path(False)
+    try:
+        for _ in range(25):
+            code = int(rng.choice([synth.F32, synth.BF16]))
+            tdt = synth.TORCH_DTYPE[code]
+            N = int(rng.integers(3, 40)) * 4096 + int(rng.integers(0, 4096))
+            K = int(rng.choice([1, 3, 8]))
+            e = rng.choice([0, -60, -90, -105, -115, -124, -130, -140, -149], size=N,
+                           p=[.4, .05, .05, .1, .1, .1, .1, .05, .05])
+            x = rng.standard_normal(N) * np.exp2(e.astype(np.float64))
+            x[rng.random(N) < 0.05] = 0.0
+            ref = torch.from_numpy(x).to(torch.float32).to(tdt)
+            cands = []
+            for _k in range(K):
+                kind = int(rng.integers(0, 4))
+                if kind == 0:
+                    c = torch.from_numpy(x * (1 + rng.standard_normal(N) * 1e-3)).to(torch.float32).to(tdt)
+                elif kind == 1:
+                    step = torch.from_numpy(rng.integers(-2, 3, N) * (rng.random(N) < 0.3)).to(torch.int64)
+                    c = synth.ulp_step(ref, code, step)
+                elif kind == 2:
+                    c = torch.where(torch.from_numpy(rng.random(N) < 0.2), torch.zeros_like(ref), ref)
+                else:
+                    c = torch.where(torch.from_numpy(rng.random(N) < 0.2), ref * 2, ref)
+                cands.append(c.contiguous())
+            atol = float(rng.choice([0.0, 1e-45, 1e-38, 1e-30, 1e-6]))
+            rtol = float(rng.choice([0.0, 1e-7, 1e-3, 1.6e-2, 0.5]))
+            want = oracle.screen(synth.to_oracle_array(ref, code), [synth.to_oracle_array(c, code) for c in cands],
+                                 code, atol, rtol, threads=8)
+            d_ref, d_cands = ref.to(dev), [c.to(dev) for c in cands]
+            for mode in (3, 1, 2):
+                ctx.set_filter(mode)
+                got = kb.records(ctx.screen(d_ref, d_cands, atol, rtol))
+                assert not same(got, want), f"mode={mode} dtype={code} N={N} K={K} tol=({atol},{rtol})"
+    finally:
+        ctx.set_filter(0)
+        ctx.set_small_path(True)
+    assert ctx.poll() == 0
+
+
 def fbits(a):
     return np.ascontiguousarray(a, dtype=np.float32).view(np.uint32)
 
