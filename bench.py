@@ -545,6 +545,7 @@ def main():
     sampler.window = (t_begin, time.perf_counter())
     elapsed_ms = e0.elapsed_time(e1)
     launches = ctx.launch_count + ctx_adj.launch_count - launches0
+    filter_used = {0: "plain", 1: "sharp", 3: "by definition"}.get(ctx.last_filter_mode, "?")
     stream_ms = ctx.read_timer(binding.KB_TIMER_SCREEN_STREAM)
     ctx.enable_timing(False)
     # the win-count kernel's own duration (a secondary figure): five more steps, untimed and
@@ -671,6 +672,7 @@ def main():
                 "traffic_source": os.path.relpath(TRAFFIC_FILE, ROOT) if traffic else None,
                 "kernel": "screen_stream_kernel<bf16>", "launch_ms_avg": avg_stream_ms,
                 "launch_ms_min": float(np.min(stream_ms)) if len(stream_ms) else None,
+                "instantiation": filter_used,
                 "algorithmic_bytes_per_launch": stream_bytes, "launches_timed": int(len(stream_ms)),
                 "timed": f"every {TIMED_EVERY}th launch of the timed region",
                 "share_of_step": avg_stream_ms / ms_per_step}
