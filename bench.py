@@ -548,11 +548,14 @@ def main():
     filter_used = {0: "plain", 1: "sharp", 3: "by definition"}.get(ctx.last_filter_mode, "?")
     stream_ms = ctx.read_timer(binding.KB_TIMER_SCREEN_STREAM)
     ctx.enable_timing(False)
-    # the win-count kernel's own duration (a secondary figure): five more steps, untimed and
-    # uncounted, with its event pair on
+    # the win-count kernel's own duration (a secondary figure): ten adjudications by themselves,
+    # untimed and uncounted, with its event pair on (inside the step the kernel shares the GPU
+    # with the resident streaming CTAs, and an event pair around it would measure its wait)
+    torch.cuda.synchronize()
     ctx_adj.enable_timing(True)
-    for _ in range(5):
-        step()
+    with torch.cuda.stream(side):
+        for _ in range(10):
+            ctx_adj.adjudicate(d_timings)
     torch.cuda.synchronize()
     wins_ms = ctx_adj.read_timer(binding.KB_TIMER_WINS)
     ctx_adj.enable_timing(False)
