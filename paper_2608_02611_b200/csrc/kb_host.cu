@@ -37,10 +37,12 @@ struct kb_ctx {
   int ws_parity = 0;
   uint32_t used_K[2] = {0, 0};
   bool ws_dirty = true;
-  // Choice between the two instantiations of the streaming kernel.  The plain one reports, in a
-  // host-visible word, the share of its warp steps that took a fruitless second look; when the
-  // last report says a quarter or more, the next calls use the sharp instantiation, and every
-  // so often one of them probes the plain one again.  filter_mode: 0 automatic, 1 plain, 2 sharp.
+  // Choice between the instantiations of the streaming kernel.  The plain one reports, in a
+  // host-visible word, the share of its warp steps that took a fruitless second look: one byte
+  // for looks taken while the candidate was lean, one for looks (and exact paths) beyond the lean
+  // bound that changed nothing.  When the last report says a quarter or more, the next calls use
+  // the sharp instantiation (first byte) or the by-definition one (second byte), and every so
+  // often one of them probes the plain one again.
   unsigned int* h_hint = nullptr;   // pinned, mapped
   unsigned int* d_hint = nullptr;   // its device address
   int filter_mode = 0;              // 0 automatic, 1 plain, 2 sharp, 3 by definition
